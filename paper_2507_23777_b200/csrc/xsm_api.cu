@@ -1,0 +1,592 @@
+// Host side of the C ABI declared in include/xsm.h: argument checks, workspace layout, phase tables,
+// launches.  No device memory is allocated here; everything lives in the caller's workspace.
+#include "../../include/xsm.h"
+#include "xsm_internal.h"
+
+#include <limits.h>
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+using namespace xsm;
+
+namespace {
+
+constexpr int kSizingGrid = 256;      // CTA count assumed when sizing split-partial buffers
+constexpr int kKvStagePositions = 256;
+constexpr int kChunkSteps = 64;       // decoding steps per persistent-kernel launch in xsm_generate
+
+thread_local std::string g_create_error;
+
+struct Layout {
+    size_t total = 0;
+    size_t phases, jobs, inv_freq, wkc_off, wvc_off;
+    size_t len, window, cand, acc_len, finished, n_gen, n_blocks, ingest_left, step_idx, block_table, free_stack,
+        scalars, hist, steps, tok_log, step_tokens, step_n_new, prompt;
+    size_t h, qkv, attn, qc, cattn, act, y, logits0, hlogits, rope_cs, part, cpart, part_ctr, cpart_ctr;
+    size_t stage_cond, stage_kv, stage_tok, ckv_pool, kv_pool;
+    int n_pages = 0, max_blocks = 0, cpages = 0, tok_ld = 0, n_phases = 0, n_jobs = 0;
+    size_t page_bytes = 0;
+};
+
+size_t esize(const xsm_model_config &c) { return c.dtype == 1 ? 2 : 4; }
+
+size_t take(size_t &cur, size_t bytes) {
+    size_t o = cur;
+    cur = (cur + bytes + 255) / 256 * 256;
+    return o;
+}
+
+// workspace_bytes == 0: size the pool for max_batch full sequences
+bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
+    const size_t B = c.max_batch, K1 = c.n_draft + 1, M = B * K1, d = c.d_model, V = c.vocab, f = c.d_ff;
+    const size_t P = c.page_size, H = c.n_heads, dh = c.d_head;
+    L.max_blocks = (int)((c.max_seq_len + K1 + P - 1) / P);
+    L.cpages = (int)((c.n_cond + P - 1) / P);
+    L.tok_ld = c.max_seq_len + (int)K1;
+    L.n_phases = c.n_layers * 8 + 3 + (c.n_draft > 0 ? 1 : 0);
+    L.n_jobs = c.n_layers * 6 + 1 + 2 * c.n_draft;
+    size_t cur = 0;
+    L.phases = take(cur, sizeof(Phase) * L.n_phases);
+    L.jobs = take(cur, sizeof(GemvJob) * L.n_jobs);
+    L.inv_freq = take(cur, sizeof(double) * (dh / 2 + 1));
+    L.wkc_off = take(cur, sizeof(size_t) * c.n_layers);
+    L.wvc_off = take(cur, sizeof(size_t) * c.n_layers);
+    L.len = take(cur, 4 * B);
+    L.window = take(cur, 4 * M);
+    L.cand = take(cur, 4 * M);
+    L.acc_len = take(cur, 4 * B);
+    L.finished = take(cur, 4 * B);
+    L.n_gen = take(cur, 4 * B);
+    L.n_blocks = take(cur, 4 * B);
+    L.ingest_left = take(cur, 4 * B);
+    L.step_idx = take(cur, 4 * B);
+    L.block_table = take(cur, 4 * B * L.max_blocks);
+    L.scalars = take(cur, 256);   // n_free, n_active, status, bar
+    L.hist = take(cur, 8 * B * (kMaxDraft + 1));
+    L.steps = take(cur, 8 * B);
+    L.tok_log = take(cur, 4 * B * L.tok_ld);
+    L.step_tokens = take(cur, 4 * M);
+    L.step_n_new = take(cur, 4 * B);
+    L.prompt = take(cur, 4 * B * (c.max_seq_len + 1));
+    L.h = take(cur, 4 * M * d);
+    L.qkv = take(cur, 4 * M * 3 * d);
+    L.attn = take(cur, 4 * M * d);
+    L.qc = take(cur, 4 * M * d);
+    L.cattn = take(cur, 4 * M * d);
+    L.act = take(cur, 4 * M * f);
+    L.y = take(cur, 4 * M * d * (c.n_draft > 0 ? c.n_draft : 1));
+    L.logits0 = take(cur, 4 * M * V);
+    L.hlogits = take(cur, 4 * M * V * (c.n_draft > 0 ? c.n_draft : 1));
+    L.rope_cs = take(cur, 8 * M * (dh / 2));
+    const size_t part_items = B * H + 2 * kSizingGrid;
+    L.part = take(cur, 4 * part_items * K1 * (dh + 2));
+    L.cpart = take(cur, 4 * part_items * K1 * (dh + 2));
+    L.part_ctr = take(cur, 4 * B * H);
+    L.cpart_ctr = take(cur, 4 * B * H);
+    L.stage_cond = take(cur, esize(c) * B * c.n_cond * c.d_cond);
+    L.stage_kv = take(cur, 4 * 2 * (size_t)kKvStagePositions * d);
+    L.stage_tok = take(cur, 4 * B * (c.max_seq_len + 1));
+    L.ckv_pool = take(cur, esize(c) * (size_t)c.n_layers * 2 * B * L.cpages * H * P * dh);
+    L.page_bytes = esize(c) * (size_t)c.n_layers * 2 * H * P * dh;
+    // the rest is the shared page pool, preceded by its free stack (4 bytes per page)
+    if (workspace_bytes == 0) {
+        L.n_pages = (int)(B * L.max_blocks);
+    } else {
+        if (workspace_bytes < cur + 512) return false;
+        size_t n = (workspace_bytes - cur - 512) / (L.page_bytes + 4);
+        if (n > (size_t)INT_MAX / 2) n = INT_MAX / 2;
+        if (n < (size_t)L.max_blocks) return false;
+        L.n_pages = (int)n;
+    }
+    L.free_stack = take(cur, 4 * (size_t)L.n_pages);
+    L.kv_pool = cur;
+    L.total = cur + L.page_bytes * L.n_pages;
+    return true;
+}
+
+const char *check_config(const xsm_model_config &c) {
+    if (c.n_layers < 1 || c.d_model < 32 || c.n_heads < 1 || c.d_head < 2 || c.d_ff < 32 || c.vocab < 2 ||
+        c.n_cond < 1 || c.d_cond < 32 || c.max_batch < 1 || c.max_seq_len < 1)
+        return "a model dimension is out of range";
+    if (c.n_heads * c.d_head != c.d_model) return "n_heads * d_head must equal d_model";
+    if (c.d_model % 32 || c.d_ff % 32 || c.d_cond % 32) return "d_model, d_ff and d_cond must be multiples of 32";
+    if ((c.d_head & 1) || c.d_head > 128) return "d_head must be even and at most 128";
+    if (c.n_draft < 0 || c.n_draft > XSM_MAX_DRAFT) return "n_draft must be in [0, 16]";
+    if (c.head_hidden != c.d_model) return "head_hidden must equal d_model (the head block is residual)";
+    if (c.head_kind != 0) return "only MLP heads (head_kind 0) are implemented";
+    if (c.dtype != 0 && c.dtype != 1) return "dtype must be 0 (fp32) or 1 (bf16)";
+    if (c.page_size < 16 || c.page_size % 16) return "page_size must be a positive multiple of 16";
+    if ((long long)c.max_batch * (c.n_draft + 1) > kMaxTokens) return "max_batch * (n_draft + 1) exceeds 512";
+    if (c.vocab > (1 << 20)) return "vocab too large";
+    if (!(c.rope_theta > 1.0f) || !(c.rms_eps > 0.0f)) return "rope_theta must be > 1 and rms_eps > 0";
+    if (c.bos_id < 0 || c.bos_id >= c.vocab || c.eos_id >= c.vocab) return "bos_id / eos_id out of range";
+    return nullptr;
+}
+
+struct WeightOffsets {
+    size_t E, gf, W0;
+    std::vector<size_t> g1, wq, wo, g2, wqc, wkc, wvc, woc, g3, wgate, wup, wdown, W1, Wout;
+    size_t total;
+};
+
+WeightOffsets weight_offsets(const xsm_model_config &c) {
+    WeightOffsets w;
+    const size_t d = c.d_model, f = c.d_ff, V = c.vocab, dc = c.d_cond, hd = c.head_hidden;
+    size_t o = 0;
+    w.E = o; o += V * d;
+    for (int l = 0; l < c.n_layers; ++l) {
+        w.g1.push_back(o); o += d;
+        w.wq.push_back(o); o += 3 * d * d;      // Wq, Wk, Wv are consecutive
+        w.wo.push_back(o); o += d * d;
+        w.g2.push_back(o); o += d;
+        w.wqc.push_back(o); o += d * d;
+        w.wkc.push_back(o); o += d * dc;
+        w.wvc.push_back(o); o += d * dc;
+        w.woc.push_back(o); o += d * d;
+        w.g3.push_back(o); o += d;
+        w.wgate.push_back(o); o += f * d;
+        w.wup.push_back(o); o += f * d;
+        w.wdown.push_back(o); o += d * f;
+    }
+    w.gf = o; o += d;
+    w.W0 = o; o += V * d;
+    for (int i = 0; i < c.n_draft; ++i) {
+        w.W1.push_back(o); o += hd * d;
+        w.Wout.push_back(o); o += V * hd;
+    }
+    w.total = o;
+    return w;
+}
+
+}  // namespace
+
+struct xsm_ctx {
+    xsm_model_config cfg;
+    xsm_decode_config dc;
+    Layout lay;
+    WeightOffsets wo;
+    const char *weights;
+    char *ws;
+    size_t ws_bytes;
+    cudaStream_t stream;
+    Dev dev;
+    int grid, phase_launch, prefilled, batch;
+    uint64_t launches;
+    std::string err;
+    std::vector<Phase> h_phases;
+    std::vector<GemvJob> h_jobs;
+    int *pinned;              // [4] n_active, status
+    cudaEvent_t ev0, ev1;
+    double last_wall_ms;
+};
+
+namespace {
+
+xsm_status fail(xsm_ctx *ctx, xsm_status st, const std::string &msg) {
+    if (ctx) ctx->err = msg; else g_create_error = msg;
+    return st;
+}
+xsm_status cuda_fail(xsm_ctx *ctx, cudaError_t e, const char *what) {
+    return fail(ctx, XSM_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+#define XSM_CUDA(ctx, call)                                             \
+    do {                                                                \
+        cudaError_t e_ = (call);                                        \
+        if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call);        \
+    } while (0)
+
+template <typename T> T *at(xsm_ctx *ctx, size_t off) { return reinterpret_cast<T *>(ctx->ws + off); }
+const void *wptr(const xsm_ctx *ctx, size_t elem_off) { return ctx->weights + elem_off * esize(ctx->cfg); }
+
+// phase and job tables for the current batch
+void build_tables(xsm_ctx *ctx) {
+    const xsm_model_config &c = ctx->cfg;
+    const Dev &D = ctx->dev;
+    const WeightOffsets &w = ctx->wo;
+    const int d = c.d_model, f = c.d_ff, V = c.vocab, K = c.n_draft;
+    const size_t M = D.M;
+    ctx->h_phases.clear();
+    ctx->h_jobs.clear();
+    auto job = [&](const void *W, const void *W2, int rows, int kdim, const float *x, const void *gain, float *out,
+                   int out_ld, int epi) {
+        GemvJob j;
+        j.W = W; j.W2 = W2; j.x = x; j.gain = gain; j.out = out;
+        j.rows = rows; j.kdim = kdim; j.x_ld = kdim; j.out_ld = out_ld; j.epi = epi; j.pad = 0;
+        ctx->h_jobs.push_back(j);
+        return (int)ctx->h_jobs.size() - 1;
+    };
+    auto gemv1 = [&](int layer, int j0, int n) { ctx->h_phases.push_back(Phase{PH_GEMV, layer, j0, n}); };
+    for (int l = 0; l < c.n_layers; ++l) {
+        gemv1(l, job(wptr(ctx, w.wq[l]), nullptr, 3 * d, d, D.h, wptr(ctx, w.g1[l]), D.qkv, 3 * d, EPI_STORE), 1);
+        ctx->h_phases.push_back(Phase{PH_ATTN_SELF, l, 0, 0});
+        gemv1(l, job(wptr(ctx, w.wo[l]), nullptr, d, d, D.attn, nullptr, D.h, d, EPI_ADD), 1);
+        gemv1(l, job(wptr(ctx, w.wqc[l]), nullptr, d, d, D.h, wptr(ctx, w.g2[l]), D.qc, d, EPI_STORE), 1);
+        ctx->h_phases.push_back(Phase{PH_ATTN_CROSS, l, 0, 0});
+        gemv1(l, job(wptr(ctx, w.woc[l]), nullptr, d, d, D.cattn, nullptr, D.h, d, EPI_ADD), 1);
+        gemv1(l, job(wptr(ctx, w.wgate[l]), wptr(ctx, w.wup[l]), f, d, D.h, wptr(ctx, w.g3[l]), D.act, f, EPI_GATEUP), 1);
+        gemv1(l, job(wptr(ctx, w.wdown[l]), nullptr, d, f, D.act, nullptr, D.h, d, EPI_ADD), 1);
+    }
+    int j0 = job(wptr(ctx, w.W0), nullptr, V, d, D.h, wptr(ctx, w.gf), D.logits0, V, EPI_STORE);
+    for (int i = 0; i < K; ++i)
+        job(wptr(ctx, w.W1[i]), nullptr, d, d, D.h, wptr(ctx, w.gf), D.y + (size_t)i * M * d, d, EPI_HEADY);
+    gemv1(-1, j0, 1 + K);
+    if (K > 0) {
+        j0 = (int)ctx->h_jobs.size();
+        for (int i = 0; i < K; ++i)
+            job(wptr(ctx, w.Wout[i]), nullptr, V, d, D.y + (size_t)i * M * d, nullptr, D.hlogits + (size_t)i * M * V, V,
+                EPI_STORE);
+        gemv1(-1, j0, K);
+    }
+    ctx->h_phases.push_back(Phase{PH_SAMPLE, -1, 0, 0});
+    ctx->h_phases.push_back(Phase{PH_COMMIT, -1, 0, 0});
+}
+
+xsm_status check_device_status(xsm_ctx *ctx) {
+    XSM_CUDA(ctx, cudaMemcpyAsync(ctx->pinned, ctx->dev.n_active, 8, cudaMemcpyDeviceToHost, ctx->stream));
+    XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    const int st = ctx->pinned[1];
+    if (st == XSM_ERR_TIMEOUT) return fail(ctx, XSM_ERR_TIMEOUT, "a grid barrier wait ran out of patience");
+    if (st == XSM_ERR_CAPACITY) return fail(ctx, XSM_ERR_CAPACITY, "the page pool ran dry during decoding");
+    if (st != 0) return fail(ctx, XSM_ERR_CUDA, "device status word is set");
+    return XSM_OK;
+}
+
+// n_steps decoding steps on the stream
+xsm_status run_steps(xsm_ctx *ctx, int n_steps) {
+    const int np = (int)ctx->h_phases.size();
+    if (!ctx->phase_launch) {
+        XSM_CUDA(ctx, launch_step(ctx->dev, ctx->cfg.dtype, 0, np, n_steps, 1, ctx->grid, ctx->stream));
+        ctx->launches += 1;
+    } else {
+        for (int t = 0; t < n_steps; ++t)
+            for (int p = 0; p < np; ++p) {
+                XSM_CUDA(ctx, launch_step(ctx->dev, ctx->cfg.dtype, p, p + 1, 1, 0, ctx->grid, ctx->stream));
+                ctx->launches += 1;
+            }
+    }
+    return XSM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t xsm_weights_bytes(const xsm_model_config *cfg) {
+    if (!cfg || check_config(*cfg)) return 0;
+    return weight_offsets(*cfg).total * esize(*cfg);
+}
+
+size_t xsm_workspace_bytes(const xsm_model_config *cfg) {
+    if (!cfg || check_config(*cfg)) return 0;
+    Layout L;
+    make_layout(*cfg, 0, L);
+    return L.total;
+}
+
+xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *d_workspace, size_t workspace_bytes,
+                      void *cuda_stream, xsm_ctx **out) {
+    if (!cfg || !d_weights || !d_workspace || !out) return fail(nullptr, XSM_ERR_INVALID_ARG, "null argument");
+    if (const char *m = check_config(*cfg)) return fail(nullptr, XSM_ERR_INVALID_ARG, m);
+    if (((uintptr_t)d_weights & 255) || ((uintptr_t)d_workspace & 255))
+        return fail(nullptr, XSM_ERR_INVALID_ARG, "weights and workspace must be 256-byte aligned");
+    Layout L;
+    if (!make_layout(*cfg, workspace_bytes, L))
+        return fail(nullptr, XSM_ERR_CAPACITY, "workspace cannot hold the buffers plus one sequence of cache pages");
+    xsm_ctx *ctx = new xsm_ctx();
+    ctx->cfg = *cfg;
+    ctx->lay = L;
+    ctx->wo = weight_offsets(*cfg);
+    ctx->weights = (const char *)d_weights;
+    ctx->ws = (char *)d_workspace;
+    ctx->ws_bytes = workspace_bytes;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    ctx->phase_launch = 0; ctx->prefilled = 0; ctx->batch = 0; ctx->launches = 0; ctx->last_wall_ms = 0;
+    ctx->pinned = nullptr; ctx->ev0 = ctx->ev1 = nullptr;
+    auto bail = [&](cudaError_t e, const char *what) {
+        g_create_error = std::string(what) + ": " + cudaGetErrorString(e);
+        if (ctx->pinned) cudaFreeHost(ctx->pinned);
+        if (ctx->ev0) cudaEventDestroy(ctx->ev0);
+        if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+        delete ctx;
+        return XSM_ERR_CUDA;
+    };
+    cudaError_t e;
+    int grid = 0;
+    if ((e = step_kernel_setup(cfg->dtype, &grid)) != cudaSuccess) return bail(e, "step kernel setup");
+    if (grid < 1) { delete ctx; return fail(nullptr, XSM_ERR_CUDA, "the step kernel does not fit on this device"); }
+    ctx->grid = grid;
+    if ((e = cudaHostAlloc((void **)&ctx->pinned, 64, cudaHostAllocDefault)) != cudaSuccess) return bail(e, "cudaHostAlloc");
+    if ((e = cudaEventCreate(&ctx->ev0)) != cudaSuccess) return bail(e, "cudaEventCreate");
+    if ((e = cudaEventCreate(&ctx->ev1)) != cudaSuccess) return bail(e, "cudaEventCreate");
+
+    // constant tables
+    std::vector<double> inv_freq(cfg->d_head / 2 + 1);
+    for (int i = 0; i < cfg->d_head / 2; ++i) inv_freq[i] = pow((double)cfg->rope_theta, -2.0 * i / cfg->d_head);
+    if ((e = cudaMemcpyAsync(ctx->ws + L.inv_freq, inv_freq.data(), sizeof(double) * (cfg->d_head / 2),
+                             cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) return bail(e, "upload");
+    if ((e = cudaMemcpyAsync(ctx->ws + L.wkc_off, ctx->wo.wkc.data(), sizeof(size_t) * cfg->n_layers,
+                             cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) return bail(e, "upload");
+    if ((e = cudaMemcpyAsync(ctx->ws + L.wvc_off, ctx->wo.wvc.data(), sizeof(size_t) * cfg->n_layers,
+                             cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) return bail(e, "upload");
+    if ((e = cudaStreamSynchronize(ctx->stream)) != cudaSuccess) return bail(e, "sync");
+
+    Dev &D = ctx->dev;
+    memset(&D, 0, sizeof(D));
+    D.L = cfg->n_layers; D.d = cfg->d_model; D.H = cfg->n_heads; D.dh = cfg->d_head; D.f = cfg->d_ff;
+    D.V = cfg->vocab; D.C = cfg->n_cond; D.dc = cfg->d_cond; D.K = cfg->n_draft; D.K1 = cfg->n_draft + 1;
+    D.P = cfg->page_size; D.max_blocks = L.max_blocks; D.n_pages = L.n_pages; D.cpages = L.cpages;
+    D.max_seq_len = cfg->max_seq_len; D.tok_ld = L.tok_ld;
+    D.eps = cfg->rms_eps; D.scale = (float)(1.0 / sqrt((double)cfg->d_head)); D.bos = cfg->bos_id; D.eos = cfg->eos_id;
+    D.max_new = INT_MAX;
+    D.phases = at<Phase>(ctx, L.phases); D.jobs = at<GemvJob>(ctx, L.jobs);
+    D.E = wptr(ctx, ctx->wo.E); D.inv_freq = at<double>(ctx, L.inv_freq);
+    D.len = at<int>(ctx, L.len); D.window = at<int>(ctx, L.window); D.cand = at<int>(ctx, L.cand);
+    D.acc_len = at<int>(ctx, L.acc_len); D.finished = at<int>(ctx, L.finished); D.n_gen = at<int>(ctx, L.n_gen);
+    D.n_blocks = at<int>(ctx, L.n_blocks); D.block_table = at<int>(ctx, L.block_table);
+    D.ingest_left = at<int>(ctx, L.ingest_left); D.step_idx = at<uint32_t>(ctx, L.step_idx);
+    D.free_stack = at<int>(ctx, L.free_stack);
+    int *sc = at<int>(ctx, L.scalars);
+    D.n_active = sc; D.status = sc + 1; D.n_free = sc + 2; D.bar = reinterpret_cast<unsigned *>(sc + 16);
+    D.hist = at<unsigned long long>(ctx, L.hist); D.steps = at<unsigned long long>(ctx, L.steps);
+    D.tok_log = at<int>(ctx, L.tok_log); D.step_tokens = at<int>(ctx, L.step_tokens);
+    D.step_n_new = at<int>(ctx, L.step_n_new); D.prompt = at<int>(ctx, L.prompt);
+    D.h = at<float>(ctx, L.h); D.qkv = at<float>(ctx, L.qkv); D.attn = at<float>(ctx, L.attn);
+    D.qc = at<float>(ctx, L.qc); D.cattn = at<float>(ctx, L.cattn); D.act = at<float>(ctx, L.act);
+    D.y = at<float>(ctx, L.y); D.logits0 = at<float>(ctx, L.logits0); D.hlogits = at<float>(ctx, L.hlogits);
+    D.rope_cs = at<float2>(ctx, L.rope_cs); D.part = at<float>(ctx, L.part); D.cpart = at<float>(ctx, L.cpart);
+    D.part_ctr = at<unsigned>(ctx, L.part_ctr); D.cpart_ctr = at<unsigned>(ctx, L.cpart_ctr);
+    D.kv_pool = ctx->ws + L.kv_pool; D.ckv_pool = ctx->ws + L.ckv_pool;
+    *out = ctx;
+    return XSM_OK;
+}
+
+xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_t *d_prompt, int prompt_len,
+                       const xsm_decode_config *dc) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    if (!d_cond || !d_prompt || !dc) return fail(ctx, XSM_ERR_INVALID_ARG, "null argument");
+    const xsm_model_config &c = ctx->cfg;
+    if (batch < 1 || batch > c.max_batch) return fail(ctx, XSM_ERR_INVALID_ARG, "batch must be in [1, max_batch]");
+    if (prompt_len < 1 || prompt_len - 1 > c.max_seq_len) return fail(ctx, XSM_ERR_INVALID_ARG, "prompt_len out of range");
+    if (dc->verify_mode < 0 || dc->verify_mode > 2 || dc->sample_mode < 0 || dc->sample_mode > 1)
+        return fail(ctx, XSM_ERR_INVALID_ARG, "unknown verify_mode or sample_mode");
+    if (dc->verify_mode == 1 && dc->k_accept < 1) return fail(ctx, XSM_ERR_INVALID_ARG, "k_accept must be >= 1");
+    if (dc->sample_mode == 1 && (dc->k_sample < 1 || dc->k_sample > 64 || !(dc->temperature > 0.f)))
+        return fail(ctx, XSM_ERR_INVALID_ARG, "k_sample must be in [1, 64] and temperature > 0");
+    if ((long long)batch * ctx->lay.max_blocks > ctx->lay.n_pages)
+        return fail(ctx, XSM_ERR_CAPACITY, "the page pool cannot hold `batch` sequences of max_seq_len positions");
+    ctx->dc = *dc;
+    ctx->batch = batch;
+    Dev &D = ctx->dev;
+    D.B = batch; D.M = batch * D.K1;
+    D.verify_mode = dc->verify_mode; D.k_accept = dc->k_accept; D.delta = dc->delta;
+    D.sample_mode = dc->sample_mode; D.k_sample = dc->k_sample; D.temperature = dc->temperature;
+    D.key0 = (uint32_t)dc->seed; D.key1 = (uint32_t)(dc->seed >> 32);
+    D.max_new = INT_MAX; D.prompt_len = prompt_len;
+    const int bh = batch * D.H;
+    int s_self = (2 * ctx->grid) / bh;
+    D.S_self = s_self < 1 ? 1 : (s_self > 64 ? 64 : s_self);
+    int s_cross = ctx->grid / bh;
+    if (s_cross > D.cpages) s_cross = D.cpages;
+    D.S_cross = s_cross < 1 ? 1 : s_cross;
+    build_tables(ctx);
+    D.n_phases = (int)ctx->h_phases.size();
+    if ((int)ctx->h_phases.size() > ctx->lay.n_phases || (int)ctx->h_jobs.size() > ctx->lay.n_jobs)
+        return fail(ctx, XSM_ERR_STATE, "internal: phase table overflow");
+    XSM_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->lay.phases, ctx->h_phases.data(), sizeof(Phase) * ctx->h_phases.size(),
+                                  cudaMemcpyHostToDevice, ctx->stream));
+    XSM_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->lay.jobs, ctx->h_jobs.data(), sizeof(GemvJob) * ctx->h_jobs.size(),
+                                  cudaMemcpyHostToDevice, ctx->stream));
+    if ((const void *)d_prompt != (const void *)D.prompt)
+        XSM_CUDA(ctx, cudaMemcpyAsync((void *)D.prompt, d_prompt, sizeof(int32_t) * batch * prompt_len,
+                                      cudaMemcpyDeviceToDevice, ctx->stream));
+    // the tables above are read from host vectors that may be rebuilt by the next prefill
+    XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    XSM_CUDA(ctx, launch_cross_kv(D, c.dtype, ctx->weights, at<size_t>(ctx, ctx->lay.wkc_off),
+                                  at<size_t>(ctx, ctx->lay.wvc_off), d_cond, ctx->stream));
+    XSM_CUDA(ctx, launch_init(D, c.dtype, ctx->stream));
+    ctx->launches += 3;
+    ctx->prefilled = 1;
+    const int ingest_steps = (prompt_len - 1 + D.K1 - 1) / D.K1;
+    if (ingest_steps > 0) {
+        xsm_status st = run_steps(ctx, ingest_steps);
+        if (st != XSM_OK) return st;
+    }
+    return XSM_OK;
+}
+
+xsm_status xsm_spec_step(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_n_new) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "xsm_spec_step before xsm_prefill");
+    ctx->dev.max_new = INT_MAX;
+    xsm_status st = run_steps(ctx, 1);
+    if (st != XSM_OK) return st;
+    const Dev &D = ctx->dev;
+    if (d_new_tokens)
+        XSM_CUDA(ctx, cudaMemcpyAsync(d_new_tokens, D.step_tokens, sizeof(int32_t) * D.M, cudaMemcpyDeviceToDevice, ctx->stream));
+    if (d_n_new)
+        XSM_CUDA(ctx, cudaMemcpyAsync(d_n_new, D.step_n_new, sizeof(int32_t) * D.B, cudaMemcpyDeviceToDevice, ctx->stream));
+    return XSM_OK;
+}
+
+xsm_status xsm_generate(xsm_ctx *ctx, int max_new_tokens, int32_t *d_tokens, int32_t *d_lengths, xsm_stats *host_stats) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "xsm_generate before xsm_prefill");
+    if (max_new_tokens < 1 || max_new_tokens > ctx->cfg.max_seq_len)
+        return fail(ctx, XSM_ERR_INVALID_ARG, "max_new_tokens must be in [1, max_seq_len]");
+    Dev &D = ctx->dev;
+    D.max_new = max_new_tokens;
+    XSM_CUDA(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
+    long long budget = (long long)max_new_tokens + 2;   // every step commits at least one token per live sequence
+    while (budget > 0) {
+        const int n = (int)(budget < kChunkSteps ? budget : kChunkSteps);
+        xsm_status st = run_steps(ctx, n);
+        if (st != XSM_OK) return st;
+        budget -= n;
+        st = check_device_status(ctx);
+        if (st != XSM_OK) return st;
+        if (ctx->pinned[0] <= 0) break;
+    }
+    XSM_CUDA(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
+    if (d_tokens || d_lengths) {
+        XSM_CUDA(ctx, launch_export(D, max_new_tokens, d_tokens, d_lengths, ctx->stream));
+        ctx->launches += 1;
+    }
+    XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    float ms = 0.f;
+    XSM_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
+    ctx->last_wall_ms = ms;
+    if (host_stats) {
+        std::vector<unsigned long long> hist((size_t)D.B * (kMaxDraft + 1)), steps(D.B);
+        std::vector<int> ngen(D.B);
+        XSM_CUDA(ctx, cudaMemcpy(hist.data(), D.hist, 8 * hist.size(), cudaMemcpyDeviceToHost));
+        XSM_CUDA(ctx, cudaMemcpy(steps.data(), D.steps, 8 * steps.size(), cudaMemcpyDeviceToHost));
+        XSM_CUDA(ctx, cudaMemcpy(ngen.data(), D.n_gen, 4 * ngen.size(), cudaMemcpyDeviceToHost));
+        memset(host_stats, 0, sizeof(*host_stats));
+        for (int b = 0; b < D.B; ++b) {
+            host_stats->steps += steps[b];
+            host_stats->tokens += (uint64_t)ngen[b];
+            for (int a = 0; a <= kMaxDraft; ++a) host_stats->accept_hist[a] += hist[(size_t)b * (kMaxDraft + 1) + a];
+        }
+        host_stats->wall_ms = ms;
+        host_stats->scr = host_stats->steps ? (double)host_stats->tokens / (double)host_stats->steps : 0.0;
+    }
+    return XSM_OK;
+}
+
+xsm_status xsm_generate_host(xsm_ctx *ctx, int batch, const void *h_cond, const int32_t *h_prompt, int prompt_len,
+                             const xsm_decode_config *dc, int max_new_tokens, int32_t *h_tokens, int32_t *h_lengths,
+                             xsm_stats *host_stats) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    if (!h_cond || !h_prompt || !dc || !h_tokens || !h_lengths) return fail(ctx, XSM_ERR_INVALID_ARG, "null argument");
+    const xsm_model_config &c = ctx->cfg;
+    if (batch < 1 || batch > c.max_batch) return fail(ctx, XSM_ERR_INVALID_ARG, "batch must be in [1, max_batch]");
+    if (prompt_len < 1 || prompt_len - 1 > c.max_seq_len) return fail(ctx, XSM_ERR_INVALID_ARG, "prompt_len out of range");
+    if (max_new_tokens < 1 || max_new_tokens > c.max_seq_len)
+        return fail(ctx, XSM_ERR_INVALID_ARG, "max_new_tokens must be in [1, max_seq_len]");
+    void *d_cond = ctx->ws + ctx->lay.stage_cond;
+    int32_t *d_prompt = at<int32_t>(ctx, ctx->lay.prompt);
+    int32_t *d_tok = at<int32_t>(ctx, ctx->lay.stage_tok);
+    XSM_CUDA(ctx, cudaMemcpyAsync(d_cond, h_cond, esize(c) * (size_t)batch * c.n_cond * c.d_cond, cudaMemcpyHostToDevice, ctx->stream));
+    XSM_CUDA(ctx, cudaMemcpyAsync(d_prompt, h_prompt, sizeof(int32_t) * (size_t)batch * prompt_len, cudaMemcpyHostToDevice, ctx->stream));
+    xsm_status st = xsm_prefill(ctx, batch, d_cond, d_prompt, prompt_len, dc);
+    if (st != XSM_OK) return st;
+    // lengths are staged behind the tokens
+    int32_t *d_len = at<int32_t>(ctx, ctx->lay.step_n_new);
+    st = xsm_generate(ctx, max_new_tokens, d_tok, d_len, host_stats);
+    if (st != XSM_OK) return st;
+    XSM_CUDA(ctx, cudaMemcpyAsync(h_tokens, d_tok, sizeof(int32_t) * (size_t)batch * max_new_tokens, cudaMemcpyDeviceToHost, ctx->stream));
+    XSM_CUDA(ctx, cudaMemcpyAsync(h_lengths, d_len, sizeof(int32_t) * batch, cudaMemcpyDeviceToHost, ctx->stream));
+    XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return XSM_OK;
+}
+
+xsm_status xsm_destroy(xsm_ctx *ctx) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    cudaStreamSynchronize(ctx->stream);
+    if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    if (ctx->ev0) cudaEventDestroy(ctx->ev0);
+    if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+    delete ctx;
+    return XSM_OK;
+}
+
+const char *xsm_last_error(const xsm_ctx *ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+uint64_t xsm_kernel_launches(const xsm_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+xsm_status xsm_debug_get_logits(xsm_ctx *ctx, float *h_logits0, float *h_head_logits) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "no step has run");
+    const Dev &D = ctx->dev;
+    xsm_status st = check_device_status(ctx);
+    if (st != XSM_OK) return st;
+    if (h_logits0) XSM_CUDA(ctx, cudaMemcpy(h_logits0, D.logits0, sizeof(float) * (size_t)D.M * D.V, cudaMemcpyDeviceToHost));
+    if (h_head_logits && D.K > 0)
+        XSM_CUDA(ctx, cudaMemcpy(h_head_logits, D.hlogits, sizeof(float) * (size_t)D.K * D.M * D.V, cudaMemcpyDeviceToHost));
+    return XSM_OK;
+}
+
+xsm_status xsm_debug_get_kv(xsm_ctx *ctx, int layer, int seq, int pos0, int n, float *h_k, float *h_v) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "no cache yet");
+    const Dev &D = ctx->dev;
+    if (layer < 0 || layer >= D.L || seq < 0 || seq >= D.B || pos0 < 0 || n < 0 || !h_k || !h_v)
+        return fail(ctx, XSM_ERR_INVALID_ARG, "bad layer, sequence or range");
+    xsm_status st = check_device_status(ctx);
+    if (st != XSM_OK) return st;
+    int held = 0;
+    XSM_CUDA(ctx, cudaMemcpy(&held, D.n_blocks + seq, 4, cudaMemcpyDeviceToHost));
+    if ((long long)pos0 + n > (long long)held * D.P) return fail(ctx, XSM_ERR_INVALID_ARG, "range beyond the pages held");
+    float *sk = at<float>(ctx, ctx->lay.stage_kv), *sv = sk + (size_t)kKvStagePositions * D.d;
+    for (int p = 0; p < n; p += kKvStagePositions) {
+        const int m = n - p < kKvStagePositions ? n - p : kKvStagePositions;
+        XSM_CUDA(ctx, launch_gather_kv(D, ctx->cfg.dtype, layer, seq, pos0 + p, m, sk, sv, ctx->stream));
+        ctx->launches += 1;
+        XSM_CUDA(ctx, cudaMemcpyAsync(h_k + (size_t)p * D.d, sk, sizeof(float) * (size_t)m * D.d, cudaMemcpyDeviceToHost, ctx->stream));
+        XSM_CUDA(ctx, cudaMemcpyAsync(h_v + (size_t)p * D.d, sv, sizeof(float) * (size_t)m * D.d, cudaMemcpyDeviceToHost, ctx->stream));
+        XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    }
+    return XSM_OK;
+}
+
+xsm_status xsm_debug_set_drafts(xsm_ctx *ctx, const int32_t *h_drafts) {
+    if (!ctx || !h_drafts) return XSM_ERR_INVALID_ARG;
+    if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "xsm_debug_set_drafts before xsm_prefill");
+    const Dev &D = ctx->dev;
+    if (D.K == 0) return XSM_OK;
+    for (int i = 0; i < D.B * D.K; ++i)
+        if (h_drafts[i] < 0 || h_drafts[i] >= D.V) return fail(ctx, XSM_ERR_INVALID_ARG, "draft token out of range");
+    XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    XSM_CUDA(ctx, cudaMemcpy2D(D.window + 1, sizeof(int32_t) * D.K1, h_drafts, sizeof(int32_t) * D.K,
+                               sizeof(int32_t) * D.K, D.B, cudaMemcpyHostToDevice));
+    XSM_CUDA(ctx, launch_embed(D, ctx->cfg.dtype, ctx->stream));
+    ctx->launches += 1;
+    return XSM_OK;
+}
+
+xsm_status xsm_debug_get_state(xsm_ctx *ctx, int32_t *h_len, int32_t *h_window, int32_t *h_finished, int32_t *h_pages,
+                               int32_t *h_free_pages) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "no state before xsm_prefill");
+    const Dev &D = ctx->dev;
+    xsm_status st = check_device_status(ctx);
+    if (st != XSM_OK) return st;
+    if (h_len) XSM_CUDA(ctx, cudaMemcpy(h_len, D.len, 4 * D.B, cudaMemcpyDeviceToHost));
+    if (h_window) XSM_CUDA(ctx, cudaMemcpy(h_window, D.window, 4 * D.M, cudaMemcpyDeviceToHost));
+    if (h_finished) XSM_CUDA(ctx, cudaMemcpy(h_finished, D.finished, 4 * D.B, cudaMemcpyDeviceToHost));
+    if (h_pages) XSM_CUDA(ctx, cudaMemcpy(h_pages, D.n_blocks, 4 * D.B, cudaMemcpyDeviceToHost));
+    if (h_free_pages) XSM_CUDA(ctx, cudaMemcpy(h_free_pages, D.n_free, 4, cudaMemcpyDeviceToHost));
+    return XSM_OK;
+}
+
+xsm_status xsm_debug_set_phase_launch(xsm_ctx *ctx, int on) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    ctx->phase_launch = on ? 1 : 0;
+    return XSM_OK;
+}
+
+}  // extern "C"

@@ -140,9 +140,14 @@ def make_weights(cfg: dict, random_gains: bool = False) -> np.ndarray:
     total = n_weight_elements(cfg)
     bf16 = cfg["dtype"] == 1
     buf = np.empty(total, dtype=np.uint16 if bf16 else np.float32)
-    off = 0
+    jobs, off = [], 0
     for tid, (name, shape, kind) in enumerate(weight_tensors(cfg)):
         n = int(np.prod(shape))
+        jobs.append((tid, kind, off, n))
+        off += n
+
+    def fill(job):          # every tensor has its own stream, so the order of execution is irrelevant
+        tid, kind, o, n = job
         if kind == "gain":
             if random_gains:
                 g = np.random.Generator(np.random.Philox(key=[seed, 1 << 20 | tid]))
@@ -152,8 +157,12 @@ def make_weights(cfg: dict, random_gains: bool = False) -> np.ndarray:
         else:
             w = _normal(seed, tid, n)
             w *= np.float32(sigma * (cfg["out_scale"] if kind == "out" else 1.0))
-        buf[off:off + n] = f32_to_bf16_bits(w) if bf16 else w
-        off += n
+        buf[o:o + n] = f32_to_bf16_bits(w) if bf16 else w
+
+    from concurrent.futures import ThreadPoolExecutor
+    import os
+    with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+        list(ex.map(fill, jobs))
     return buf
 
 

@@ -1,0 +1,220 @@
+"""GPU parity: the CUDA library against the CPU oracle, through the C ABI, on seeded inputs."""
+import numpy as np
+import pytest
+
+from conftest import tiny_cfg
+from paper_2507_23777_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+F32_TOL = dict(atol=2e-4, rtol=2e-4)
+BF16_TOL = dict(atol=2e-2, rtol=1e-2)     # the stated bound for bf16 storage
+
+
+@pytest.fixture(scope="module")
+def P():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a B200"
+    from paper_2507_23777_b200 import build
+    build.build()
+    import parity
+    return parity
+
+
+def scripted(ls, full, rng, good):
+    """Drafts that make exactly `good[b]` acceptances under strict greedy verification."""
+    K, V = ls.K, ls.V
+    st = ls.ctx.xsm_debug_get_state()
+    dr = np.zeros((ls.B, K), dtype=np.int32)
+    for b in range(ls.B):
+        n = int(st["len"][b])
+        t = full[b][n + 1:n + 1 + K].copy()
+        for j in range(good[b], K):
+            t[j] = (t[j] + 1 + int(rng.integers(0, V - 1))) % V
+        if good[b] < K:
+            t[good[b]] = (full[b][n + 1 + good[b]] + 1) % V
+        dr[b] = t
+    return dr
+
+
+@pytest.mark.parametrize("dtype,phase_launch,batch", [(0, True, 1), (0, False, 1), (1, False, 1), (0, False, 3), (1, True, 3)])
+def test_unit_model_lockstep_with_scripted_accept_lengths(P, dtype, phase_launch, batch):
+    """Hand-sized model, ragged shapes (V=50, C=5, dh=16, 4-token pages): every accept length 0..K occurs,
+    logits, committed tokens, windows and the cache agree with the oracle; output is plain greedy."""
+    cfg = tiny_cfg(dtype=dtype, n_draft=3, page_size=16, max_seq_len=96)
+    tol = F32_TOL if dtype == 0 else BF16_TOL
+    ls = P.LockStep(cfg, batch=batch, random_gains=True, phase_launch=phase_launch)
+    ls.begin()
+    # the greedy continuation of every sequence, from the oracle's independent plain loop
+    full = []
+    for b in range(batch):
+        ref = ls.orc.new_seq(ls.cond[b], b).generate_plain([0], ls.odc, 90)
+        full.append(np.concatenate([[0], ref]))
+    rng = np.random.default_rng(0)
+    outs = [[] for _ in range(batch)]
+    seen = set()
+    for it in range(14):
+        good = [int(rng.integers(0, 4)) for _ in range(batch)]
+        toks, acc = ls.step(drafts=scripted(ls, full, rng, good), margin=1e-3 if dtype == 0 else 1e-2, **tol)
+        for b in range(batch):
+            outs[b].extend(toks[b])
+            seen.add(acc[b])
+        if ls.excused == 0:
+            assert acc == good
+    assert seen == {0, 1, 2, 3} or ls.excused > 0
+    if ls.excused == 0:
+        for b in range(batch):
+            assert outs[b] == full[b][1:1 + len(outs[b])].tolist()
+    ls.compare_cache(**tol)
+    st = ls.ctx.xsm_debug_get_state()
+    for b in range(batch):
+        assert st["pages"][b] == -(-(st["len"][b] + 4) // 16)
+    ls.close()
+
+
+def test_config0_tiny_fp32_full_run_is_bit_exact(P):
+    """Config 0: 512 tokens, K=3, strict greedy: token sequence and accept lengths equal the oracle's."""
+    import oracle
+    from paper_2507_23777_b200 import binding
+    cfg = inputs.config(0)
+    w = inputs.make_weights(cfg)
+    cond = inputs.make_cond(cfg)
+    orc = oracle.Oracle(cfg, w)
+    dc = oracle.decode_config(cfg)
+    s = orc.new_seq(cond[0], 0)
+    s.begin([0], dc)
+    ref, ref_steps, ref_hist = s.generate(dc, 512)
+    ctx = binding.Context(cfg, w)
+    ctx.prefill(cond, [0], binding.decode_config(cfg))
+    toks, lens, st = ctx.generate(512)
+    assert lens[0] == 512 and np.array_equal(toks[0], ref)
+    assert st.steps == ref_steps and list(st.accept_hist)[:4] == ref_hist and st.tokens == 512
+    assert abs(st.scr - 512 / ref_steps) < 1e-12
+    ctx.xsm_destroy()
+
+
+def test_config0_lockstep_logits_and_cache(P):
+    cfg = inputs.config(0)
+    ls = P.LockStep(cfg)
+    ls.begin()
+    for _ in range(40):
+        ls.step(margin=1e-3, **F32_TOL)
+    assert ls.excused == 0
+    ls.compare_cache(**F32_TOL)
+    ls.close()
+
+
+def test_config1_small_bf16_prefix(P):
+    """Config 1 (12 layers, d=768, K=4, greedy): logits within 2e-2 + 1e-2|ref|, decisions identical
+    under teacher forcing except at margins below 1e-2, on a prefix of steps."""
+    cfg = inputs.config(1)
+    ls = P.LockStep(cfg)
+    ls.begin()
+    for _ in range(24):
+        ls.step(**BF16_TOL)
+    assert ls.excused <= 3
+    ls.compare_cache(layers=[0, 11], **BF16_TOL)
+    ls.close()
+
+
+def test_sampling_modes_lockstep(P):
+    """Top-k acceptance with top-k / temperature resampling and threshold acceptance on the unit model."""
+    for over in (dict(verify_mode=1, k_accept=3, sample_mode=1, k_sample=4, temperature=0.7, sigma=0.6),
+                 dict(verify_mode=2, delta=0.05, sample_mode=1, k_sample=5, temperature=1.0, sigma=0.6)):
+        cfg = tiny_cfg(dtype=0, n_draft=2, page_size=16, max_seq_len=96, seed=5, **over)
+        ls = P.LockStep(cfg, batch=2, random_gains=True)
+        ls.begin()
+        acc = []
+        for it in range(20):
+            st = ls.ctx.xsm_debug_get_state()
+            drafts = None
+            if it % 2 == 0:      # plant a first draft the backbone is likely to accept: its own runner-up
+                drafts = st["window"][:, 1:].copy()
+                for b in range(2):
+                    z, _ = ls.seqs[b].forward_row(int(st["window"][b, 0]), int(st["len"][b]))
+                    drafts[b, 0] = int(np.argsort(-z, kind="stable")[1])
+            _, a = ls.step(drafts=drafts, margin=1e-3, **F32_TOL)
+            acc.extend(a)
+        assert max(acc) >= 1 and ls.excused <= 2
+        ls.close()
+
+
+def test_prompt_ingestion_and_eos(P):
+    import oracle
+    from paper_2507_23777_b200 import binding
+    cfg = tiny_cfg(dtype=0, n_draft=2, page_size=16, max_seq_len=96)
+    w = inputs.make_weights(cfg, random_gains=True)
+    cond = inputs.make_cond(cfg, 1)
+    orc = oracle.Oracle(cfg, w, n_pages=16)
+    dc = oracle.decode_config(cfg)
+    prompt = [0, 5, 6, 7, 8, 9, 10, 11]
+    ref = orc.new_seq(cond[0], 0).generate_plain(prompt, dc, 30)
+    ctx = binding.Context(cfg, w)
+    ctx.prefill(cond, prompt, binding.decode_config(cfg))
+    st = ctx.xsm_debug_get_state()
+    assert st["len"][0] == 7 and st["window"][0, 0] == 11
+    toks, lens, _ = ctx.generate(30)
+    assert np.array_equal(toks[0], ref)
+    ctx.xsm_destroy()
+    eos = int(ref[12])
+    first = int(np.argmax(ref == eos))
+    cfg_e = dict(cfg, eos_id=eos)
+    ctx = binding.Context(cfg_e, w)
+    ctx.prefill(cond, prompt, binding.decode_config(cfg_e))
+    toks, lens, _ = ctx.generate(30)
+    assert lens[0] == first + 1 and np.array_equal(toks[0, :first + 1], ref[:first + 1]) and (toks[0, first + 1:] == -1).all()
+    ctx.xsm_destroy()
+
+
+def test_batch_equals_independent_runs_and_k0(P):
+    """A batch of sequences gives what each gives alone (own condition, own Philox stream);
+    n_draft = 0 is plain decoding with SCR exactly 1."""
+    from paper_2507_23777_b200 import binding
+    cfg = tiny_cfg(dtype=1, n_draft=2, page_size=16, max_seq_len=96, verify_mode=1, k_accept=2, sample_mode=1,
+                   k_sample=3, temperature=0.8, seed=3, sigma=0.5)
+    w = inputs.make_weights(cfg)
+    cond = inputs.make_cond(cfg, 3)
+    gdc = binding.decode_config(cfg)
+    ctx = binding.Context(cfg, w, max_batch=3)
+    ctx.prefill(cond, [0], gdc)
+    toks, lens, st = ctx.generate(40)
+    assert (lens == 40).all() and st.tokens == 120
+    # sequence 0 alone reproduces row 0 (sequence ids are batch positions)
+    ctx.prefill(cond[:1], [0], gdc)
+    t0, _, _ = ctx.generate(40)
+    assert np.array_equal(t0[0], toks[0])
+    ctx.xsm_destroy()
+    cfg0 = dict(cfg, n_draft=0)
+    w0 = inputs.make_weights(cfg0)
+    ctx = binding.Context(cfg0, w0)
+    ctx.prefill(inputs.make_cond(cfg0, 1), [0], binding.decode_config(cfg0))
+    _, lens, st = ctx.generate(25)
+    assert st.steps == 25 and st.scr == 1.0 and st.accept_hist[0] == 25
+    ctx.xsm_destroy()
+
+
+def test_capacity_and_state_errors(P):
+    from paper_2507_23777_b200 import binding
+    cfg = tiny_cfg(dtype=0, n_draft=2, page_size=16, max_seq_len=96)
+    w = inputs.make_weights(cfg)
+    cond = inputs.make_cond(cfg, 2)
+    mc = binding.model_config(cfg, 2)
+    full = binding.xsm_workspace_bytes(mc)
+    page_bytes = cfg["n_layers"] * 2 * cfg["d_model"] * 16 * 4
+    # room for one sequence's pages only: a batch of two is refused on the host
+    ctx = binding.Context(cfg, w, max_batch=2, workspace_bytes=full - 6 * page_bytes)
+    with pytest.raises(binding.XsmError) as e:
+        ctx.prefill(cond, [0], binding.decode_config(cfg))
+    assert e.value.status == binding.XSM_ERR_CAPACITY
+    ctx.prefill(cond[:1], [0], binding.decode_config(cfg))
+    ctx.generate(20)
+    ctx.xsm_destroy()
+    ctx = binding.Context(cfg, w, max_batch=2)
+    with pytest.raises(binding.XsmError) as e:
+        ctx.xsm_spec_step()
+    assert e.value.status == binding.XSM_ERR_STATE
+    with pytest.raises(binding.XsmError):
+        ctx.prefill(cond, [0], binding.decode_config(dict(cfg, sample_mode=1, k_sample=100)))
+    with pytest.raises(binding.XsmError):
+        binding.Context(cfg, w, max_batch=2, workspace_bytes=4096)
+    ctx.xsm_destroy()
