@@ -96,9 +96,15 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     if (workspace_bytes == 0) {
         L.n_pages = (int)(B * L.max_blocks);
     } else {
-        if (workspace_bytes < cur + 512) return false;
-        size_t n = (workspace_bytes - cur - 512) / (L.page_bytes + 4);
+        if (workspace_bytes <= cur) return false;
+        size_t n = (workspace_bytes - cur) / (L.page_bytes + 4);   // upper bound; the stack is 256-byte padded
         if (n > (size_t)INT_MAX / 2) n = INT_MAX / 2;
+        while (n > 0) {
+            size_t c2 = cur;
+            take(c2, 4 * n);
+            if (c2 + L.page_bytes * n <= workspace_bytes) break;
+            --n;
+        }
         if (n < (size_t)L.max_blocks) return false;
         L.n_pages = (int)n;
     }
