@@ -1,0 +1,275 @@
+"""Benchmark of the speculative decoding hot path on synthetic mesh-model-shaped inputs.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--config I] [--k0]
+
+One "step" is one whole generation of the workload's token count (prefill + every decoding step of
+Algorithm 1) for one batch of synthetic meshes.  The metric is generated mesh tokens per second per
+mesh.  `value` is measured with the condition latents already on the device; `e2e` goes through
+xsm_generate_host with pinned host buffers (host-to-device copy of the condition and prompt, device-
+to-host copy of the tokens, both inside the timed region).  `--impl reference` times the CPU oracle
+instead (rank 0 only).  With N > 1 every rank runs an independent replica (meshes are independent;
+there is no exchange step), and `value` is the aggregate over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2507_23777_b200 import inputs, metrics  # noqa: E402
+
+METRIC = "generated mesh tokens/s per mesh"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "200"], stdout=subprocess.PIPE, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) >= 6 and r[2 + i] == "Active" for r in self.rows)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def workload(args):
+    cfg = inputs.config(args.config)
+    if args.k0:
+        cfg["n_draft"] = 0
+    if args.tokens:
+        cfg["gen_tokens"] = args.tokens
+    return cfg
+
+
+def oracle_sample(cfg, weights, cond, seconds_budget=20.0, min_steps=4):
+    """Times the oracle, as it stands, on the first decoding steps of the workload."""
+    import oracle
+    oracle.build()
+    orc = oracle.Oracle(cfg, weights, n_pages=2 * ((256 + cfg["n_draft"] + 1) // cfg["page_size"] + 2))
+    dc = oracle.decode_config(cfg)
+    s = orc.new_seq(cond[0], 0)
+    s.begin([cfg["bos_id"]], dc)
+    t0 = time.perf_counter()
+    toks = steps = 0
+    while (time.perf_counter() - t0 < seconds_budget or steps < min_steps) and steps < 256:
+        t, _, _, _ = s.step(dc)
+        toks += len(t)
+        steps += 1
+    dt = time.perf_counter() - t0
+    return toks / dt, steps, dt, os.cpu_count()
+
+
+def run_reference(args):
+    cfg = workload(args)
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = inputs.make_weights(cfg)
+    cond = inputs.make_cond(cfg, 1)
+    vals, sample = [], ""
+    per = max(4.0, min(30.0, 120.0 / max(1, args.steps + args.warmup)))
+    for i in range(args.warmup + args.steps):
+        v, steps, dt, cores = oracle_sample(cfg, w, cond, seconds_budget=per)
+        if i >= args.warmup:
+            vals.append((v, dt))
+        sample = f"first {steps} decoding steps of one mesh (context < {steps * (cfg['n_draft'] + 1)} tokens)"
+    value = float(np.mean([v for v, _ in vals]))
+    ms = float(np.mean([dt for _, dt in vals])) * 1e3
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64 accumulate over fp32 state", "data": "synthetic",
+        "config": {"workload": f"config {args.config} ({cfg['name']}): oracle on a bounded prefix", "batch": 1,
+                   "n_draft": cfg["n_draft"]},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2507_23777_b200 import binding, build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    build.build()
+    cfg = workload(args)
+    cfg["seed"] = cfg["seed"] + 1000 * rank if world > 1 else cfg["seed"]   # every replica has its own meshes
+    B, T, K = cfg["batch"], cfg["gen_tokens"], cfg["n_draft"]
+    w = inputs.make_weights(dict(cfg, seed=args.config))
+    cond = inputs.make_cond(cfg, B)
+    ctx = binding.Context(cfg, w, max_batch=B)
+    gdc = binding.decode_config(cfg)
+    d_cond = ctx.cond_to_device(cond)
+    prompt = np.full((B, 1), cfg["bos_id"], dtype=np.int32)
+    d_prompt = torch.from_numpy(prompt).cuda()
+    d_tokens = torch.empty((B, T), dtype=torch.int32, device="cuda")
+    d_lengths = torch.empty(B, dtype=torch.int32, device="cuda")
+    h_cond = torch.from_numpy(ctx.cond_to_host(cond).view(np.int16 if cfg["dtype"] == 1 else np.float32)).pin_memory()
+    h_prompt = torch.from_numpy(prompt).pin_memory()
+    h_tokens = torch.empty((B, T), dtype=torch.int32).pin_memory()
+    h_lengths = torch.empty(B, dtype=torch.int32).pin_memory()
+
+    def one_pass():
+        ctx.xsm_prefill(d_cond, d_prompt, 1, gdc)
+        return ctx.xsm_generate(T, d_tokens, d_lengths)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_pass()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    l0 = ctx.xsm_kernel_launches()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    stats, kernel_ms = [], 0.0
+    for _ in range(args.steps):
+        st = one_pass()
+        stats.append((st.steps, st.tokens, list(st.accept_hist)))
+        kernel_ms += st.wall_ms
+    ev1.record()
+    barrier()
+    launches = ctx.xsm_kernel_launches() - l0
+    ms = ev0.elapsed_time(ev1)
+    # end to end through host buffers
+    ctx.xsm_generate_host(h_cond.numpy(), h_prompt.numpy(), gdc, T, h_tokens.numpy(), h_lengths.numpy())
+    barrier()
+    e0 = time.perf_counter()
+    ev0.record()
+    n_e2e = max(1, min(args.steps, 2))
+    for _ in range(n_e2e):
+        ctx.xsm_generate_host(h_cond.numpy(), h_prompt.numpy(), gdc, T, h_tokens.numpy(), h_lengths.numpy())
+    ev1.record()
+    barrier()
+    ms_e2e = max(ev0.elapsed_time(ev1), (time.perf_counter() - e0) * 1e3)
+    clocks = sampler.stop() if rank == 0 else None
+    assert int(h_lengths.numpy().min()) == T
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    tokens_total = sum(s[1] for s in stats)
+    steps_total = sum(s[0] for s in stats)
+    scr = tokens_total / steps_total
+    value = world * tokens_total / B / (ms / 1e3)
+    e2e = world * n_e2e * T / (ms_e2e / 1e3)
+    peaks, which = measured_peaks()
+    # roofline of the persistent step kernel: algorithmic bytes of all its steps / time inside xsm_generate
+    alg = metrics.algorithmic_bytes(cfg, B)
+    mean_n = (T / 2.0)
+    bytes_per_step = alg["fixed"] + alg["per_position"] * mean_n
+    steps_per_pass = steps_total / args.steps / 1.0
+    n_step_launches = sum(-(-int(s[0] // B) // 64) for s in stats) or 1
+    achieved = bytes_per_step * (steps_total / B) / (kernel_ms / 1e3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 weights and cache, f32 arithmetic" if cfg["dtype"] == 1 else "f32", "data": "synthetic",
+        "config": {"workload": f"config {args.config} ({cfg['name']}): batch {B}, K={K} heads, {T} tokens per mesh, "
+                               f"verify_mode {cfg['verify_mode']}, k={cfg['k_accept']}, T={cfg['temperature']}",
+                   "weights": "iid N(0, sigma) as configured (heads untrained)", "l2": "inputs larger than L2 "
+                   f"({alg['fixed'] / 1e6:.0f} MB of weights streamed per decoding step)", "parallelism": "replicas"},
+        "scr": scr, "decode_steps_per_pass": steps_per_pass, "step_latency_us": kernel_ms * 1e3 / (steps_total / B),
+        "accept_hist": [int(sum(s[2][a] for s in stats)) for a in range(K + 1)],
+        "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": int(h_cond.numel() * h_cond.element_size() + h_prompt.numel() * 4),
+                "d2h_bytes_per_step": int(h_tokens.numel() * 4 + h_lengths.numel() * 4)},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": metrics.measured_traffic(args.config),
+                     "peak_source": f"{which} copy bandwidth (MEASURED_PEAKS.json)" if which == "measured" else "fallback",
+                     "kernel": "step_kernel (persistent; one launch = up to 64 decoding steps)",
+                     "bytes_per_launch": bytes_per_step * steps_total / B / n_step_launches,
+                     "avg_launch_ms": kernel_ms / n_step_launches},
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        v, steps, dt, cores = oracle_sample(cfg, w, cond, seconds_budget=15.0)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"first {steps} decoding steps of one mesh ({dt:.1f} s)"}
+    print(json.dumps(line))
+    ctx.xsm_destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="xsm", choices=["xsm", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload: index into the five configurations")
+    ap.add_argument("--k0", action="store_true", help="non-speculative path of the same library (n_draft = 0)")
+    ap.add_argument("--tokens", type=int, default=0, help="override tokens per mesh")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -60,3 +60,21 @@ def test_no_cpu_fallback():
     cfg = inputs.config(0)
     with pytest.raises(RuntimeError):
         binding.Context(cfg, inputs.make_weights(cfg))
+
+
+def test_speedup_formula_reproduces_tables_3_and_4():
+    """speedup = SCR * latency(A) / latency(row) (Sec. 5.1) against the printed rows."""
+    from paper_2507_23777_b200 import metrics
+    rows = [l.split() for l in open(os.path.join(ROOT, "tests", "golden", "table3_table4_speedup.txt")) if l[0] != "#"]
+    base = float(rows[0][2])
+    assert rows[0][0] == "A" and len(rows) == 7
+    for name, scr, lat, printed in rows:
+        assert abs(metrics.speedup(float(scr), base, float(lat)) - float(printed)) < 0.011, name
+
+
+def test_algorithmic_bytes_match_hand_count():
+    from paper_2507_23777_b200 import metrics
+    a = metrics.algorithmic_bytes(inputs.config(2), 1)      # medium: 24 layers, d 1024, f 4096, V 4096, K 4
+    assert a["backbone"] == 24 * (6 * 1024 ** 2 + 3 * 1024 * 4096) * 2 == 905969664
+    assert a["fixed"] == 905969664 + 8388608 + 41943040 + 24 * 2 * 257 * 1024 * 2
+    assert a["per_position"] == 98304
