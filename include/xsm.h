@@ -164,7 +164,14 @@ XSM_API xsm_status xsm_debug_set_drafts(xsm_ctx *ctx, const int32_t *h_drafts);
 XSM_API xsm_status xsm_debug_get_state(xsm_ctx *ctx, int32_t *h_len, int32_t *h_window, int32_t *h_finished,
                                int32_t *h_pages, int32_t *h_free_pages);
 
-/* Runs the step one phase per launch instead of as one persistent kernel (1) or back (0). */
+/* Runs one decoding step (as xsm_spec_step does, without returning its tokens) and records its timeline:
+ * h_times HOST uint64 [n_rows][n_ctas] nanoseconds of the GPU's global timer; row 0 = the step starts, row
+ * 1 + 2p = stage p of the step has its inputs in shared memory, row 2 + 2p = stage p has published its
+ * outputs; one column per CTA of the persistent kernel; 0 = that CTA had nothing to wait for in that stage.
+ * capacity = number of uint64 words h_times can hold.  Synchronises the stream. */
+XSM_API xsm_status xsm_debug_trace_step(xsm_ctx *ctx, uint64_t *h_times, size_t capacity, int *n_rows, int *n_ctas);
+
+/* Runs the step one stage per launch instead of as one persistent kernel (1) or back (0). */
 XSM_API xsm_status xsm_debug_set_phase_launch(xsm_ctx *ctx, int on);
 
 #ifdef __cplusplus

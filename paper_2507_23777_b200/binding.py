@@ -22,6 +22,7 @@ EXPORTS = [
     "xsm_weights_bytes", "xsm_workspace_bytes", "xsm_create", "xsm_prefill", "xsm_spec_step", "xsm_generate",
     "xsm_generate_host", "xsm_destroy", "xsm_last_error", "xsm_kernel_launches", "xsm_debug_get_logits",
     "xsm_debug_get_kv", "xsm_debug_set_drafts", "xsm_debug_get_state", "xsm_debug_set_phase_launch",
+    "xsm_debug_trace_step",
 ]
 
 
@@ -81,6 +82,7 @@ def load(path: str | None = None):
     L.xsm_debug_set_drafts.argtypes = [vp, ip]
     L.xsm_debug_get_state.argtypes = [vp, ip, ip, ip, ip, ip]
     L.xsm_debug_set_phase_launch.argtypes = [vp, C.c_int]
+    L.xsm_debug_trace_step.argtypes = [vp, vp, C.c_size_t, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     if path is None:
         _lib = L
     return L
@@ -213,6 +215,14 @@ class Context:
         self._check(self.lib.xsm_debug_get_state(self._h, _np_ptr(ln), _np_ptr(win), _np_ptr(fin), _np_ptr(pages),
                                                  _np_ptr(free)))
         return dict(len=ln, window=win, finished=fin, pages=pages, free_pages=int(free[0]))
+
+    def xsm_debug_trace_step(self) -> np.ndarray:
+        """Timeline of one decoding step: uint64 [1 + 2 * stages, CTAs] nanoseconds (see include/xsm.h)."""
+        cap = (1 + 2 * (8 * self.cfg["n_layers"] + 4)) * 256
+        buf = np.zeros(cap, dtype=np.uint64)
+        rows, ctas = C.c_int(), C.c_int()
+        self._check(self.lib.xsm_debug_trace_step(self._h, _np_ptr(buf), cap, C.byref(rows), C.byref(ctas)))
+        return buf[:rows.value * ctas.value].reshape(rows.value, ctas.value)
 
     def xsm_debug_set_phase_launch(self, on: bool):
         self._check(self.lib.xsm_debug_set_phase_launch(self._h, int(on)))

@@ -15,8 +15,9 @@ using namespace xsm;
 
 namespace {
 
-constexpr int kSizingGrid = 256;      // CTA count assumed when sizing split-partial buffers
+constexpr int kSizingGrid = 256;      // CTA count assumed when sizing split-partial buffers and per-CTA marks
 constexpr int kKvStagePositions = 256;
+constexpr int kMinSlots = 5;          // ring slots the shared-memory plan keeps at least
 constexpr int kChunkSteps = 64;       // decoding steps per persistent-kernel launch in xsm_generate
 
 thread_local std::string g_create_error;
@@ -26,8 +27,9 @@ struct Layout {
     size_t phases, jobs, inv_freq, wkc_off, wvc_off;
     size_t len, window, cand, acc_len, finished, n_gen, n_blocks, ingest_left, step_idx, block_table, free_stack,
         scalars, hist, steps, tok_log, step_tokens, step_n_new, prompt;
-    size_t h, qkv, attn, qc, cattn, act, y, logits0, hlogits, rope_cs, part, cpart, part_ctr, cpart_ctr;
-    size_t stage_cond, stage_kv, stage_tok, ckv_pool, kv_pool;
+    size_t h, rope_cs;
+    size_t xchg_begin, hpub, qkv, attn, qc, cattn, act, y, logits0, hlogits, part, cpart, candx, header, done, xchg_end;
+    size_t stage_cond, stage_kv, stage_tok, trace, ckv_pool, kv_pool;
     int n_pages = 0, max_blocks = 0, cpages = 0, tok_ld = 0, n_phases = 0, n_jobs = 0;
     size_t page_bytes = 0;
 };
@@ -50,7 +52,7 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.n_phases = c.n_layers * 8 + 3 + (c.n_draft > 0 ? 1 : 0);
     L.n_jobs = c.n_layers * 6 + 1 + 2 * c.n_draft;
     size_t cur = 0;
-    L.phases = take(cur, sizeof(Phase) * L.n_phases);
+    L.phases = take(cur, sizeof(Stage) * L.n_phases);
     L.jobs = take(cur, sizeof(GemvJob) * L.n_jobs);
     L.inv_freq = take(cur, sizeof(double) * (dh / 2 + 1));
     L.wkc_off = take(cur, sizeof(size_t) * c.n_layers);
@@ -73,6 +75,10 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.step_n_new = take(cur, 4 * B);
     L.prompt = take(cur, 4 * B * (c.max_seq_len + 1));
     L.h = take(cur, 4 * M * d);
+    L.rope_cs = take(cur, 8 * M * (dh / 2));
+    // tagged exchange buffers, cleared together at every xsm_prefill
+    L.xchg_begin = cur;
+    L.hpub = take(cur, 4 * M * d);
     L.qkv = take(cur, 4 * M * 3 * d);
     L.attn = take(cur, 4 * M * d);
     L.qc = take(cur, 4 * M * d);
@@ -81,15 +87,17 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.y = take(cur, 4 * M * d * (c.n_draft > 0 ? c.n_draft : 1));
     L.logits0 = take(cur, 4 * M * V);
     L.hlogits = take(cur, 4 * M * V * (c.n_draft > 0 ? c.n_draft : 1));
-    L.rope_cs = take(cur, 8 * M * (dh / 2));
-    const size_t part_items = B * H + 2 * kSizingGrid;
+    const size_t part_items = B * H + kSizingGrid;      // >= B * H * S_max for every batch
     L.part = take(cur, 4 * part_items * K1 * (dh + 2));
     L.cpart = take(cur, 4 * part_items * K1 * (dh + 2));
-    L.part_ctr = take(cur, 4 * B * H);
-    L.cpart_ctr = take(cur, 4 * B * H);
+    L.candx = take(cur, 4 * B * (K1 + 1));
+    L.header = take(cur, 4 * B * kHeaderWords);
+    L.done = take(cur, 4 * kSizingGrid);
+    L.xchg_end = cur;
     L.stage_cond = take(cur, esize(c) * B * c.n_cond * c.d_cond);
     L.stage_kv = take(cur, 4 * 2 * (size_t)kKvStagePositions * d);
     L.stage_tok = take(cur, 4 * B * (c.max_seq_len + 1));
+    L.trace = take(cur, 8 * (size_t)(1 + 2 * L.n_phases) * kSizingGrid);
     L.ckv_pool = take(cur, esize(c) * (size_t)c.n_layers * 2 * B * L.cpages * H * P * dh);
     L.page_bytes = esize(c) * (size_t)c.n_layers * 2 * H * P * dh;
     // the rest is the shared page pool, preceded by its free stack (4 bytes per page)
@@ -119,14 +127,18 @@ const char *check_config(const xsm_model_config &c) {
         c.n_cond < 1 || c.d_cond < 32 || c.max_batch < 1 || c.max_seq_len < 1)
         return "a model dimension is out of range";
     if (c.n_heads * c.d_head != c.d_model) return "n_heads * d_head must equal d_model";
-    if (c.d_model % 32 || c.d_ff % 32 || c.d_cond % 32) return "d_model, d_ff and d_cond must be multiples of 32";
-    if ((c.d_head & 1) || c.d_head > 128) return "d_head must be even and at most 128";
-    if (c.n_draft < 0 || c.n_draft > XSM_MAX_DRAFT) return "n_draft must be in [0, 16]";
+    if (c.d_model % 128 || c.d_ff % 128) return "d_model and d_ff must be multiples of 128";
+    if (c.d_cond % 32) return "d_cond must be a multiple of 32";
+    if (c.d_head != 32 && c.d_head != 64 && c.d_head != 128) return "d_head must be 32, 64 or 128";
+    if (c.n_draft < 0 || c.n_draft >= XSM_MAX_DRAFT) return "n_draft must be in [0, 15]";
     if (c.head_hidden != c.d_model) return "head_hidden must equal d_model (the head block is residual)";
     if (c.head_kind != 0) return "only MLP heads (head_kind 0) are implemented";
     if (c.dtype != 0 && c.dtype != 1) return "dtype must be 0 (fp32) or 1 (bf16)";
-    if (c.page_size < 16 || c.page_size % 16) return "page_size must be a positive multiple of 16";
-    if ((long long)c.max_batch * (c.n_draft + 1) > kMaxTokens) return "max_batch * (n_draft + 1) exceeds 512";
+    if (c.page_size < 32 || c.page_size % 32) return "page_size must be a positive multiple of 32";
+    if ((long long)c.page_size * c.d_head * (c.dtype == 1 ? 2 : 4) > 16384 * (c.dtype == 1 ? 1 : 4))
+        return "page_size * d_head is too large for one cache tile";
+    if (c.max_batch > kMaxBatch) return "max_batch exceeds 128";
+    if ((long long)c.max_batch * (c.n_draft + 1) > kMaxTokens) return "max_batch * (n_draft + 1) exceeds 128";
     if (c.vocab > (1 << 20)) return "vocab too large";
     if (!(c.rope_theta > 1.0f) || !(c.rms_eps > 0.0f)) return "rope_theta must be > 1 and rms_eps > 0";
     if (c.bos_id < 0 || c.bos_id >= c.vocab || c.eos_id >= c.vocab) return "bos_id / eos_id out of range";
@@ -180,10 +192,11 @@ struct xsm_ctx {
     size_t ws_bytes;
     cudaStream_t stream;
     Dev dev;
-    int grid, phase_launch, prefilled, batch;
+    int grid, sm_count, smem_bytes, phase_launch, prefilled, batch;
+    uint32_t serial;          // decoding steps launched since the last xsm_prefill
     uint64_t launches;
     std::string err;
-    std::vector<Phase> h_phases;
+    std::vector<Stage> h_stages;
     std::vector<GemvJob> h_jobs;
     int *pinned;              // [4] n_active, status
     cudaEvent_t ev0, ev1;
@@ -208,54 +221,118 @@ xsm_status cuda_fail(xsm_ctx *ctx, cudaError_t e, const char *what) {
 template <typename T> T *at(xsm_ctx *ctx, size_t off) { return reinterpret_cast<T *>(ctx->ws + off); }
 const void *wptr(const xsm_ctx *ctx, size_t elem_off) { return ctx->weights + elem_off * esize(ctx->cfg); }
 
-// phase and job tables for the current batch
+// Shared memory of the step kernel for a batch of `batch` sequences: header, ring slots, activation area
+// (also the scratch of attention, verification and the cross-warp reduction), sums of squares.
+// Returns nullptr or the reason why the shape cannot run.
+const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_bytes) {
+    const int K1 = c.n_draft + 1, M = batch * K1, dh = c.d_head;
+    const int kmax = c.d_model > c.d_ff ? c.d_model : c.d_ff;
+    const int tail = (kMaxTokens + 1536) * 4;                        // sums of squares and their partials
+    const int avail = kSmemMax - kSmemHeader - tail;
+    // what the other users of the activation area need
+    const int np = c.dtype == 1 ? (M <= 8 ? 8 : M <= 16 ? 16 : M <= 32 ? 32 : M <= 80 ? 80 : 128) : 8;
+    int need = kConsumerWarps * np * 16 * 4;                          // reduction of the projections
+    const int attn = 2 * 16 * (dh + 8) * 2 + 6 * K1 * dh * 4 + (kConsumerWarps + 1) * K1 * (dh + 2) * 4;
+    if (attn > need) need = attn;
+    const int samp = (((c.vocab + 3) & ~3) + 256) * 4;
+    if (samp > need) need = samp;
+    const int full = M * (kmax * 4 + 16);                             // all activations of the widest projection
+    int acts = full > need ? full : need;
+    if (acts > avail - kMinSlots * kSlotBytes) acts = avail - kMinSlots * kSlotBytes;
+    if (acts < need) return "the shape needs more shared memory than one CTA has";
+    acts = (acts + 127) / 128 * 128;
+    if (acts > avail - kMinSlots * kSlotBytes) acts -= 128;
+    int kca = ((acts / M - 16) / 4) / 128 * 128;
+    if (kca > kmax) kca = kmax;
+    if (kca < 128) return "batch * (n_draft + 1) is too large for the activation staging area";
+    if (c.dtype == 0 && kca < kmax) return "fp32 models need all activations of a projection in shared memory: reduce the batch";
+    if (c.dtype == 0 && M > 24) return "fp32 models support at most 24 token rows per step";
+    int slots = (avail - acts) / kSlotBytes;
+    if (slots > kMaxSlots) slots = kMaxSlots;
+    D.n_slots = slots;
+    D.acts_bytes = acts;
+    D.kca = kca;
+    D.tile_bytes = c.page_size * dh * (c.dtype == 1 ? 2 : 4);
+    D.kv_one_item = 2 * D.tile_bytes <= kSlotBytes ? 1 : 0;
+    smem_bytes = kSmemHeader + slots * kSlotBytes + acts + tail;
+    return nullptr;
+}
+
+// stage and job tables for the current batch
 void build_tables(xsm_ctx *ctx) {
     const xsm_model_config &c = ctx->cfg;
     const Dev &D = ctx->dev;
     const WeightOffsets &w = ctx->wo;
-    const int d = c.d_model, f = c.d_ff, V = c.vocab, K = c.n_draft;
+    const int d = c.d_model, f = c.d_ff, V = c.vocab, K = c.n_draft, L = c.n_layers;
     const size_t M = D.M;
-    ctx->h_phases.clear();
+    const int hw = 3 * L + 1;      // writes of the residual stream per step: the embedding and three per layer
+    ctx->h_stages.clear();
     ctx->h_jobs.clear();
     auto job = [&](const void *W, const void *W2, int rows, int kdim, const float *x, const void *gain, float *out,
-                   int out_ld, int epi) {
+                   int out_ld, int epi, TagRef in, TagRef outt) {
         GemvJob j;
-        j.W = W; j.W2 = W2; j.x = x; j.gain = gain; j.out = out;
-        j.rows = rows; j.kdim = kdim; j.x_ld = kdim; j.out_ld = out_ld; j.epi = epi; j.pad = 0;
+        memset(&j, 0, sizeof(j));
+        j.W = W; j.W2 = W2; j.x = x; j.gain = gain; j.out = out; j.hm = epi == EPI_ADD ? D.h : nullptr;
+        j.rows = rows; j.kdim = kdim; j.out_ld = out_ld; j.epi = epi; j.in = in; j.outt = outt;
         ctx->h_jobs.push_back(j);
         return (int)ctx->h_jobs.size() - 1;
     };
-    auto gemv1 = [&](int layer, int j0, int n) { ctx->h_phases.push_back(Phase{PH_GEMV, layer, j0, n}); };
-    for (int l = 0; l < c.n_layers; ++l) {
-        gemv1(l, job(wptr(ctx, w.wq[l]), nullptr, 3 * d, d, D.h, wptr(ctx, w.g1[l]), D.qkv, 3 * d, EPI_STORE), 1);
-        ctx->h_phases.push_back(Phase{PH_ATTN_SELF, l, 0, 0});
-        gemv1(l, job(wptr(ctx, w.wo[l]), nullptr, d, d, D.attn, nullptr, D.h, d, EPI_ADD), 1);
-        gemv1(l, job(wptr(ctx, w.wqc[l]), nullptr, d, d, D.h, wptr(ctx, w.g2[l]), D.qc, d, EPI_STORE), 1);
-        ctx->h_phases.push_back(Phase{PH_ATTN_CROSS, l, 0, 0});
-        gemv1(l, job(wptr(ctx, w.woc[l]), nullptr, d, d, D.cattn, nullptr, D.h, d, EPI_ADD), 1);
-        gemv1(l, job(wptr(ctx, w.wgate[l]), wptr(ctx, w.wup[l]), f, d, D.h, wptr(ctx, w.g3[l]), D.act, f, EPI_GATEUP), 1);
-        gemv1(l, job(wptr(ctx, w.wdown[l]), nullptr, d, f, D.act, nullptr, D.h, d, EPI_ADD), 1);
+    auto gemv1 = [&](int layer, int j0, int n) {
+        Stage s;
+        memset(&s, 0, sizeof(s));
+        s.kind = ST_GEMV; s.layer = layer; s.job0 = j0; s.njobs = n;
+        ctx->h_stages.push_back(s);
+    };
+    auto attn = [&](int kind, int layer) {
+        Stage s;
+        memset(&s, 0, sizeof(s));
+        s.kind = kind; s.layer = layer;
+        s.in = TagRef{L, layer}; s.outt = TagRef{L, layer}; s.part = TagRef{L, layer};
+        ctx->h_stages.push_back(s);
+    };
+    for (int l = 0; l < L; ++l) {
+        const TagRef per_layer{L, l};
+        gemv1(l, job(wptr(ctx, w.wq[l]), nullptr, 3 * d, d, D.hpub, wptr(ctx, w.g1[l]), D.qkv, 3 * d, EPI_STORE,
+                     TagRef{hw, 3 * l}, per_layer), 1);
+        attn(ST_ATTN_SELF, l);
+        gemv1(l, job(wptr(ctx, w.wo[l]), nullptr, d, d, D.attn, nullptr, D.hpub, d, EPI_ADD, per_layer,
+                     TagRef{hw, 3 * l + 1}), 1);
+        gemv1(l, job(wptr(ctx, w.wqc[l]), nullptr, d, d, D.hpub, wptr(ctx, w.g2[l]), D.qc, d, EPI_STORE,
+                     TagRef{hw, 3 * l + 1}, per_layer), 1);
+        attn(ST_ATTN_CROSS, l);
+        gemv1(l, job(wptr(ctx, w.woc[l]), nullptr, d, d, D.cattn, nullptr, D.hpub, d, EPI_ADD, per_layer,
+                     TagRef{hw, 3 * l + 2}), 1);
+        gemv1(l, job(wptr(ctx, w.wgate[l]), wptr(ctx, w.wup[l]), f, d, D.hpub, wptr(ctx, w.g3[l]), D.act, f, EPI_GATEUP,
+                     TagRef{hw, 3 * l + 2}, per_layer), 1);
+        gemv1(l, job(wptr(ctx, w.wdown[l]), nullptr, d, f, D.act, nullptr, D.hpub, d, EPI_ADD, per_layer,
+                     TagRef{hw, 3 * l + 3}), 1);
     }
-    int j0 = job(wptr(ctx, w.W0), nullptr, V, d, D.h, wptr(ctx, w.gf), D.logits0, V, EPI_STORE);
+    const TagRef once{1, 0};
+    int j0 = job(wptr(ctx, w.W0), nullptr, V, d, D.hpub, wptr(ctx, w.gf), D.logits0, V, EPI_STORE, TagRef{hw, 3 * L}, once);
     for (int i = 0; i < K; ++i)
-        job(wptr(ctx, w.W1[i]), nullptr, d, d, D.h, wptr(ctx, w.gf), D.y + (size_t)i * M * d, d, EPI_HEADY);
+        job(wptr(ctx, w.W1[i]), nullptr, d, d, D.hpub, wptr(ctx, w.gf), D.y + (size_t)i * M * d, d, EPI_HEADY,
+            TagRef{hw, 3 * L}, once);
     gemv1(-1, j0, 1 + K);
     if (K > 0) {
         j0 = (int)ctx->h_jobs.size();
         for (int i = 0; i < K; ++i)
             job(wptr(ctx, w.Wout[i]), nullptr, V, d, D.y + (size_t)i * M * d, nullptr, D.hlogits + (size_t)i * M * V, V,
-                EPI_STORE);
+                EPI_STORE, once, once);
         gemv1(-1, j0, K);
     }
-    ctx->h_phases.push_back(Phase{PH_SAMPLE, -1, 0, 0});
-    ctx->h_phases.push_back(Phase{PH_COMMIT, -1, 0, 0});
+    Stage s;
+    memset(&s, 0, sizeof(s));
+    s.kind = ST_SAMPLE; s.layer = -1;
+    ctx->h_stages.push_back(s);
+    s.kind = ST_COMMIT;
+    ctx->h_stages.push_back(s);
 }
 
 xsm_status check_device_status(xsm_ctx *ctx) {
     XSM_CUDA(ctx, cudaMemcpyAsync(ctx->pinned, ctx->dev.n_active, 8, cudaMemcpyDeviceToHost, ctx->stream));
     XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     const int st = ctx->pinned[1];
-    if (st == XSM_ERR_TIMEOUT) return fail(ctx, XSM_ERR_TIMEOUT, "a grid barrier wait ran out of patience");
+    if (st == XSM_ERR_TIMEOUT) return fail(ctx, XSM_ERR_TIMEOUT, "a bounded device-side wait ran out of patience");
     if (st == XSM_ERR_CAPACITY) return fail(ctx, XSM_ERR_CAPACITY, "the page pool ran dry during decoding");
     if (st != 0) return fail(ctx, XSM_ERR_CUDA, "device status word is set");
     return XSM_OK;
@@ -263,16 +340,19 @@ xsm_status check_device_status(xsm_ctx *ctx) {
 
 // n_steps decoding steps on the stream
 xsm_status run_steps(xsm_ctx *ctx, int n_steps) {
-    const int np = (int)ctx->h_phases.size();
+    const int np = (int)ctx->h_stages.size();
     if (!ctx->phase_launch) {
-        XSM_CUDA(ctx, launch_step(ctx->dev, ctx->cfg.dtype, 0, np, n_steps, 1, ctx->grid, ctx->stream));
+        XSM_CUDA(ctx, launch_step(ctx->dev, ctx->cfg.dtype, 0, np, n_steps, ctx->serial, ctx->grid, ctx->smem_bytes, ctx->stream));
         ctx->launches += 1;
+        ctx->serial += (uint32_t)n_steps;
     } else {
-        for (int t = 0; t < n_steps; ++t)
+        for (int t = 0; t < n_steps; ++t) {
             for (int p = 0; p < np; ++p) {
-                XSM_CUDA(ctx, launch_step(ctx->dev, ctx->cfg.dtype, p, p + 1, 1, 0, ctx->grid, ctx->stream));
+                XSM_CUDA(ctx, launch_step(ctx->dev, ctx->cfg.dtype, p, p + 1, 1, ctx->serial, ctx->grid, ctx->smem_bytes, ctx->stream));
                 ctx->launches += 1;
             }
+            ctx->serial += 1u;
+        }
     }
     return XSM_OK;
 }
@@ -302,6 +382,10 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     Layout L;
     if (!make_layout(*cfg, workspace_bytes, L))
         return fail(nullptr, XSM_ERR_CAPACITY, "workspace cannot hold the buffers plus one sequence of cache pages");
+    Dev probe;
+    memset(&probe, 0, sizeof(probe));
+    int smem_one = 0;
+    if (const char *m = plan_smem(*cfg, 1, probe, smem_one)) return fail(nullptr, XSM_ERR_INVALID_ARG, m);
     xsm_ctx *ctx = new xsm_ctx();
     ctx->cfg = *cfg;
     ctx->lay = L;
@@ -310,7 +394,7 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     ctx->ws = (char *)d_workspace;
     ctx->ws_bytes = workspace_bytes;
     ctx->stream = (cudaStream_t)cuda_stream;
-    ctx->phase_launch = 0; ctx->prefilled = 0; ctx->batch = 0; ctx->launches = 0; ctx->last_wall_ms = 0;
+    ctx->phase_launch = 0; ctx->prefilled = 0; ctx->batch = 0; ctx->launches = 0; ctx->last_wall_ms = 0; ctx->serial = 0;
     ctx->pinned = nullptr; ctx->ev0 = ctx->ev1 = nullptr;
     auto bail = [&](cudaError_t e, const char *what) {
         g_create_error = std::string(what) + ": " + cudaGetErrorString(e);
@@ -322,8 +406,13 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     };
     cudaError_t e;
     int grid = 0;
-    if ((e = step_kernel_setup(cfg->dtype, &grid)) != cudaSuccess) return bail(e, "step kernel setup");
+    if ((e = step_kernel_setup(cfg->dtype, kSmemMax, &grid)) != cudaSuccess) return bail(e, "step kernel setup");
     if (grid < 1) { delete ctx; return fail(nullptr, XSM_ERR_CUDA, "the step kernel does not fit on this device"); }
+    ctx->sm_count = grid;
+    // every CTA must own at least one row of every projection (the exchange protocol relies on it), and the
+    // buffers that are sized per CTA bound the grid from above
+    if (grid > cfg->d_model) grid = cfg->d_model;
+    if (grid > kSizingGrid) grid = kSizingGrid;
     ctx->grid = grid;
     if ((e = cudaHostAlloc((void **)&ctx->pinned, 64, cudaHostAllocDefault)) != cudaSuccess) return bail(e, "cudaHostAlloc");
     if ((e = cudaEventCreate(&ctx->ev0)) != cudaSuccess) return bail(e, "cudaEventCreate");
@@ -338,6 +427,8 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
                              cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) return bail(e, "upload");
     if ((e = cudaMemcpyAsync(ctx->ws + L.wvc_off, ctx->wo.wvc.data(), sizeof(size_t) * cfg->n_layers,
                              cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) return bail(e, "upload");
+    // the caches start at zero: slots that were never written are multiplied by zero weights and must be finite
+    if ((e = cudaMemsetAsync(ctx->ws + L.ckv_pool, 0, L.total - L.ckv_pool, ctx->stream)) != cudaSuccess) return bail(e, "memset");
     if ((e = cudaStreamSynchronize(ctx->stream)) != cudaSuccess) return bail(e, "sync");
 
     Dev &D = ctx->dev;
@@ -348,7 +439,7 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     D.max_seq_len = cfg->max_seq_len; D.tok_ld = L.tok_ld;
     D.eps = cfg->rms_eps; D.scale = (float)(1.0 / sqrt((double)cfg->d_head)); D.bos = cfg->bos_id; D.eos = cfg->eos_id;
     D.max_new = INT_MAX;
-    D.phases = at<Phase>(ctx, L.phases); D.jobs = at<GemvJob>(ctx, L.jobs);
+    D.stages = at<Stage>(ctx, L.phases); D.jobs = at<GemvJob>(ctx, L.jobs);
     D.E = wptr(ctx, ctx->wo.E); D.inv_freq = at<double>(ctx, L.inv_freq);
     D.len = at<int>(ctx, L.len); D.window = at<int>(ctx, L.window); D.cand = at<int>(ctx, L.cand);
     D.acc_len = at<int>(ctx, L.acc_len); D.finished = at<int>(ctx, L.finished); D.n_gen = at<int>(ctx, L.n_gen);
@@ -356,15 +447,16 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     D.ingest_left = at<int>(ctx, L.ingest_left); D.step_idx = at<uint32_t>(ctx, L.step_idx);
     D.free_stack = at<int>(ctx, L.free_stack);
     int *sc = at<int>(ctx, L.scalars);
-    D.n_active = sc; D.status = sc + 1; D.n_free = sc + 2; D.bar = reinterpret_cast<unsigned *>(sc + 16);
+    D.n_active = sc; D.status = sc + 1; D.n_free = sc + 2;
     D.hist = at<unsigned long long>(ctx, L.hist); D.steps = at<unsigned long long>(ctx, L.steps);
     D.tok_log = at<int>(ctx, L.tok_log); D.step_tokens = at<int>(ctx, L.step_tokens);
     D.step_n_new = at<int>(ctx, L.step_n_new); D.prompt = at<int>(ctx, L.prompt);
-    D.h = at<float>(ctx, L.h); D.qkv = at<float>(ctx, L.qkv); D.attn = at<float>(ctx, L.attn);
+    D.h = at<float>(ctx, L.h); D.rope_cs = at<float2>(ctx, L.rope_cs);
+    D.hpub = at<float>(ctx, L.hpub); D.qkv = at<float>(ctx, L.qkv); D.attn = at<float>(ctx, L.attn);
     D.qc = at<float>(ctx, L.qc); D.cattn = at<float>(ctx, L.cattn); D.act = at<float>(ctx, L.act);
     D.y = at<float>(ctx, L.y); D.logits0 = at<float>(ctx, L.logits0); D.hlogits = at<float>(ctx, L.hlogits);
-    D.rope_cs = at<float2>(ctx, L.rope_cs); D.part = at<float>(ctx, L.part); D.cpart = at<float>(ctx, L.cpart);
-    D.part_ctr = at<unsigned>(ctx, L.part_ctr); D.cpart_ctr = at<unsigned>(ctx, L.cpart_ctr);
+    D.part = at<float>(ctx, L.part); D.cpart = at<float>(ctx, L.cpart);
+    D.candx = at<uint32_t>(ctx, L.candx); D.header = at<uint32_t>(ctx, L.header); D.done = at<uint32_t>(ctx, L.done);
     D.kv_pool = ctx->ws + L.kv_pool; D.ckv_pool = ctx->ws + L.ckv_pool;
     *out = ctx;
     return XSM_OK;
@@ -384,36 +476,46 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
         return fail(ctx, XSM_ERR_INVALID_ARG, "k_sample must be in [1, 64] and temperature > 0");
     if ((long long)batch * ctx->lay.max_blocks > ctx->lay.n_pages)
         return fail(ctx, XSM_ERR_CAPACITY, "the page pool cannot hold `batch` sequences of max_seq_len positions");
+    Dev &D = ctx->dev;
+    int smem_bytes = 0;
+    if (const char *m = plan_smem(c, batch, D, smem_bytes)) return fail(ctx, XSM_ERR_CAPACITY, m);
+    ctx->smem_bytes = smem_bytes;
     ctx->dc = *dc;
     ctx->batch = batch;
-    Dev &D = ctx->dev;
     D.B = batch; D.M = batch * D.K1;
     D.verify_mode = dc->verify_mode; D.k_accept = dc->k_accept; D.delta = dc->delta;
     D.sample_mode = dc->sample_mode; D.k_sample = dc->k_sample; D.temperature = dc->temperature;
     D.key0 = (uint32_t)dc->seed; D.key1 = (uint32_t)(dc->seed >> 32);
     D.max_new = INT_MAX; D.prompt_len = prompt_len;
     const int bh = batch * D.H;
-    int s_self = (2 * ctx->grid) / bh;
-    D.S_self = s_self < 1 ? 1 : (s_self > 64 ? 64 : s_self);
-    int s_cross = ctx->grid / bh;
-    if (s_cross > D.cpages) s_cross = D.cpages;
-    D.S_cross = s_cross < 1 ? 1 : s_cross;
+    int s_max = ctx->grid / bh;
+    D.S_max = s_max < 1 ? 1 : (s_max > 64 ? 64 : s_max);
+    // the condition's keys and values of one head: one item while that is at most 96 KB, else split over CTAs
+    int s_cross = 1;
+    if ((long long)D.cpages * 2 * D.tile_bytes > 96 * 1024) {
+        s_cross = D.S_max < D.cpages ? D.S_max : D.cpages;
+        if (s_cross < 1) s_cross = 1;
+    }
+    D.S_cross = s_cross;
     build_tables(ctx);
-    D.n_phases = (int)ctx->h_phases.size();
-    if ((int)ctx->h_phases.size() > ctx->lay.n_phases || (int)ctx->h_jobs.size() > ctx->lay.n_jobs)
-        return fail(ctx, XSM_ERR_STATE, "internal: phase table overflow");
-    XSM_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->lay.phases, ctx->h_phases.data(), sizeof(Phase) * ctx->h_phases.size(),
+    D.n_stages = (int)ctx->h_stages.size();
+    if ((int)ctx->h_stages.size() > ctx->lay.n_phases || (int)ctx->h_jobs.size() > ctx->lay.n_jobs)
+        return fail(ctx, XSM_ERR_STATE, "internal: stage table overflow");
+    XSM_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->lay.phases, ctx->h_stages.data(), sizeof(Stage) * ctx->h_stages.size(),
                                   cudaMemcpyHostToDevice, ctx->stream));
     XSM_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->lay.jobs, ctx->h_jobs.data(), sizeof(GemvJob) * ctx->h_jobs.size(),
                                   cudaMemcpyHostToDevice, ctx->stream));
     if ((const void *)d_prompt != (const void *)D.prompt)
         XSM_CUDA(ctx, cudaMemcpyAsync((void *)D.prompt, d_prompt, sizeof(int32_t) * batch * prompt_len,
                                       cudaMemcpyDeviceToDevice, ctx->stream));
+    // no tag of an earlier generation may survive: the exchange buffers restart from "never written"
+    XSM_CUDA(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.xchg_begin, 0, ctx->lay.xchg_end - ctx->lay.xchg_begin, ctx->stream));
+    ctx->serial = 0;
     // the tables above are read from host vectors that may be rebuilt by the next prefill
     XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     XSM_CUDA(ctx, launch_cross_kv(D, c.dtype, ctx->weights, at<size_t>(ctx, ctx->lay.wkc_off),
                                   at<size_t>(ctx, ctx->lay.wvc_off), d_cond, ctx->stream));
-    XSM_CUDA(ctx, launch_init(D, c.dtype, ctx->stream));
+    XSM_CUDA(ctx, launch_init(D, c.dtype, ctx->serial, ctx->stream));
     ctx->launches += 3;
     ctx->prefilled = 1;
     const int ingest_steps = (prompt_len - 1 + D.K1 - 1) / D.K1;
@@ -524,15 +626,26 @@ const char *xsm_last_error(const xsm_ctx *ctx) { return ctx ? ctx->err.c_str() :
 
 uint64_t xsm_kernel_launches(const xsm_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
+// the exchange buffers hold fp32 words whose two lowest mantissa bits are a tag
+static void strip_tags(float *p, size_t n) {
+    uint32_t *u = reinterpret_cast<uint32_t *>(p);
+    for (size_t i = 0; i < n; ++i) u[i] &= ~3u;
+}
+
 xsm_status xsm_debug_get_logits(xsm_ctx *ctx, float *h_logits0, float *h_head_logits) {
     if (!ctx) return XSM_ERR_INVALID_ARG;
     if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "no step has run");
     const Dev &D = ctx->dev;
     xsm_status st = check_device_status(ctx);
     if (st != XSM_OK) return st;
-    if (h_logits0) XSM_CUDA(ctx, cudaMemcpy(h_logits0, D.logits0, sizeof(float) * (size_t)D.M * D.V, cudaMemcpyDeviceToHost));
-    if (h_head_logits && D.K > 0)
+    if (h_logits0) {
+        XSM_CUDA(ctx, cudaMemcpy(h_logits0, D.logits0, sizeof(float) * (size_t)D.M * D.V, cudaMemcpyDeviceToHost));
+        strip_tags(h_logits0, (size_t)D.M * D.V);
+    }
+    if (h_head_logits && D.K > 0) {
         XSM_CUDA(ctx, cudaMemcpy(h_head_logits, D.hlogits, sizeof(float) * (size_t)D.K * D.M * D.V, cudaMemcpyDeviceToHost));
+        strip_tags(h_head_logits, (size_t)D.K * D.M * D.V);
+    }
     return XSM_OK;
 }
 
@@ -569,7 +682,7 @@ xsm_status xsm_debug_set_drafts(xsm_ctx *ctx, const int32_t *h_drafts) {
     XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     XSM_CUDA(ctx, cudaMemcpy2D(D.window + 1, sizeof(int32_t) * D.K1, h_drafts, sizeof(int32_t) * D.K,
                                sizeof(int32_t) * D.K, D.B, cudaMemcpyHostToDevice));
-    XSM_CUDA(ctx, launch_embed(D, ctx->cfg.dtype, ctx->stream));
+    XSM_CUDA(ctx, launch_embed(D, ctx->cfg.dtype, ctx->serial, ctx->stream));
     ctx->launches += 1;
     return XSM_OK;
 }
@@ -586,6 +699,28 @@ xsm_status xsm_debug_get_state(xsm_ctx *ctx, int32_t *h_len, int32_t *h_window, 
     if (h_finished) XSM_CUDA(ctx, cudaMemcpy(h_finished, D.finished, 4 * D.B, cudaMemcpyDeviceToHost));
     if (h_pages) XSM_CUDA(ctx, cudaMemcpy(h_pages, D.n_blocks, 4 * D.B, cudaMemcpyDeviceToHost));
     if (h_free_pages) XSM_CUDA(ctx, cudaMemcpy(h_free_pages, D.n_free, 4, cudaMemcpyDeviceToHost));
+    return XSM_OK;
+}
+
+xsm_status xsm_debug_trace_step(xsm_ctx *ctx, uint64_t *h_times, size_t capacity, int *n_rows, int *n_ctas) {
+    if (!ctx || !h_times || !n_rows || !n_ctas) return XSM_ERR_INVALID_ARG;
+    if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "xsm_debug_trace_step before xsm_prefill");
+    if (ctx->phase_launch) return fail(ctx, XSM_ERR_STATE, "the timeline is taken from the persistent kernel");
+    const int rows = 1 + 2 * (int)ctx->h_stages.size();
+    const size_t words = (size_t)rows * ctx->grid;
+    if (capacity < words) return fail(ctx, XSM_ERR_CAPACITY, "h_times is too small");
+    unsigned long long *d_trace = at<unsigned long long>(ctx, ctx->lay.trace);
+    XSM_CUDA(ctx, cudaMemsetAsync(d_trace, 0, 8 * words, ctx->stream));
+    ctx->dev.trace = d_trace;
+    ctx->dev.max_new = INT_MAX;
+    xsm_status st = run_steps(ctx, 1);
+    ctx->dev.trace = nullptr;
+    if (st != XSM_OK) return st;
+    st = check_device_status(ctx);
+    if (st != XSM_OK) return st;
+    XSM_CUDA(ctx, cudaMemcpy(h_times, d_trace, 8 * words, cudaMemcpyDeviceToHost));
+    *n_rows = rows;
+    *n_ctas = ctx->grid;
     return XSM_OK;
 }
 

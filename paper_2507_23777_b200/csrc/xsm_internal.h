@@ -5,38 +5,62 @@
 
 namespace xsm {
 
-constexpr int kThreads = 512;            // threads per CTA of the persistent step kernel
-constexpr int kWarps = kThreads / 32;
-constexpr int kMaxDraft = 16;
-constexpr int kMaxTokens = 512;          // largest M = batch * (K + 1)
-constexpr int kUnitBlock = 128;          // weight rows a CTA accumulates at a time
-constexpr int kSmemBytes = 200 * 1024;   // dynamic shared memory of the step kernel
+// ---- geometry of the persistent step kernel
+constexpr int kConsumerWarps = 8;                    // warps that compute
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kThreads = kConsumerThreads + 32;      // + one producer warp that feeds the ring
+constexpr int kMaxDraft = 16;                        // size of the histogram rows (n_draft itself is <= 15)
+constexpr int kMaxTokens = 128;                      // largest M = batch * (K + 1)
+constexpr int kMaxBatch = 128;
 
-// One step of Algorithm 1 is a fixed list of phases; consecutive phases are separated by a grid barrier.
-enum PhaseKind : int { PH_GEMV = 0, PH_ATTN_SELF = 1, PH_ATTN_CROSS = 2, PH_SAMPLE = 3, PH_COMMIT = 4 };
+// Ring of shared-memory slots filled by bulk copies.  A weight item is up to 16 rows of up to 1024 bytes,
+// rows kRowPitch bytes apart (1024 + 64: rows g and g+1 land in different halves of a 128-byte bank line).
+// A cache item is one (page, head) tile of keys followed by the tile of values (or one of them when both do
+// not fit).
+constexpr int kItemRows = 16;
+constexpr int kItemRowBytes = 1024;
+constexpr int kRowPitch = kItemRowBytes + 64;
+constexpr int kSlotBytes = kItemRows * kRowPitch;    // 17408
+constexpr int kMaxSlots = 12;
+constexpr int kSmemHeader = 2048;                    // barriers and per-step scalars
+constexpr int kSmemMax = 227 * 1024;
+
+// One step of Algorithm 1 is a fixed list of stages.  A stage's output is published in global memory as
+// fp32 words whose two lowest mantissa bits carry a tag (1..3, cycling with the write index of the buffer);
+// the next stage spins on the words it needs until they carry the expected tag.  No grid barrier exists.
+enum StageKind : int { ST_GEMV = 0, ST_ATTN_SELF = 1, ST_ATTN_CROSS = 2, ST_SAMPLE = 3, ST_COMMIT = 4 };
 enum Epilogue : int {
     EPI_STORE = 0,    // out[m][r]  = W[r] . x[m]
-    EPI_ADD = 1,      // out[m][r] += W[r] . x[m]                       (residual)
+    EPI_ADD = 1,      // h[m][r]   += W[r] . x[m]; out[m][r] = h[m][r]      (residual stream)
     EPI_GATEUP = 2,   // out[m][r]  = SiLU(Wgate[r] . x[m]) * (Wup[r] . x[m])
-    EPI_HEADY = 3     // out[m][r]  = x[m][r] + SiLU(W[r] . x[m])       (x = normed input)
+    EPI_HEADY = 3     // out[m][r]  = x[m][r] + SiLU(W[r] . x[m])           (x = normed input)
 };
+
+// Write index of a tagged buffer = serial * wps + j (serial: decoding steps since xsm_prefill; wps: writes
+// of that buffer per step; j: which write of the step).  tag = 1 + index % 3.
+struct TagRef { int wps, j; };
 
 struct GemvJob {
     const void *W, *W2;      // weight rows; W2: the up projection of EPI_GATEUP
-    const float *x;          // input activations [M][kdim]
+    const float *x;          // tagged input activations [M][kdim]
     const void *gain;        // RMSNorm gain of the input (weight dtype) or nullptr: input used as is
-    float *out;
-    int rows, kdim, x_ld, out_ld, epi, pad;
+    float *out;              // tagged output [M][out_ld]
+    float *hm;               // EPI_ADD: untagged fp32 master copy of the residual stream [M][out_ld]
+    int rows, kdim, out_ld, epi;
+    TagRef in, outt;
 };
 
-struct Phase { int kind, layer, job0, njobs; };
+struct Stage {
+    int kind, layer, job0, njobs;
+    TagRef in, outt, part;   // attention: q/k/v (or q) in, attention rows out, split partials
+};
 
 // Everything a kernel needs; passed by value.
 struct Dev {
     // shape
     int L, d, H, dh, f, V, C, dc, K, K1, B, M, P;
     int max_blocks, n_pages, cpages, max_seq_len, tok_ld;
-    int S_self, S_cross;
+    int S_max, S_cross;            // most key splits of a self-attention item; splits of a cross-attention item
     float eps, scale;
     int bos, eos;
     // decoding rule
@@ -44,13 +68,15 @@ struct Dev {
     float delta, temperature;
     uint32_t key0, key1;
     int max_new;
-    // tables
-    const Phase *phases;
+    // stage tables
+    const Stage *stages;
     const GemvJob *jobs;
-    int n_phases;
+    int n_stages;
     const void *E;                 // embedding table
     const double *inv_freq;        // [dh/2] theta^(-2i/dh)
-    // per-sequence state
+    // shared-memory plan of the step kernel
+    int n_slots, acts_bytes, kca, tile_bytes, kv_one_item;
+    // per-sequence state (plain words, read by other CTAs only after they have seen the step header)
     int *len, *window, *cand, *acc_len, *finished, *n_gen, *n_blocks, *block_table, *ingest_left;
     uint32_t *step_idx;
     int *free_stack, *n_free, *n_active, *status;
@@ -58,29 +84,31 @@ struct Dev {
     int *tok_log, *step_tokens, *step_n_new;
     const int *prompt;
     int prompt_len;
-    // activations
-    float *h, *qkv, *attn, *qc, *cattn, *act, *y, *logits0, *hlogits;
+    // tagged exchange buffers
+    float *hpub, *qkv, *attn, *qc, *cattn, *act, *y, *logits0, *hlogits, *part, *cpart;
+    uint32_t *candx, *header;      // [B][K1 + 1] resampled tokens and accept length; [B][4] len, flags
+    uint32_t *done;                // [grid] "this CTA has finished the projections of the step"
+    unsigned long long *trace;     // null, or [1 + 2 * n_stages][grid] nanosecond timestamps of the launch's first step
+    // untagged
+    float *h;                      // master copy of the residual stream (each column range has one owner CTA)
     float2 *rope_cs;               // [M][dh/2] cos, sin of the window rows' positions
-    float *part, *cpart;           // split partials: [B*H*S][K1][dh+2]
-    unsigned *part_ctr, *cpart_ctr;
     // caches
-    void *kv_pool;                 // [L][2][n_pages][H][P][dh]
-    void *ckv_pool;                // [L][2][B*cpages][H][P][dh]
-    unsigned *bar;
+    void *kv_pool;                 // [L][2][n_pages][H] tiles of P x dh
+    void *ckv_pool;                // [L][2][B*cpages][H] tiles of P x dh
 };
 
-struct LaunchInfo { int grid; int coop; };
+constexpr int kHeaderWords = 4;    // per sequence: len, flags (1 finished, 2 ingesting a prompt), 0, 0
 
 // Host-side launchers (xsm_kernels.cu).  All return the CUDA error of the launch.
-cudaError_t launch_step(const Dev &D, int dtype, int ph_lo, int ph_hi, int n_steps, int barrier, int grid,
-                        cudaStream_t st);
+cudaError_t launch_step(const Dev &D, int dtype, int st_lo, int st_hi, int n_steps, uint32_t serial0, int grid,
+                        int smem_bytes, cudaStream_t st);
 cudaError_t launch_cross_kv(const Dev &D, int dtype, const void *W /*flat weights*/, const size_t *wkc_off,
                             const size_t *wvc_off, const void *cond, cudaStream_t st);
-cudaError_t launch_init(const Dev &D, int dtype, cudaStream_t st);
-cudaError_t launch_embed(const Dev &D, int dtype, cudaStream_t st);
+cudaError_t launch_init(const Dev &D, int dtype, uint32_t serial, cudaStream_t st);
+cudaError_t launch_embed(const Dev &D, int dtype, uint32_t serial, cudaStream_t st);
 cudaError_t launch_gather_kv(const Dev &D, int dtype, int layer, int seq, int pos0, int n, float *out_k,
                              float *out_v, cudaStream_t st);
 cudaError_t launch_export(const Dev &D, int max_new, int *d_tokens, int *d_lengths, cudaStream_t st);
-cudaError_t step_kernel_setup(int dtype, int *max_grid);
+cudaError_t step_kernel_setup(int dtype, int smem_bytes, int *max_grid);
 
 }  // namespace xsm

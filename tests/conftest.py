@@ -22,6 +22,15 @@ def tiny_cfg(**over):
     return c
 
 
+def gpu_cfg(**over):
+    """The smallest model the CUDA library accepts (d_model and d_ff multiples of 128, d_head 32, 32-token
+    pages) with ragged sizes everywhere else: 50-token vocabulary, 5 condition latents of width 64."""
+    c = tiny_cfg(d_model=128, n_heads=4, d_head=32, d_ff=256, n_cond=5, d_cond=64, head_hidden=128, page_size=32,
+                 max_seq_len=96)
+    c.update(over)
+    return c
+
+
 @pytest.fixture(scope="session")
 def oracle_mod():
     import oracle

@@ -2,7 +2,7 @@
 import numpy as np
 import pytest
 
-from conftest import tiny_cfg
+from conftest import gpu_cfg
 from paper_2507_23777_b200 import inputs
 
 pytestmark = pytest.mark.gpu
@@ -39,11 +39,11 @@ def scripted(ls, full, rng, good):
 
 @pytest.mark.parametrize("dtype,phase_launch,batch", [(0, True, 1), (0, False, 1), (1, False, 1), (0, False, 3), (1, True, 3)])
 def test_unit_model_lockstep_with_scripted_accept_lengths(P, dtype, phase_launch, batch):
-    """Hand-sized model, ragged shapes (V=50, C=5, dh=16, 4-token pages): every accept length 0..K occurs,
+    """Hand-sized model, ragged shapes (V=50, C=5, dh=32, 32-token pages): every accept length 0..K occurs,
     logits, committed tokens, windows and the cache agree with the oracle; output is plain greedy."""
     # bf16: weights scaled so that logits have the magnitude of the real configurations (about 0.5),
     # which is what the absolute part of the bf16 bound assumes
-    cfg = tiny_cfg(dtype=dtype, n_draft=3, page_size=16, max_seq_len=96, sigma=0.3 if dtype == 0 else 0.1)
+    cfg = gpu_cfg(dtype=dtype, n_draft=3, sigma=0.15 if dtype == 0 else 0.05)
     tol = F32_TOL if dtype == 0 else BF16_TOL
     ls = P.LockStep(cfg, batch=batch, random_gains=True, phase_launch=phase_launch)
     ls.begin()
@@ -70,7 +70,7 @@ def test_unit_model_lockstep_with_scripted_accept_lengths(P, dtype, phase_launch
     ls.compare_cache(**tol)
     st = ls.ctx.xsm_debug_get_state()
     for b in range(batch):
-        assert st["pages"][b] == -(-(st["len"][b] + 4) // 16)
+        assert st["pages"][b] == -(-(st["len"][b] + 4) // 32)
     ls.close()
 
 
@@ -121,9 +121,9 @@ def test_config1_small_bf16_prefix(P):
 
 def test_sampling_modes_lockstep(P):
     """Top-k acceptance with top-k / temperature resampling and threshold acceptance on the unit model."""
-    for over in (dict(verify_mode=1, k_accept=3, sample_mode=1, k_sample=4, temperature=0.7, sigma=0.6),
-                 dict(verify_mode=2, delta=0.05, sample_mode=1, k_sample=5, temperature=1.0, sigma=0.6)):
-        cfg = tiny_cfg(dtype=0, n_draft=2, page_size=16, max_seq_len=96, seed=5, **over)
+    for over in (dict(verify_mode=1, k_accept=3, sample_mode=1, k_sample=4, temperature=0.7, sigma=0.3),
+                 dict(verify_mode=2, delta=0.05, sample_mode=1, k_sample=5, temperature=1.0, sigma=0.3)):
+        cfg = gpu_cfg(dtype=0, n_draft=2, seed=5, **over)
         ls = P.LockStep(cfg, batch=2, random_gains=True)
         ls.begin()
         acc = []
@@ -144,7 +144,7 @@ def test_sampling_modes_lockstep(P):
 def test_prompt_ingestion_and_eos(P):
     import oracle
     from paper_2507_23777_b200 import binding
-    cfg = tiny_cfg(dtype=0, n_draft=2, page_size=16, max_seq_len=96)
+    cfg = gpu_cfg(dtype=0, n_draft=2, sigma=0.15)
     w = inputs.make_weights(cfg, random_gains=True)
     cond = inputs.make_cond(cfg, 1)
     orc = oracle.Oracle(cfg, w, n_pages=16)
@@ -172,8 +172,8 @@ def test_batch_equals_independent_runs_and_k0(P):
     """A batch of sequences gives what each gives alone (own condition, own Philox stream);
     n_draft = 0 is plain decoding with SCR exactly 1."""
     from paper_2507_23777_b200 import binding
-    cfg = tiny_cfg(dtype=1, n_draft=2, page_size=16, max_seq_len=96, verify_mode=1, k_accept=2, sample_mode=1,
-                   k_sample=3, temperature=0.8, seed=3, sigma=0.5)
+    cfg = gpu_cfg(dtype=1, n_draft=2, verify_mode=1, k_accept=2, sample_mode=1, k_sample=3, temperature=0.8, seed=3,
+                  sigma=0.25)
     w = inputs.make_weights(cfg)
     cond = inputs.make_cond(cfg, 3)
     gdc = binding.decode_config(cfg)
@@ -197,14 +197,14 @@ def test_batch_equals_independent_runs_and_k0(P):
 
 def test_capacity_and_state_errors(P):
     from paper_2507_23777_b200 import binding
-    cfg = tiny_cfg(dtype=0, n_draft=2, page_size=16, max_seq_len=96)
+    cfg = gpu_cfg(dtype=0, n_draft=2, sigma=0.15)
     w = inputs.make_weights(cfg)
     cond = inputs.make_cond(cfg, 2)
     mc = binding.model_config(cfg, 2)
     full = binding.xsm_workspace_bytes(mc)
-    page_bytes = cfg["n_layers"] * 2 * cfg["d_model"] * 16 * 4
+    page_bytes = cfg["n_layers"] * 2 * cfg["d_model"] * 32 * 4
     # room for one sequence's pages only: a batch of two is refused on the host
-    ctx = binding.Context(cfg, w, max_batch=2, workspace_bytes=full - 6 * page_bytes)
+    ctx = binding.Context(cfg, w, max_batch=2, workspace_bytes=full - 3 * page_bytes)
     with pytest.raises(binding.XsmError) as e:
         ctx.prefill(cond, [0], binding.decode_config(cfg))
     assert e.value.status == binding.XSM_ERR_CAPACITY
