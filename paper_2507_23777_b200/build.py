@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libxsm.so")
-SOURCES = ["xsm_api.cu", "xsm_kernels.cu"]
-HEADERS = ["xsm_internal.h", os.path.join("..", "..", "include", "xsm.h")]
+SOURCES = ["xsm_api.cu", "xsm_kernels.cu", "xsm_step_dh32.cu", "xsm_step_dh64.cu", "xsm_step_dh128.cu"]
+HEADERS = ["xsm_internal.h", "xsm_device.cuh", os.path.join("..", "..", "include", "xsm.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

@@ -28,7 +28,7 @@ struct Layout {
     size_t len, window, cand, acc_len, finished, n_gen, n_blocks, ingest_left, step_idx, block_table, free_stack,
         scalars, hist, steps, tok_log, step_tokens, step_n_new, prompt;
     size_t h, rope_cs;
-    size_t xchg_begin, hpub, qkv, attn, qc, cattn, act, y, logits0, hlogits, part, cpart, candx, header, done, xchg_end;
+    size_t xchg_begin, hpub, qkv, attn, qc, cattn, act, y, logits0, hlogits, part, cpart, candx, header, done, sspub, xchg_end;
     size_t stage_cond, stage_kv, stage_tok, trace, ckv_pool, kv_pool;
     int n_pages = 0, max_blocks = 0, cpages = 0, tok_ld = 0, n_phases = 0, n_jobs = 0;
     size_t page_bytes = 0;
@@ -93,6 +93,7 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.candx = take(cur, 4 * B * (K1 + 1));
     L.header = take(cur, 4 * B * kHeaderWords);
     L.done = take(cur, 4 * kSizingGrid);
+    L.sspub = take(cur, 4 * (size_t)kSizingGrid * M);
     L.xchg_end = cur;
     L.stage_cond = take(cur, esize(c) * B * c.n_cond * c.d_cond);
     L.stage_kv = take(cur, 4 * 2 * (size_t)kKvStagePositions * d);
@@ -231,7 +232,7 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     const int avail = kSmemMax - kSmemHeader - tail;
     // what the other users of the activation area need
     const int np = c.dtype == 1 ? (M <= 8 ? 8 : M <= 16 ? 16 : M <= 32 ? 32 : M <= 80 ? 80 : 128) : 8;
-    int need = kConsumerWarps * np * 16 * 4;                          // reduction of the projections
+    int need = kConsumerWarps * np * 16 * 4 + 2 * 16 * M * 4;         // reduction of the projections, new residual values
     const int attn = 2 * 16 * (dh + 8) * 2 + 6 * K1 * dh * 4 + (kConsumerWarps + 1) * K1 * (dh + 2) * 4;
     if (attn > need) need = attn;
     const int samp = (((c.vocab + 3) & ~3) + 256) * 4;
@@ -269,11 +270,12 @@ void build_tables(xsm_ctx *ctx) {
     ctx->h_stages.clear();
     ctx->h_jobs.clear();
     auto job = [&](const void *W, const void *W2, int rows, int kdim, const float *x, const void *gain, float *out,
-                   int out_ld, int epi, TagRef in, TagRef outt) {
+                   int out_ld, int epi, TagRef in, TagRef outt, const void *gain_out = nullptr, int out_plain = 0) {
         GemvJob j;
         memset(&j, 0, sizeof(j));
         j.W = W; j.W2 = W2; j.x = x; j.gain = gain; j.out = out; j.hm = epi == EPI_ADD ? D.h : nullptr;
         j.rows = rows; j.kdim = kdim; j.out_ld = out_ld; j.epi = epi; j.in = in; j.outt = outt;
+        j.gain_out = gain_out; j.out_plain = out_plain;
         ctx->h_jobs.push_back(j);
         return (int)ctx->h_jobs.size() - 1;
     };
@@ -295,20 +297,21 @@ void build_tables(xsm_ctx *ctx) {
         gemv1(l, job(wptr(ctx, w.wq[l]), nullptr, 3 * d, d, D.hpub, wptr(ctx, w.g1[l]), D.qkv, 3 * d, EPI_STORE,
                      TagRef{hw, 3 * l}, per_layer), 1);
         attn(ST_ATTN_SELF, l);
+        // a stage that adds to the residual stream publishes it with the gain of the RMSNorm that reads it next
         gemv1(l, job(wptr(ctx, w.wo[l]), nullptr, d, d, D.attn, nullptr, D.hpub, d, EPI_ADD, per_layer,
-                     TagRef{hw, 3 * l + 1}), 1);
+                     TagRef{hw, 3 * l + 1}, wptr(ctx, w.g2[l])), 1);
         gemv1(l, job(wptr(ctx, w.wqc[l]), nullptr, d, d, D.hpub, wptr(ctx, w.g2[l]), D.qc, d, EPI_STORE,
                      TagRef{hw, 3 * l + 1}, per_layer), 1);
         attn(ST_ATTN_CROSS, l);
         gemv1(l, job(wptr(ctx, w.woc[l]), nullptr, d, d, D.cattn, nullptr, D.hpub, d, EPI_ADD, per_layer,
-                     TagRef{hw, 3 * l + 2}), 1);
+                     TagRef{hw, 3 * l + 2}, wptr(ctx, w.g3[l])), 1);
         gemv1(l, job(wptr(ctx, w.wgate[l]), wptr(ctx, w.wup[l]), f, d, D.hpub, wptr(ctx, w.g3[l]), D.act, f, EPI_GATEUP,
                      TagRef{hw, 3 * l + 2}, per_layer), 1);
         gemv1(l, job(wptr(ctx, w.wdown[l]), nullptr, d, f, D.act, nullptr, D.hpub, d, EPI_ADD, per_layer,
-                     TagRef{hw, 3 * l + 3}), 1);
+                     TagRef{hw, 3 * l + 3}, l + 1 < L ? wptr(ctx, w.g1[l + 1]) : wptr(ctx, w.gf)), 1);
     }
     const TagRef once{1, 0};
-    int j0 = job(wptr(ctx, w.W0), nullptr, V, d, D.hpub, wptr(ctx, w.gf), D.logits0, V, EPI_STORE, TagRef{hw, 3 * L}, once);
+    int j0 = job(wptr(ctx, w.W0), nullptr, V, d, D.hpub, wptr(ctx, w.gf), D.logits0, V, EPI_STORE, TagRef{hw, 3 * L}, once, nullptr, 1);
     for (int i = 0; i < K; ++i)
         job(wptr(ctx, w.W1[i]), nullptr, d, d, D.hpub, wptr(ctx, w.gf), D.y + (size_t)i * M * d, d, EPI_HEADY,
             TagRef{hw, 3 * L}, once);
@@ -317,7 +320,7 @@ void build_tables(xsm_ctx *ctx) {
         j0 = (int)ctx->h_jobs.size();
         for (int i = 0; i < K; ++i)
             job(wptr(ctx, w.Wout[i]), nullptr, V, d, D.y + (size_t)i * M * d, nullptr, D.hlogits + (size_t)i * M * V, V,
-                EPI_STORE, once, once);
+                EPI_STORE, once, once, nullptr, 1);
         gemv1(-1, j0, K);
     }
     Stage s;
@@ -406,8 +409,12 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     };
     cudaError_t e;
     int grid = 0;
-    if ((e = step_kernel_setup(cfg->dtype, kSmemMax, &grid)) != cudaSuccess) return bail(e, "step kernel setup");
-    if (grid < 1) { delete ctx; return fail(nullptr, XSM_ERR_CUDA, "the step kernel does not fit on this device"); }
+    {
+        int dev = 0;
+        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return bail(e, "cudaGetDevice");
+        if ((e = cudaDeviceGetAttribute(&grid, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return bail(e, "device query");
+    }
+    if (grid < 1) { delete ctx; return fail(nullptr, XSM_ERR_CUDA, "no multiprocessors reported"); }
     ctx->sm_count = grid;
     // every CTA must own at least one row of every projection (the exchange protocol relies on it), and the
     // buffers that are sized per CTA bound the grid from above
@@ -457,6 +464,7 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     D.y = at<float>(ctx, L.y); D.logits0 = at<float>(ctx, L.logits0); D.hlogits = at<float>(ctx, L.hlogits);
     D.part = at<float>(ctx, L.part); D.cpart = at<float>(ctx, L.cpart);
     D.candx = at<uint32_t>(ctx, L.candx); D.header = at<uint32_t>(ctx, L.header); D.done = at<uint32_t>(ctx, L.done);
+    D.sspub = at<float>(ctx, L.sspub); D.gain_first = wptr(ctx, ctx->wo.g1[0]); D.grid = grid;
     D.kv_pool = ctx->ws + L.kv_pool; D.ckv_pool = ctx->ws + L.ckv_pool;
     *out = ctx;
     return XSM_OK;
@@ -480,6 +488,13 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
     int smem_bytes = 0;
     if (const char *m = plan_smem(c, batch, D, smem_bytes)) return fail(ctx, XSM_ERR_CAPACITY, m);
     ctx->smem_bytes = smem_bytes;
+    {   // the step kernel instance for this batch must fit one CTA per multiprocessor
+        Dev probe = D;
+        probe.M = batch * D.K1;
+        int resident = 0;
+        XSM_CUDA(ctx, step_kernel_setup(probe, c.dtype, smem_bytes, &resident));
+        if (resident < ctx->grid) return fail(ctx, XSM_ERR_CUDA, "the step kernel does not fit on this device");
+    }
     ctx->dc = *dc;
     ctx->batch = batch;
     D.B = batch; D.M = batch * D.K1;

@@ -1,0 +1,1746 @@
+// Kernels of the speculative decoding step (Algorithm 1, lines 3-12) for sm_100a.
+//
+// One decoding step is a fixed list of stages (projection, attention, ..., verify/resample, commit).  The
+// step kernel is persistent: one CTA per SM walks the whole list, and a launch may run many steps.
+//
+//  * Streaming.  Every byte that must come from HBM in a step (weight rows, cached keys and values, the
+//    condition's keys and values) has an address that is known when the step starts.  A producer warp walks
+//    the CTA's share of the step in order and pulls it into a ring of shared-memory slots with bulk copies
+//    (cp.async.bulk, completion on an mbarrier); eight consumer warps compute out of the ring.  HBM stays
+//    busy while the consumers wait for activations of the previous stage.
+//  * Exchange.  Activations travel between CTAs as fp32 words in global memory whose two lowest mantissa
+//    bits carry a tag that cycles with the write index of the buffer.  A consumer spins on the words it
+//    needs until they carry the expected tag: data and flag arrive in one L2 round trip, and no grid
+//    barrier exists.  A word is reused only after every reader of its previous content has produced data
+//    that the next writer has itself consumed (every CTA owns rows of every projection), so one copy of
+//    each buffer is enough.
+//  * Arithmetic.  bf16 weights: mma.sync.m16n8k16 with weight rows on M and the token rows on N, the
+//    fp32 activations split into bf16 hi + lo so that nothing that matters is lost; fp32 accumulation.
+//    fp32 weights: FMA.  Attention over the bf16 cache: flash-decoding with mma.sync, queries and
+//    probabilities as hi + lo pairs, base-2 online softmax, splits over keys merged by the last split.
+//  * Every wait is bounded.  When one runs out the CTA raises the status word; every CTA that sees it stops
+//    waiting on global memory, still drains its ring, and leaves at the end of the step.
+#pragma once
+#include "xsm_internal.h"
+
+#include <cuda_bf16.h>
+#include <math.h>
+
+namespace xsm {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int XSM_STATUS_TIMEOUT = 5, XSM_STATUS_CAPACITY = 3;
+constexpr unsigned kSpinLimit = 1u << 21;      // polls of a tagged word (each an L2 round trip)
+constexpr unsigned kMbarSpinLimit = 1u << 22;  // mbarrier try_wait calls
+constexpr float kNegBig = -1.0e30f;            // "no key seen yet" (finite: tags must not turn it into a NaN)
+constexpr float kLog2e = 1.4426950408889634f;
+
+// ------------------------------------------------------------------------------------------ helpers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint4 ld_relaxed_u4(const void *p) {
+    uint4 r;
+    asm volatile("ld.relaxed.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p) : "memory");
+    return r;
+}
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const void *p) {
+    uint32_t r;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(r) : "l"(p) : "memory");
+    return r;
+}
+__device__ __forceinline__ void st_relaxed_u32(void *p, uint32_t v) {
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint4 lds_u4(uint32_t a) {
+    uint4 r;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(a));
+    return r;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// global -> shared bulk copy; bytes and both addresses are multiples of 16
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Timeline of the first step of a launch, when the host asked for one: row 0 = the step's start, rows
+// 1 + 2p and 2 + 2p = stage p has its inputs / has published its outputs; one column per CTA.
+__device__ __forceinline__ void trace_mark(const Dev &D, int row) {
+    if (D.trace != nullptr && threadIdx.x == 0) D.trace[(size_t)row * gridDim.x + blockIdx.x] = global_ns();
+}
+
+// barrier among the consumer warps only (the producer warp never joins it)
+__device__ __forceinline__ void csync() { asm volatile("bar.sync 1, %0;" :: "n"(kConsumerThreads) : "memory"); }
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float silu_f(float v) { return v / (1.0f + expf(-v)); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// x = hi + lo with hi, lo bf16: 16 mantissa bits of x survive, products with bf16 weights stay exact in fp32.
+__device__ __forceinline__ void split_bf16(float x, unsigned &hi, unsigned &lo) {
+    bf16 h = __float2bfloat16_rn(x);
+    bf16 l = __float2bfloat16_rn(x - __bfloat162float(h));
+    hi = __bfloat16_as_ushort(h);
+    lo = __bfloat16_as_ushort(l);
+}
+// four values -> {hi01, hi23, lo01, lo23}
+__device__ __forceinline__ uint4 split4(float a, float b, float c, float d) {
+    unsigned h0, l0, h1, l1, h2, l2, h3, l3;
+    split_bf16(a, h0, l0); split_bf16(b, h1, l1); split_bf16(c, h2, l2); split_bf16(d, h3, l3);
+    return make_uint4(h0 | (h1 << 16), h2 | (h3 << 16), l0 | (l1 << 16), l2 | (l3 << 16));
+}
+
+// D = A(16x16, row) * B(16x8, col) + D, bf16 inputs, fp32 accumulate
+__device__ __forceinline__ void mma16816(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
+                                         unsigned b0, unsigned b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(unsigned (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(unsigned (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+// Philox4x32-10 (Salmon et al., SC'11): returns word 0.
+__device__ __forceinline__ uint32_t philox_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                                 uint32_t k1) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+        uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+        uint32_t n0 = h1 ^ c1 ^ k0, n2 = h0 ^ c3 ^ k1;
+        c0 = n0; c1 = l1; c2 = n2; c3 = l0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    return c0;
+}
+__device__ __forceinline__ uint32_t rand24(const Dev &D, int seq, uint32_t step, uint32_t slot, uint32_t purpose) {
+    return philox_word0(step, slot, purpose, 0u, D.key0 ^ (uint32_t)seq, D.key1) >> 8;
+}
+
+// ------------------------------------------------------------------------------------------- tags
+
+__device__ __forceinline__ uint32_t tag_of(uint32_t serial, TagRef r) { return 1u + (serial * (uint32_t)r.wps + (uint32_t)r.j) % 3u; }
+// the mantissa is rounded to 22 bits (to nearest, in magnitude) before the tag takes the two lowest bits
+__device__ __forceinline__ uint32_t tagged(float v, uint32_t tag) { return ((__float_as_uint(v) + 2u) & ~3u) | tag; }
+__device__ __forceinline__ float untag(uint32_t w) { return __uint_as_float(w & ~3u); }
+__device__ __forceinline__ bool tags_ok(const uint4 &v, uint32_t tag) {
+    return (((v.x ^ tag) | (v.y ^ tag) | (v.z ^ tag) | (v.w ^ tag)) & 3u) == 0u;
+}
+// integers travel as (value << 2) | tag
+__device__ __forceinline__ uint32_t tagged_int(int v, uint32_t tag) { return ((uint32_t)v << 2) | tag; }
+__device__ __forceinline__ int untag_int(uint32_t w) { return (int)(w >> 2); }
+
+// bf16 models: an activation travels as one word, bits 31..16 = hi = bf16(x), bits 15..2 = the leading bits of
+// lo = bf16(x - hi), bits 1..0 = tag (14 bits of mantissa survive; weights and cache have 8).  The reader gets
+// the two MMA operands by byte permutation, without arithmetic.  fp32 models publish tagged fp32 words.
+__device__ __forceinline__ uint32_t pack_act(float v, uint32_t tag) {
+    const bf16 h = __float2bfloat16_rn(v);
+    const bf16 l = __float2bfloat16_rn(v - __bfloat162float(h));
+    return ((uint32_t)__bfloat16_as_ushort(h) << 16) | ((uint32_t)__bfloat16_as_ushort(l) & 0xFFFCu) | tag;
+}
+__device__ __forceinline__ float unpack_act(uint32_t w) {
+    return __uint_as_float(w & 0xFFFF0000u) + __uint_as_float((w & 0xFFFCu) << 16);
+}
+template <typename WT> __device__ __forceinline__ uint32_t publish_word(float v, uint32_t tag, bool plain) {
+    return (sizeof(WT) == 2 && !plain) ? pack_act(v, tag) : tagged(v, tag);
+}
+template <typename WT> __device__ __forceinline__ float read_word(uint32_t w) {
+    return sizeof(WT) == 2 ? unpack_act(w) : untag(w);
+}
+
+// Per-CTA control block in shared memory (after the barriers).
+struct Ctl {
+    volatile int dead;          // a wait ran out somewhere: stop waiting on global memory
+    int go;                     // written by the consumers before they release the producer for a step
+    int trace_row;              // row of the timeline that the running stage fills when its inputs are in (0: off)
+    int len[kMaxBatch];
+    int flags[kMaxBatch];       // 1 finished, 2 ingesting
+    unsigned char row_dead[kMaxTokens];   // token rows of finished sequences (not fetched, read as zeros)
+};
+
+struct Smem {
+    uint32_t full0, empty0, go_bar;   // shared-space addresses of full[0], empty[0], go
+    Ctl *ctl;
+    char *ring;
+    char *acts;
+    float *ss;                        // [kMaxTokens] sum of squares / 1 / rms
+    float *sspart;                    // warp partial sums of squares of the chunk being staged
+    int n_slots;
+};
+
+
+__device__ __forceinline__ Smem carve(char *smem, const Dev &D) {
+    Smem s;
+    s.full0 = smem_u32(smem);
+    s.empty0 = s.full0 + 8u * kMaxSlots;
+    s.go_bar = s.empty0 + 8u * kMaxSlots;
+    s.ctl = reinterpret_cast<Ctl *>(smem + 256);   // 2 * 12 * 8 + 8 = 200 bytes of barriers before it
+    s.ring = smem + kSmemHeader;
+    s.n_slots = D.n_slots;
+    s.acts = s.ring + (size_t)D.n_slots * kSlotBytes;
+    s.ss = reinterpret_cast<float *>(s.acts + D.acts_bytes);
+    s.sspart = s.ss + kMaxTokens;
+    return s;
+}
+static_assert(256 + sizeof(Ctl) <= kSmemHeader, "control block overflows the header");
+
+__device__ __forceinline__ void raise_timeout(const Dev &D, Ctl *ctl) {
+    atomicExch(D.status, XSM_STATUS_TIMEOUT);
+    ctl->dead = 1;
+}
+
+// Spins until the four words at p carry `tag`.  Gives up when the CTA is dead or the status word is raised.
+__device__ __forceinline__ uint4 poll_u4(const Dev &D, Ctl *ctl, const void *p, uint32_t tag) {
+    uint4 v = ld_relaxed_u4(p);
+    unsigned it = 0;
+    while (!tags_ok(v, tag)) {
+        if (ctl->dead) break;
+        if (++it > kSpinLimit) { raise_timeout(D, ctl); break; }
+        if ((it & 1023u) == 0u && ld_relaxed_u32(D.status) != 0u) { ctl->dead = 1; break; }
+        v = ld_relaxed_u4(p);
+    }
+    return v;
+}
+__device__ __forceinline__ uint32_t poll_u32(const Dev &D, Ctl *ctl, const void *p, uint32_t tag) {
+    uint32_t v = ld_relaxed_u32(p);
+    unsigned it = 0;
+    while ((v & 3u) != tag) {
+        if (ctl->dead) break;
+        if (++it > kSpinLimit) { raise_timeout(D, ctl); break; }
+        if ((it & 1023u) == 0u && ld_relaxed_u32(D.status) != 0u) { ctl->dead = 1; break; }
+        v = ld_relaxed_u32(p);
+    }
+    return v;
+}
+
+// ------------------------------------------------------------------------------------------- ring
+
+struct Ring {
+    uint32_t pos;   // items passed so far (same sequence on the producer and on every consumer warp)
+};
+__device__ __forceinline__ uint32_t ring_slot(const Smem &S, uint32_t pos) { return pos % (uint32_t)S.n_slots; }
+__device__ __forceinline__ uint32_t ring_parity(const Smem &S, uint32_t pos) { return (pos / (uint32_t)S.n_slots) & 1u; }
+
+__device__ __forceinline__ void mbar_wait(const Dev &D, Ctl *ctl, uint32_t bar, uint32_t parity) {
+    for (unsigned it = 0; it < kMbarSpinLimit; ++it)
+        if (mbar_try_wait(bar, parity)) return;
+    raise_timeout(D, ctl);
+}
+
+// consumer: wait until the item at ring position r.pos has landed; returns its slot
+__device__ __forceinline__ char *ring_wait(const Dev &D, const Smem &S, const Ring &r) {
+    const uint32_t slot = ring_slot(S, r.pos);
+    mbar_wait(D, S.ctl, S.full0 + 8u * slot, ring_parity(S, r.pos));
+    return S.ring + (size_t)slot * kSlotBytes;
+}
+// consumer (whole warp): done with the item
+__device__ __forceinline__ void ring_release(const Smem &S, Ring &r) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(S.empty0 + 8u * ring_slot(S, r.pos));
+    r.pos += 1;
+}
+// producer (lane 0 decides, the warp follows): claim the next slot, announce `bytes`
+__device__ __forceinline__ void ring_claim(const Dev &D, const Smem &S, const Ring &r, uint32_t bytes, uint32_t &dst,
+                                           uint32_t &bar) {
+    const uint32_t slot = ring_slot(S, r.pos);
+    bar = S.full0 + 8u * slot;
+    dst = smem_u32(S.ring + (size_t)slot * kSlotBytes);
+    if ((threadIdx.x & 31) == 0) {
+        mbar_wait(D, S.ctl, S.empty0 + 8u * slot, ring_parity(S, r.pos) ^ 1u);
+        mbar_arrive_expect_tx(bar, bytes);
+    }
+    __syncwarp();
+}
+
+// ------------------------------------------------------------------------------ projection: plan
+
+// The rows of a stage's jobs form one range that is cut evenly over the CTAs; a CTA's piece of one job is a
+// segment.  A segment is processed as tile groups of up to 8 tiles (a tile: 16 weight rows, or 8 gate rows
+// + 8 up rows), the activations in chunks of D.kca columns, a tile in items of at most kItemRowBytes per row.
+struct SegPlan {
+    int tile_units;   // units (output rows) per tile: 16, or 8 for gate/up
+    int n_tiles;
+    int ksub;         // columns per item
+};
+template <typename WT> __device__ __forceinline__ SegPlan seg_plan(const GemvJob &J, int lo, int hi) {
+    SegPlan p;
+    p.tile_units = J.epi == EPI_GATEUP ? 8 : 16;
+    p.n_tiles = (hi - lo + p.tile_units - 1) / p.tile_units;
+    p.ksub = kItemRowBytes / (int)sizeof(WT);
+    return p;
+}
+
+// ---------------------------------------------------------------------------- projection: producer
+
+template <typename WT>
+static __device__ void produce_segment(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi) {
+    const SegPlan p = seg_plan<WT>(J, lo, hi);
+    const int lane = threadIdx.x & 31;
+    const int kca = min(J.kdim, D.kca);
+    for (int tg0 = 0; tg0 < p.n_tiles; tg0 += kConsumerWarps) {
+        const int tg = min(kConsumerWarps, p.n_tiles - tg0);
+        for (int ac0 = 0; ac0 < J.kdim; ac0 += kca) {
+            const int acw = min(kca, J.kdim - ac0);
+            for (int t = 0; t < tg; ++t) {
+                const int u0 = lo + (tg0 + t) * p.tile_units, nu = min(p.tile_units, hi - u0);
+                for (int sc = 0; sc < acw; sc += p.ksub) {
+                    const int kw = min(p.ksub, acw - sc), k0 = ac0 + sc;
+                    const uint32_t row_bytes = (uint32_t)kw * (uint32_t)sizeof(WT);
+                    const int nrows = J.epi == EPI_GATEUP ? 2 * nu : nu;
+                    uint32_t dst, bar;
+                    ring_claim(D, S, ring, row_bytes * (uint32_t)nrows, dst, bar);
+                    if (lane < 16) {
+                        const WT *src = nullptr;
+                        if (J.epi == EPI_GATEUP) {
+                            const int i = lane & 7;
+                            if (i < nu) src = reinterpret_cast<const WT *>(lane < 8 ? J.W : J.W2) + (size_t)(u0 + i) * J.kdim + k0;
+                        } else if (lane < nu) {
+                            src = reinterpret_cast<const WT *>(J.W) + (size_t)(u0 + lane) * J.kdim + k0;
+                        }
+                        if (src) bulk_g2s(dst + (uint32_t)lane * kRowPitch, src, row_bytes, bar);
+                    }
+                    ring.pos += 1;
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------- projection: consumer
+
+// Stages columns [ac0, ac0+acw) of the tagged input of job J into shared memory: polls the words, strips the
+// tags, accumulates the sum of squares of every row, applies the RMSNorm gain, and stores bf16 hi+lo pairs
+// (bf16 weights) or fp32 (fp32 weights), 16 bytes per 4 columns, rows (acw*4 + 16) bytes apart.  Rows of
+// finished sequences are filled with zeros without waiting.
+template <typename WT> __device__ __forceinline__ float4 load_gain4(const WT *gain, int k);
+template <> __device__ __forceinline__ float4 load_gain4<float>(const float *gain, int k) {
+    return __ldg(reinterpret_cast<const float4 *>(gain + k));
+}
+template <> __device__ __forceinline__ float4 load_gain4<bf16>(const bf16 *gain, int k) {
+    const uint2 u = __ldg(reinterpret_cast<const uint2 *>(gain + k));
+    return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                       __uint_as_float(u.y & 0xffff0000u));
+}
+
+constexpr int kPollBatch = 8;   // tagged 16-byte loads a thread keeps in flight
+
+// walks the (row, 16-byte word) pairs of a staging pass without dividing: thread t starts at word t of row 0
+struct RowWalk {
+    int m, c4;
+    __device__ __forceinline__ RowWalk(int tid, int v4_per_row) { m = tid / v4_per_row; c4 = tid - m * v4_per_row; }
+    __device__ __forceinline__ void next(int v4_per_row) {
+        c4 += kConsumerThreads;
+        while (c4 >= v4_per_row) { c4 -= v4_per_row; ++m; }
+    }
+};
+
+template <typename WT>
+static __device__ void stage_acts(const Dev &D, const Smem &S, const GemvJob &J, int ac0, int acw, uint32_t tag);
+
+// fp32 models: tagged fp32 words in, fp32 out; the reader applies the gain and sums the squares.
+template <>
+__device__ void stage_acts<float>(const Dev &D, const Smem &S, const GemvJob &J, int ac0, int acw, uint32_t tag) {
+    const int M = D.M, tid = threadIdx.x;
+    const int v4_per_row = acw >> 2, total = M * v4_per_row;
+    const int pitch = acw * 4 + 16;
+    const float *gain = reinterpret_cast<const float *>(J.gain);
+    const float *x = J.x;
+    const int kdim = J.kdim;
+    const bool first = ac0 == 0;
+    RowWalk rd(tid, v4_per_row), wr(tid, v4_per_row);
+    for (int i0 = 0; i0 < total; i0 += kConsumerThreads * kPollBatch) {
+        uint4 w[kPollBatch];
+        float4 gn[kPollBatch];
+        // issue every load of the batch before looking at any of them
+#pragma unroll
+        for (int u = 0; u < kPollBatch; ++u) {
+            w[u] = make_uint4(tag, tag, tag, tag);          // rows that are not fetched read as zeros
+            gn[u] = make_float4(1.f, 1.f, 1.f, 1.f);
+            if (rd.m < M) {
+                const int k = ac0 + (rd.c4 << 2);
+                if (!S.ctl->row_dead[rd.m]) w[u] = ld_relaxed_u4(x + (size_t)rd.m * kdim + k);
+                if (gain != nullptr) gn[u] = load_gain4<float>(gain, k);
+            }
+            rd.next(v4_per_row);
+        }
+#pragma unroll
+        for (int u = 0; u < kPollBatch; ++u) {
+            const int i = i0 + u * kConsumerThreads + tid;
+            float ssq = 0.f;
+            if (wr.m < M) {
+                if (!tags_ok(w[u], tag)) w[u] = poll_u4(D, S.ctl, x + (size_t)wr.m * kdim + ac0 + (wr.c4 << 2), tag);
+                float4 v = make_float4(untag(w[u].x), untag(w[u].y), untag(w[u].z), untag(w[u].w));
+                if (gain != nullptr) {
+                    ssq = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+                    v.x *= gn[u].x; v.y *= gn[u].y; v.z *= gn[u].z; v.w *= gn[u].w;
+                }
+                *reinterpret_cast<float4 *>(S.acts + (size_t)wr.m * pitch + ((size_t)wr.c4 << 4)) = v;
+            }
+            if (gain != nullptr && i0 + u * kConsumerThreads < total) {
+                // acw is a multiple of 128: the 32 lanes of a warp hold words of one row
+                ssq = warp_sum(ssq);
+                if ((tid & 31) == 0 && i < total) S.sspart[i >> 5] = ssq;
+            }
+            wr.next(v4_per_row);
+        }
+    }
+    csync();
+    if (gain != nullptr && tid < M) {   // deterministic: fixed slots, fixed order
+        const int per_row = v4_per_row >> 5;
+        float s = first ? 0.f : S.ss[tid];
+        for (int q = 0; q < per_row; ++q) s += S.sspart[tid * per_row + q];
+        S.ss[tid] = s;
+    }
+    // the next csync() of the caller orders ss before its readers
+}
+
+// bf16 models: packed hi + lo words in (gain already applied by the writer), {hi01, hi23, lo01, lo23} out; the
+// sum of squares of a normed input arrives as one partial per writer CTA.
+template <>
+__device__ void stage_acts<bf16>(const Dev &D, const Smem &S, const GemvJob &J, int ac0, int acw, uint32_t tag) {
+    const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int v4_per_row = acw >> 2, total = M * v4_per_row;
+    const int pitch = acw * 4 + 16;
+    const float *x = J.x;
+    const int kdim = J.kdim;
+    RowWalk rd(tid, v4_per_row), wr(tid, v4_per_row);
+    for (int i0 = 0; i0 < total; i0 += kConsumerThreads * kPollBatch) {
+        uint4 w[kPollBatch];
+#pragma unroll
+        for (int u = 0; u < kPollBatch; ++u) {
+            w[u] = make_uint4(tag, tag, tag, tag);
+            if (rd.m < M && !S.ctl->row_dead[rd.m]) w[u] = ld_relaxed_u4(x + (size_t)rd.m * kdim + ac0 + (rd.c4 << 2));
+            rd.next(v4_per_row);
+        }
+#pragma unroll
+        for (int u = 0; u < kPollBatch; ++u) {
+            if (wr.m < M) {
+                if (!tags_ok(w[u], tag)) w[u] = poll_u4(D, S.ctl, x + (size_t)wr.m * kdim + ac0 + (wr.c4 << 2), tag);
+                uint4 o;
+                o.x = __byte_perm(w[u].x, w[u].y, 0x7632);
+                o.y = __byte_perm(w[u].z, w[u].w, 0x7632);
+                o.z = __byte_perm(w[u].x, w[u].y, 0x5410) & 0xFFFCFFFCu;
+                o.w = __byte_perm(w[u].z, w[u].w, 0x5410) & 0xFFFCFFFCu;
+                *reinterpret_cast<uint4 *>(S.acts + (size_t)wr.m * pitch + ((size_t)wr.c4 << 4)) = o;
+            }
+            wr.next(v4_per_row);
+        }
+    }
+    if (J.gain != nullptr && ac0 == 0) {
+        // sum of squares of row m = sum over the writer CTAs' shares, one warp per row, fixed order
+        const int G = (int)gridDim.x;
+        for (int m = warp; m < M; m += kConsumerWarps) {
+            float s = 0.f;
+            if (!S.ctl->row_dead[m]) {
+                uint32_t v[8];            // G <= 256: at most 8 shares per lane, all requested at once
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int c = lane + 32 * q;
+                    v[q] = c < G ? ld_relaxed_u32(D.sspub + (size_t)c * M + m) : tag;
+                }
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int c = lane + 32 * q;
+                    if (c < G && (v[q] & 3u) != tag) v[q] = poll_u32(D, S.ctl, D.sspub + (size_t)c * M + m, tag);
+                    s += untag(v[q]);
+                }
+            }
+            s = warp_sum(s);
+            if (lane == 0) S.ss[m] = s;
+        }
+    }
+    csync();
+}
+
+// bf16 weights.  Warp (tile, part): A = 16 weight rows x 32 columns per step out of the ring slot (lane
+// g = lane/4, t = lane%4 loads 16 bytes = 8 consecutive columns of rows g and g+8; the same column
+// permutation is applied to the activation fragments, so the products pair up), B = activations of 8 tokens.
+template <int NT>
+__device__ __forceinline__ void mma_item_bf16(const char *slot, const char *acts, int pitch, int kcol0, int kw, int part,
+                                              int parts, int M, float (&acc)[NT][2][4]) {
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const uint32_t wa_addr = smem_u32(slot) + (uint32_t)g * kRowPitch + (uint32_t)t * 16u;
+    const uint32_t wb_addr = wa_addr + 8u * kRowPitch;
+    const uint32_t x_addr = smem_u32(acts) + (uint32_t)(kcol0 + t * 8) * 4u;
+    const int nkb = kw >> 5;
+    for (int kb = part; kb < nkb; kb += parts) {
+        const uint4 wa = lds_u4(wa_addr + (uint32_t)kb * 64u), wb = lds_u4(wb_addr + (uint32_t)kb * 64u);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int m = nt * 8 + g;
+            uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = xa;
+            if (m < M) {
+                const uint32_t a = x_addr + (uint32_t)m * (uint32_t)pitch + (uint32_t)kb * 128u;
+                xa = lds_u4(a);
+                xb = lds_u4(a + 16u);
+            }
+            mma16816(acc[nt][0], wa.x, wb.x, wa.y, wb.y, xa.x, xa.y);
+            mma16816(acc[nt][1], wa.x, wb.x, wa.y, wb.y, xa.z, xa.w);
+            mma16816(acc[nt][0], wa.z, wb.z, wa.w, wb.w, xb.x, xb.y);
+            mma16816(acc[nt][1], wa.z, wb.z, wa.w, wb.w, xb.z, xb.w);
+        }
+    }
+}
+
+// What one output element becomes (after the dot product v, already scaled by 1/rms when the job has a gain).
+// hprev: the residual stream's value when the caller has fetched it ahead (have_prev), EPI_ADD only.
+// Returns the value before any gain of the next stage is applied (the residual stream's new value for EPI_ADD).
+template <typename WT>
+__device__ __forceinline__ float epilogue_store(const GemvJob &J, int m, int u, float v, float v2, float inv, uint32_t tag_out,
+                                                bool have_prev = false, float hprev = 0.f) {
+    float *o = J.out + (size_t)m * J.out_ld + u;
+    float r, pub;
+    if (J.epi == EPI_STORE) pub = r = v;
+    else if (J.epi == EPI_GATEUP) pub = r = silu_f(v) * v2;
+    else if (J.epi == EPI_ADD) {
+        float *hm = J.hm + (size_t)m * J.out_ld + u;
+        pub = r = (have_prev ? hprev : __ldcg(hm)) + v;
+        __stcg(hm, r);
+        // bf16 models: the reader's RMSNorm gain is applied here, once, instead of by every reader
+        if (sizeof(WT) == 2 && J.gain_out != nullptr) pub = r * to_f(reinterpret_cast<const WT *>(J.gain_out)[u]);
+    } else {   // EPI_HEADY: residual on the normalised input (this CTA has already waited for that word);
+               // inv = 1 / rms(x[m]), times gain[u] where the input is published without its gain (fp32 models)
+        pub = r = read_word<WT>(ld_relaxed_u32(J.x + (size_t)m * J.kdim + u)) * inv + silu_f(v);
+    }
+    st_relaxed_u32(o, publish_word<WT>(pub, tag_out, J.out_plain != 0));
+    return r;
+}
+
+template <typename WT, int NT>
+static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi,
+                                     uint32_t serial) {
+    const SegPlan p = seg_plan<WT>(J, lo, hi);
+    const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int kca = min(J.kdim, D.kca);
+    const bool one_chunk = kca >= J.kdim;
+    const uint32_t tag_in = tag_of(serial, J.in), tag_out = tag_of(serial, J.outt);
+    const WT *gain = reinterpret_cast<const WT *>(J.gain);
+    constexpr int NP = NT * 8;
+    bool staged = false;
+    float ss_share = 0.f;
+    for (int tg0 = 0; tg0 < p.n_tiles; tg0 += kConsumerWarps) {
+        const int tg = min(kConsumerWarps, p.n_tiles - tg0);
+        const int parts = kConsumerWarps / tg;
+        const int my_tile = warp / parts, my_part = warp - my_tile * parts;   // my_tile >= tg: idle warp
+        float acc[NT][2][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[nt][0][q] = acc[nt][1][q] = 0.f;
+        // the residual stream's old values of this group's outputs, fetched while the inputs are awaited
+        const int outs = tg * p.tile_units * M;     // (tile, token, unit)
+        float hpre[4] = {0.f, 0.f, 0.f, 0.f};
+        if (J.epi == EPI_ADD) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int i = tid + q * kConsumerThreads;
+                if (i < outs) {
+                    const int tl = i / (p.tile_units * M), rem = i - tl * p.tile_units * M;
+                    const int n = rem / p.tile_units, u = lo + (tg0 + tl) * p.tile_units + rem - n * p.tile_units;
+                    if (u < hi) hpre[q] = __ldcg(J.hm + (size_t)n * J.out_ld + u);
+                }
+            }
+        }
+        for (int ac0 = 0; ac0 < J.kdim; ac0 += kca) {
+            const int acw = min(kca, J.kdim - ac0), pitch = acw * 4 + 16;
+            if (!(one_chunk && staged)) {
+                csync();                       // everyone is done with the previous content of the area
+                stage_acts<WT>(D, S, J, ac0, acw, tag_in);
+                csync();
+                staged = true;
+                if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
+            }
+            for (int tl = 0; tl < tg; ++tl) {
+                for (int sc = 0; sc < acw; sc += p.ksub) {
+                    const int kw = min(p.ksub, acw - sc);
+                    const char *slot = ring_wait(D, S, ring);
+                    if (tl == my_tile) mma_item_bf16<NT>(slot, S.acts, pitch, sc, kw, my_part, parts, M, acc);
+                    ring_release(S, ring);
+                }
+            }
+        }
+        // cross-warp reduction through the activation area, then the epilogue
+        csync();
+        float *red = reinterpret_cast<float *>(S.acts);   // [warp][NP][16]
+        staged = false;
+        if (my_tile < tg) {
+            float *r = red + (size_t)warp * NP * 16;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const int n0 = nt * 8 + 2 * t;
+                r[n0 * 16 + g] = acc[nt][0][0] + acc[nt][1][0];
+                r[(n0 + 1) * 16 + g] = acc[nt][0][1] + acc[nt][1][1];
+                r[n0 * 16 + g + 8] = acc[nt][0][2] + acc[nt][1][2];
+                r[(n0 + 1) * 16 + g + 8] = acc[nt][0][3] + acc[nt][1][3];
+            }
+        }
+        if (gain != nullptr && tid < M) S.ss[tid] = 1.0f / sqrtf(S.ss[tid] / (float)J.kdim + D.eps);   // restaged, hence raw, in every tile group
+        csync();
+        float *hv = red + (size_t)kConsumerWarps * NP * 16;    // new values of the residual stream, for their squares
+        const bool want_ss = J.epi == EPI_ADD && J.gain_out != nullptr;
+        for (int i = tid; i < outs; i += kConsumerThreads) {
+            const int tl = i / (p.tile_units * M), rem = i - tl * p.tile_units * M;
+            const int n = rem / p.tile_units, ui = rem - n * p.tile_units;
+            const int u = lo + (tg0 + tl) * p.tile_units + ui;
+            float r = 0.f;
+            if (u < hi) {
+                float v = 0.f, v2 = 0.f;
+                for (int q = 0; q < parts; ++q) {
+                    const float *rr = red + (size_t)(tl * parts + q) * NP * 16 + n * 16;
+                    v += rr[ui];
+                    if (J.epi == EPI_GATEUP) v2 += rr[ui + 8];
+                }
+                float inv = 1.f;
+                if (gain != nullptr) { inv = S.ss[n]; v *= inv; v2 *= inv; }
+                const int q = (i - tid) / kConsumerThreads;
+                r = epilogue_store<WT>(J, n, u, v, v2, inv, tag_out, q < 4, q == 0 ? hpre[0] : q == 1 ? hpre[1] : q == 2 ? hpre[2] : hpre[3]);
+            }
+            if (want_ss) hv[i] = r;
+        }
+        if (want_ss) {
+            // this CTA's share of the sum of squares of every row, in a fixed order
+            csync();
+            if (tid < M) {
+                for (int tl = 0; tl < tg; ++tl)
+                    for (int ui = 0; ui < p.tile_units; ++ui) {
+                        const float r = hv[(tl * M + tid) * p.tile_units + ui];
+                        ss_share = fmaf(r, r, ss_share);
+                    }
+                if (tg0 + kConsumerWarps >= p.n_tiles) st_relaxed_u32(D.sspub + (size_t)blockIdx.x * M + tid, tagged(ss_share, tag_out));
+            }
+        }
+    }
+}
+
+// fp32 weights: the 16 rows of a tile form 8 pairs (q, q+8) (for gate/up: the gate and the up row of unit q);
+// warp w owns pairs w, w + kConsumerWarps, ...; lanes stride over the columns; the activations of all tokens
+// must fit the staging area in one chunk.
+template <int MT>
+__device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi,
+                                    uint32_t serial) {
+    constexpr int PPW = (8 + kConsumerWarps - 1) / kConsumerWarps;   // pairs per warp
+    const SegPlan p = seg_plan<float>(J, lo, hi);
+    const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t tag_in = tag_of(serial, J.in), tag_out = tag_of(serial, J.outt);
+    const float *gain = reinterpret_cast<const float *>(J.gain);
+    const int pitch = J.kdim * 4 + 16;
+    csync();
+    stage_acts<float>(D, S, J, 0, J.kdim, tag_in);
+    csync();
+    if (gain != nullptr && tid < M) S.ss[tid] = 1.0f / sqrtf(S.ss[tid] / (float)J.kdim + D.eps);
+    csync();
+    for (int tl = 0; tl < p.n_tiles; ++tl) {
+        float acc[PPW][2][MT];
+#pragma unroll
+        for (int s = 0; s < PPW; ++s)
+#pragma unroll
+            for (int n = 0; n < MT; ++n) acc[s][0][n] = acc[s][1][n] = 0.f;
+        for (int sc = 0; sc < J.kdim; sc += p.ksub) {
+            const int kw = min(p.ksub, J.kdim - sc);
+            const char *slot = ring_wait(D, S, ring);
+#pragma unroll
+            for (int s = 0; s < PPW; ++s) {
+                const int q = warp + s * kConsumerWarps;
+                if (q < 8) {
+                    const float *ra = reinterpret_cast<const float *>(slot + (size_t)q * kRowPitch);
+                    const float *rb = reinterpret_cast<const float *>(slot + (size_t)(q + 8) * kRowPitch);
+                    for (int k = lane * 4; k < kw; k += 128) {
+                        const float4 wa = *reinterpret_cast<const float4 *>(ra + k), wb = *reinterpret_cast<const float4 *>(rb + k);
+#pragma unroll
+                        for (int n = 0; n < MT; ++n) {
+                            if (n < M) {
+                                const float4 x = *reinterpret_cast<const float4 *>(S.acts + (size_t)n * pitch + (size_t)(sc + k) * 4);
+                                acc[s][0][n] = fmaf(wa.x, x.x, acc[s][0][n]); acc[s][0][n] = fmaf(wa.y, x.y, acc[s][0][n]);
+                                acc[s][0][n] = fmaf(wa.z, x.z, acc[s][0][n]); acc[s][0][n] = fmaf(wa.w, x.w, acc[s][0][n]);
+                                acc[s][1][n] = fmaf(wb.x, x.x, acc[s][1][n]); acc[s][1][n] = fmaf(wb.y, x.y, acc[s][1][n]);
+                                acc[s][1][n] = fmaf(wb.z, x.z, acc[s][1][n]); acc[s][1][n] = fmaf(wb.w, x.w, acc[s][1][n]);
+                            }
+                        }
+                    }
+                }
+            }
+            ring_release(S, ring);
+        }
+        const int u0 = lo + tl * p.tile_units;
+#pragma unroll
+        for (int s = 0; s < PPW; ++s) {
+            const int q = warp + s * kConsumerWarps;
+            if (q >= 8) continue;
+#pragma unroll
+            for (int n = 0; n < MT; ++n) {
+                if (n < M) {
+                    float va = warp_sum(acc[s][0][n]), vb = warp_sum(acc[s][1][n]);
+                    if (lane == 0) {
+                        const float inv = gain != nullptr ? S.ss[n] : 1.f;
+                        va *= inv; vb *= inv;
+                        if (J.epi == EPI_GATEUP) {
+                            if (u0 + q < hi) epilogue_store<float>(J, n, u0 + q, va, vb, inv, tag_out);
+                        } else {
+                            if (u0 + q < hi)
+                                epilogue_store<float>(J, n, u0 + q, va, 0.f, J.epi == EPI_HEADY ? inv * gain[u0 + q] : inv, tag_out);
+                            if (u0 + q + 8 < hi)
+                                epilogue_store<float>(J, n, u0 + q + 8, vb, 0.f, J.epi == EPI_HEADY ? inv * gain[u0 + q + 8] : inv, tag_out);
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
+// NTM: token tiles of 8 (bf16 weights) or token rows (fp32 weights) the kernel is compiled for
+template <typename WT, int NTM> struct ConsumeSegment;
+template <int NTM> struct ConsumeSegment<bf16, NTM> {
+    static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi, uint32_t serial) {
+        consume_segment_bf16<bf16, NTM>(D, S, ring, J, lo, hi, serial);
+    }
+};
+template <int NTM> struct ConsumeSegment<float, NTM> {
+    static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi, uint32_t serial) {
+        consume_segment_f32<NTM>(D, S, ring, J, lo, hi, serial);
+    }
+};
+
+// A projection stage, seen by the producer warp (PRODUCER) or by the consumer warps.
+template <typename WT, int NTM, bool PRODUCER>
+static __device__ void gemv_stage(const Dev &D, const Smem &S, Ring &ring, const Stage &st, uint32_t serial) {
+    long long total = 0;
+    for (int j = 0; j < st.njobs; ++j) total += D.jobs[st.job0 + j].rows;
+    const long long u_lo = total * blockIdx.x / gridDim.x, u_hi = total * (blockIdx.x + 1) / gridDim.x;
+    long long base = 0;
+    for (int j = 0; j < st.njobs; ++j) {
+        const GemvJob &J = D.jobs[st.job0 + j];
+        const long long lo = max(u_lo - base, 0LL), hi = min(u_hi - base, (long long)J.rows);
+        if (lo < hi) {
+            if (PRODUCER) produce_segment<WT>(D, S, ring, J, (int)lo, (int)hi);
+            else ConsumeSegment<WT, NTM>::run(D, S, ring, J, (int)lo, (int)hi, serial);
+        }
+        base += J.rows;
+    }
+}
+
+// -------------------------------------------------------------------------------- attention: plan
+
+// Cache tiles.  One (page, head) tile holds P rows (positions) of dh elements.  bf16 tiles are stored with
+// their 16-byte chunks permuted so that ldmatrix over 8 consecutive rows touches every bank once; fp32
+// tiles are stored plain.
+template <typename KVT>
+__device__ __forceinline__ KVT *kv_tile(const Dev &D, void *pool, int pool_pages, int layer, int kv, int page, int head) {
+    return reinterpret_cast<KVT *>(pool) + ((((size_t)layer * 2 + kv) * pool_pages + page) * D.H + head) * (size_t)D.P * D.dh;
+}
+// physical 16-byte chunk of logical chunk c of row r, rows of row_bytes
+__device__ __forceinline__ int swz(int r, int c, int row_bytes) {
+    return row_bytes >= 128 ? (c ^ (r & 7)) : (c ^ ((r >> 1) & 3));
+}
+// element offset of (row r, element e) inside a tile
+template <typename KVT> __device__ __forceinline__ size_t tile_off(int r, int e, int dh);
+template <> __device__ __forceinline__ size_t tile_off<float>(int r, int e, int dh) { return (size_t)r * dh + e; }
+template <> __device__ __forceinline__ size_t tile_off<bf16>(int r, int e, int dh) {
+    return (size_t)r * dh + (size_t)swz(r, e >> 3, dh * 2) * 8 + (e & 7);
+}
+
+struct AttnItem { int b, h, s, S; };
+
+// number of key splits of sequence b's self-attention this step
+__device__ __forceinline__ int self_splits(const Dev &D, int len) {
+    const int np = (len + D.P - 1) / D.P;
+    return min(max((np + 3) / 4, 1), D.S_max);
+}
+// the idx-th live item of the stage (sequences that are finished have none); false when idx is past the end
+__device__ __forceinline__ bool attn_item_at(const Dev &D, const Ctl *ctl, bool cross, int idx, AttnItem &it) {
+    for (int b = 0; b < D.B; ++b) {
+        if (ctl->flags[b] & 1) continue;
+        const int S = cross ? D.S_cross : self_splits(D, ctl->len[b]);
+        const int n = D.H * S;
+        if (idx < n) { it.b = b; it.h = idx / S; it.s = idx - it.h * S; it.S = S; return true; }
+        idx -= n;
+    }
+    return false;
+}
+// pages [p_lo, p_hi) of cached keys that split s of S covers
+__device__ __forceinline__ void split_pages(int n_keys, int P, int s, int S, int &p_lo, int &p_hi) {
+    const int np = (n_keys + P - 1) / P, pp = (np + S - 1) / S;
+    p_lo = min(np, s * pp);
+    p_hi = min(np, (s + 1) * pp);
+}
+
+// ---------------------------------------------------------------------------- attention: producer
+
+template <typename KVT>
+static __device__ void produce_attn(const Dev &D, const Smem &S, Ring &ring, const Stage &st) {
+    if (sizeof(KVT) != 2) return;   // the fp32 cache is read straight from global memory
+    const bool cross = st.kind == ST_ATTN_CROSS;
+    const int lane = threadIdx.x & 31;
+    void *pool = cross ? D.ckv_pool : D.kv_pool;
+    const int pool_pages = cross ? D.B * D.cpages : D.n_pages;
+    AttnItem it;
+    for (int idx = blockIdx.x; attn_item_at(D, S.ctl, cross, idx, it); idx += gridDim.x) {
+        int p_lo, p_hi;
+        split_pages(cross ? D.C : S.ctl->len[it.b], D.P, it.s, it.S, p_lo, p_hi);
+        for (int pg = p_lo; pg < p_hi; ++pg) {
+            const int page = cross ? it.b * D.cpages + pg : __ldcg(D.block_table + (size_t)it.b * D.max_blocks + pg);
+            const KVT *kt = kv_tile<KVT>(D, pool, pool_pages, st.layer, 0, page, it.h);
+            const KVT *vt = kv_tile<KVT>(D, pool, pool_pages, st.layer, 1, page, it.h);
+            uint32_t dst, bar;
+            if (D.kv_one_item) {
+                ring_claim(D, S, ring, 2u * (uint32_t)D.tile_bytes, dst, bar);
+                if (lane == 0) bulk_g2s(dst, kt, (uint32_t)D.tile_bytes, bar);
+                if (lane == 1) bulk_g2s(dst + (uint32_t)D.tile_bytes, vt, (uint32_t)D.tile_bytes, bar);
+                ring.pos += 1;
+            } else {
+                ring_claim(D, S, ring, (uint32_t)D.tile_bytes, dst, bar);
+                if (lane == 0) bulk_g2s(dst, kt, (uint32_t)D.tile_bytes, bar);
+                ring.pos += 1;
+                ring_claim(D, S, ring, (uint32_t)D.tile_bytes, dst, bar);
+                if (lane == 0) bulk_g2s(dst, vt, (uint32_t)D.tile_bytes, bar);
+                ring.pos += 1;
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------- attention: consumer
+
+// Shared-memory plan of an attention item inside the activation area (K1 <= 16 query rows).
+template <int DH> struct AttnSmem {
+    static constexpr int QP = DH + 8;                 // bf16 elements between query rows (16 bytes of padding)
+    bf16 *qh, *ql;                                    // [16][QP] rotated, scaled queries as hi + lo (rows >= K1 zero)
+    float *qf, *kw, *vw;                              // [K1][DH] fp32: queries, window keys (rotated), window values
+    float *raw;                                       // [3][K1][DH] unrotated q, k, v; later the merged state
+    float *st;                                        // [kConsumerWarps + 1][K1][DH + 2] per-warp softmax states
+    __device__ AttnSmem(char *base, int K1) {
+        qh = reinterpret_cast<bf16 *>(base);
+        ql = qh + 16 * QP;
+        qf = reinterpret_cast<float *>(ql + 16 * QP);
+        kw = qf + K1 * DH;
+        vw = kw + K1 * DH;
+        raw = vw + K1 * DH;
+        st = raw + 3 * K1 * DH;
+    }
+};
+
+// Online-softmax state of one warp for query rows g and g+8 (base-2 exponentials).
+template <int DH> struct WarpState {
+    float o[DH / 8][4];
+    float m[2], l[2];
+};
+
+// 32 keys of one tile against the 16 query rows: S = Q K^T (hi + lo queries), online softmax, O += P V.
+template <int DH>
+__device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t k_tile, uint32_t v_tile, int key0, int nvalid,
+                                          WarpState<DH> &ws) {
+    constexpr int QPB = (DH + 8) * 2, RB = DH * 2;
+    const int lane = threadIdx.x & 31, t = lane & 3;
+    float s[4][4];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < DH / 16; ++ks) {
+        unsigned qh[4], ql[4];
+        const uint32_t qo = (uint32_t)(lane & 15) * QPB + (uint32_t)(ks * 16 + (lane >> 4) * 8) * 2u;
+        ldmatrix_x4(qh, q_hi + qo);
+        ldmatrix_x4(ql, q_lo + qo);
+#pragma unroll
+        for (int np = 0; np < 2; ++np) {      // key tiles 2np, 2np+1 (8 keys each)
+            const int row = key0 + np * 16 + (lane & 7) + ((lane >> 4) << 3);
+            const int chunk = 2 * ks + ((lane >> 3) & 1);
+            unsigned kb[4];
+            ldmatrix_x4(kb, k_tile + (uint32_t)row * RB + (uint32_t)swz(row, chunk, RB) * 16u);
+            mma16816(s[2 * np], qh[0], qh[1], qh[2], qh[3], kb[0], kb[1]);
+            mma16816(s[2 * np], ql[0], ql[1], ql[2], ql[3], kb[0], kb[1]);
+            mma16816(s[2 * np + 1], qh[0], qh[1], qh[2], qh[3], kb[2], kb[3]);
+            mma16816(s[2 * np + 1], ql[0], ql[1], ql[2], ql[3], kb[2], kb[3]);
+        }
+    }
+    // mask the keys past the end, row maxima over the 32 keys
+    float mx0 = kNegBig, mx1 = kNegBig;
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+        const int k0 = nt * 8 + 2 * t;
+        if (k0 >= nvalid) { s[nt][0] = -INFINITY; s[nt][2] = -INFINITY; }
+        if (k0 + 1 >= nvalid) { s[nt][1] = -INFINITY; s[nt][3] = -INFINITY; }
+        mx0 = fmaxf(mx0, fmaxf(s[nt][0], s[nt][1]));
+        mx1 = fmaxf(mx1, fmaxf(s[nt][2], s[nt][3]));
+    }
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+    const float m0 = fmaxf(ws.m[0], mx0), m1 = fmaxf(ws.m[1], mx1);
+    const float c0 = exp2f(ws.m[0] - m0), c1 = exp2f(ws.m[1] - m1);
+    ws.m[0] = m0; ws.m[1] = m1;
+    float l0 = 0.f, l1 = 0.f;
+    unsigned ph[2][4], pl[2][4];   // P as A fragments of the two 16-key steps, hi and lo
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+        const float p0 = exp2f(s[nt][0] - m0), p1 = exp2f(s[nt][1] - m0);
+        const float p2 = exp2f(s[nt][2] - m1), p3 = exp2f(s[nt][3] - m1);
+        l0 += p0 + p1; l1 += p2 + p3;
+        unsigned h0, h1, h2, h3, e0, e1, e2, e3;
+        split_bf16(p0, h0, e0); split_bf16(p1, h1, e1); split_bf16(p2, h2, e2); split_bf16(p3, h3, e3);
+        const int kk = nt >> 1, hi2 = (nt & 1) * 2;     // a0,a1 from the even key tile, a2,a3 from the odd one
+        ph[kk][hi2] = h0 | (h1 << 16); ph[kk][hi2 + 1] = h2 | (h3 << 16);
+        pl[kk][hi2] = e0 | (e1 << 16); pl[kk][hi2 + 1] = e2 | (e3 << 16);
+    }
+    ws.l[0] = ws.l[0] * c0 + l0;
+    ws.l[1] = ws.l[1] * c1 + l1;
+#pragma unroll
+    for (int dn = 0; dn < DH / 8; ++dn) { ws.o[dn][0] *= c0; ws.o[dn][1] *= c0; ws.o[dn][2] *= c1; ws.o[dn][3] *= c1; }
+#pragma unroll
+    for (int kk = 0; kk < 2; ++kk) {
+#pragma unroll
+        for (int dp = 0; dp < DH / 16; ++dp) {   // value columns 16dp .. 16dp+15 (chunks 2dp, 2dp+1)
+            const int row = key0 + kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+            const int chunk = 2 * dp + (lane >> 4);
+            unsigned vb[4];
+            ldmatrix_x4_trans(vb, v_tile + (uint32_t)row * RB + (uint32_t)swz(row, chunk, RB) * 16u);
+            mma16816(ws.o[2 * dp], ph[kk][0], ph[kk][1], ph[kk][2], ph[kk][3], vb[0], vb[1]);
+            mma16816(ws.o[2 * dp], pl[kk][0], pl[kk][1], pl[kk][2], pl[kk][3], vb[0], vb[1]);
+            mma16816(ws.o[2 * dp + 1], ph[kk][0], ph[kk][1], ph[kk][2], ph[kk][3], vb[2], vb[3]);
+            mma16816(ws.o[2 * dp + 1], pl[kk][0], pl[kk][1], pl[kk][2], pl[kk][3], vb[2], vb[3]);
+        }
+    }
+}
+
+// One (sequence, head, split) item.  Self-attention: the K+1 window rows (positions len+j) against the
+// cached keys of this split's pages; the last split also takes the window's own keys (row j sees window
+// keys 0..j, fp32) and appends them to the cache.  Cross-attention: the same rows against the cached
+// condition keys, no mask, no rotation.  Splits leave (m, l, O) partials; the last split merges them.
+template <typename KVT, int DH>
+static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const Stage &st, const AttnItem &it, uint32_t serial) {
+    constexpr bool MMA = sizeof(KVT) == 2;
+    const bool cross = st.kind == ST_ATTN_CROSS;
+    const int K1 = D.K1, P = D.P, d = D.d, half = DH / 2, b = it.b, h = it.h;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n = cross ? D.C : S.ctl->len[b];
+    const bool win = !cross && it.s == it.S - 1;
+    const bool merger = it.s == it.S - 1;
+    const float *qsrc = cross ? D.qc : D.qkv;
+    const int q_ld = cross ? d : 3 * d;
+    void *pool = cross ? D.ckv_pool : D.kv_pool;
+    const int pool_pages = cross ? D.B * D.cpages : D.n_pages;
+    float *part = cross ? D.cpart : D.part;
+    float *out = cross ? D.cattn : D.attn;
+    const uint32_t tag_in = tag_of(serial, st.in), tag_out = tag_of(serial, st.outt), tag_part = tag_of(serial, st.part);
+    AttnSmem<DH> A(S.acts, K1);
+    const float qscale = D.scale * kLog2e;
+    int p_lo, p_hi;
+    split_pages(n, P, it.s, it.S, p_lo, p_hi);
+
+    csync();
+    // the rotation table and the pages of the appended rows are fetched while q is awaited
+    constexpr int kRot = (16 * DH + kConsumerThreads - 1) / kConsumerThreads;
+    float2 cs_pre[kRot];
+#pragma unroll
+    for (int q = 0; q < kRot; ++q) {
+        const int i = tid + q * kConsumerThreads, j = i / DH, e = i - j * DH;
+        cs_pre[q] = make_float2(1.f, 0.f);
+        if (!cross && j < K1) cs_pre[q] = __ldcg(D.rope_cs + (size_t)(b * K1 + j) * half + (e % half));
+    }
+    int page_pre[2] = {0, 0};
+    if (win) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int i = tid + q * kConsumerThreads;
+            if (i < 2 * K1 * (DH / 8)) {
+                const int j = (i % (K1 * (DH / 8))) / (DH / 8);
+                page_pre[q] = __ldcg(D.block_table + (size_t)b * D.max_blocks + (n + j) / P);
+            }
+        }
+    }
+    // 1. fetch q (and the window's k, v) of this head
+    const int nsrc = win ? 3 : 1;
+    for (int i = tid; i < nsrc * K1 * (DH / 4); i += kConsumerThreads) {
+        const int which = i / (K1 * (DH / 4)), rem = i - which * K1 * (DH / 4), j = rem / (DH / 4), c4 = rem - j * (DH / 4);
+        const uint4 w = poll_u4(D, S.ctl, qsrc + (size_t)(b * K1 + j) * q_ld + which * d + h * DH + c4 * 4, tag_in);
+        *reinterpret_cast<float4 *>(A.raw + ((size_t)which * K1 + j) * DH + c4 * 4) =
+            make_float4(read_word<KVT>(w.x), read_word<KVT>(w.y), read_word<KVT>(w.z), read_word<KVT>(w.w));
+    }
+    csync();
+    if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
+    // 2. rotate, scale, split; zero the unused query rows
+#pragma unroll
+    for (int qq = 0; qq < kRot; ++qq) {
+        const int i = tid + qq * kConsumerThreads;
+        if (i >= 16 * DH) break;
+        const int j = i / DH, e = i - j * DH;
+        float q = 0.f;
+        if (j < K1) {
+            q = A.raw[j * DH + e];
+            if (!cross) {
+                const float2 cs = cs_pre[qq];
+                const float o = A.raw[j * DH + (e < half ? e + half : e - half)];
+                q = e < half ? q * cs.x - o * cs.y : o * cs.y + q * cs.x;
+                if (win) {
+                    const float kr = A.raw[(K1 + j) * DH + e], ko = A.raw[(K1 + j) * DH + (e < half ? e + half : e - half)];
+                    A.kw[j * DH + e] = e < half ? kr * cs.x - ko * cs.y : ko * cs.y + kr * cs.x;
+                    A.vw[j * DH + e] = A.raw[(2 * K1 + j) * DH + e];
+                }
+            }
+            q *= qscale;
+            A.qf[j * DH + e] = q;
+        }
+        if (MMA) {
+            unsigned hi, lo;
+            split_bf16(q, hi, lo);
+            A.qh[j * A.QP + e] = __ushort_as_bfloat16((unsigned short)hi);
+            A.ql[j * A.QP + e] = __ushort_as_bfloat16((unsigned short)lo);
+        }
+    }
+    csync();
+    // 3. append the window's keys and values to the cache (positions n .. n+K1-1)
+    if (win) {
+#pragma unroll
+        for (int qq = 0; qq < 2; ++qq) {
+            const int i = tid + qq * kConsumerThreads;
+            if (i >= 2 * K1 * (DH / 8)) break;
+            const int kv = i / (K1 * (DH / 8)), rem = i - kv * K1 * (DH / 8), j = rem / (DH / 8), c = rem - j * (DH / 8);
+            const int pos = n + j, page = page_pre[qq], r = pos % P;
+            const float *src = (kv ? A.vw : A.kw) + j * DH + c * 8;
+            KVT *tile = kv_tile<KVT>(D, pool, pool_pages, st.layer, kv, page, h);
+            KVT *dst = tile + tile_off<KVT>(r, c * 8, DH);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) dst[q] = from_f<KVT>(src[q]);
+        }
+    }
+    // 4. the cached keys of this split
+    WarpState<DH> ws;
+#pragma unroll
+    for (int dn = 0; dn < DH / 8; ++dn) ws.o[dn][0] = ws.o[dn][1] = ws.o[dn][2] = ws.o[dn][3] = 0.f;
+    ws.m[0] = ws.m[1] = kNegBig;
+    ws.l[0] = ws.l[1] = 0.f;
+    float *my_st = A.st + (size_t)warp * K1 * (DH + 2);
+    if (MMA) {
+        const uint32_t q_hi = smem_u32(A.qh), q_lo = smem_u32(A.ql);
+        const int upp = P / 32;   // 32-key units per page
+        int unit = 0;
+        for (int pg = p_lo; pg < p_hi; ++pg) {
+            const char *ks = ring_wait(D, S, ring);
+            const char *vs = ks + D.tile_bytes;
+            Ring r2 = ring;
+            if (!D.kv_one_item) { r2.pos += 1; vs = ring_wait(D, S, r2); }
+            const int nv_page = min(P, n - pg * P);
+            for (int u = 0; u < upp; ++u, ++unit) {
+                const int nv = min(32, nv_page - u * 32);
+                if (nv > 0 && (unit % kConsumerWarps) == warp)
+                    attn_unit<DH>(q_hi, q_lo, smem_u32(ks), smem_u32(vs), u * 32, nv, ws);
+            }
+            ring_release(S, ring);
+            if (!D.kv_one_item) ring_release(S, ring);
+        }
+        // quad-reduce the denominators, park the state in shared memory
+        const int g = lane >> 2, t = lane & 3;
+        ws.l[0] += __shfl_xor_sync(0xffffffffu, ws.l[0], 1); ws.l[0] += __shfl_xor_sync(0xffffffffu, ws.l[0], 2);
+        ws.l[1] += __shfl_xor_sync(0xffffffffu, ws.l[1], 1); ws.l[1] += __shfl_xor_sync(0xffffffffu, ws.l[1], 2);
+        if (g < K1) {
+#pragma unroll
+            for (int dn = 0; dn < DH / 8; ++dn) {
+                my_st[g * (DH + 2) + dn * 8 + 2 * t] = ws.o[dn][0];
+                my_st[g * (DH + 2) + dn * 8 + 2 * t + 1] = ws.o[dn][1];
+            }
+            if (t == 0) { my_st[g * (DH + 2) + DH] = ws.m[0]; my_st[g * (DH + 2) + DH + 1] = ws.l[0]; }
+        }
+        if (g + 8 < K1) {
+#pragma unroll
+            for (int dn = 0; dn < DH / 8; ++dn) {
+                my_st[(g + 8) * (DH + 2) + dn * 8 + 2 * t] = ws.o[dn][2];
+                my_st[(g + 8) * (DH + 2) + dn * 8 + 2 * t + 1] = ws.o[dn][3];
+            }
+            if (t == 0) { my_st[(g + 8) * (DH + 2) + DH] = ws.m[1]; my_st[(g + 8) * (DH + 2) + DH + 1] = ws.l[1]; }
+        }
+    } else {
+        // fp32 cache: one key per warp at a time, straight from global memory, all query rows at once
+        constexpr int EPL = (DH + 31) / 32;
+        const int e0 = lane * EPL;
+        const bool lane_on = e0 < DH;
+        const int key_lo = min(n, p_lo * P), key_hi = min(n, p_hi * P);
+        for (int j0 = 0; j0 < K1; j0 += 8) {
+            const int nq = min(8, K1 - j0);
+            float q[8][EPL], acc[8][EPL], mx[8], l[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                mx[j] = kNegBig; l[j] = 0.f;
+#pragma unroll
+                for (int i = 0; i < EPL; ++i) { acc[j][i] = 0.f; q[j][i] = (j < nq && lane_on) ? A.qf[(j0 + j) * DH + e0 + i] : 0.f; }
+            }
+            for (int key = key_lo + warp; key < key_hi; key += kConsumerWarps) {
+                const int page = cross ? b * D.cpages + key / P : __ldcg(D.block_table + (size_t)b * D.max_blocks + key / P);
+                const KVT *kt = kv_tile<KVT>(D, pool, pool_pages, st.layer, 0, page, h) + (size_t)(key % P) * DH + e0;
+                const KVT *vt = kv_tile<KVT>(D, pool, pool_pages, st.layer, 1, page, h) + (size_t)(key % P) * DH + e0;
+                float kf[EPL], vf[EPL];
+#pragma unroll
+                for (int i = 0; i < EPL; ++i) {
+                    kf[i] = lane_on ? to_f(__ldcg(kt + i)) : 0.f;
+                    vf[i] = lane_on ? to_f(__ldcg(vt + i)) : 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (j < nq) {
+                        float dsum = 0.f;
+#pragma unroll
+                        for (int i = 0; i < EPL; ++i) dsum = fmaf(q[j][i], kf[i], dsum);
+                        dsum = warp_sum(dsum);
+                        const float mn = fmaxf(mx[j], dsum), corr = exp2f(mx[j] - mn), pw = exp2f(dsum - mn);
+                        l[j] = l[j] * corr + pw;
+#pragma unroll
+                        for (int i = 0; i < EPL; ++i) acc[j][i] = acc[j][i] * corr + pw * vf[i];
+                        mx[j] = mn;
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (j < nq) {
+                    float *sw = my_st + (size_t)(j0 + j) * (DH + 2);
+                    if (lane_on) {
+#pragma unroll
+                        for (int i = 0; i < EPL; ++i) sw[e0 + i] = acc[j][i];
+                    }
+                    if (lane == 0) { sw[DH] = mx[j]; sw[DH + 1] = l[j]; }
+                }
+            }
+        }
+    }
+    // 5. the window's own keys under the causal mask: query row j (one warp each) against window keys 0..j
+    {
+        float *wst = A.st + (size_t)kConsumerWarps * K1 * (DH + 2);
+        constexpr int EPL = (DH + 31) / 32;
+        for (int j = warp; j < K1; j += kConsumerWarps) {
+            float m = kNegBig, l = 0.f, acc[EPL];
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) acc[i] = 0.f;
+            if (win) {
+                for (int wk = 0; wk <= j; ++wk) {
+                    float dsum = 0.f;
+#pragma unroll
+                    for (int i = 0; i < EPL; ++i) {
+                        const int e = lane + 32 * i;
+                        if (e < DH) dsum = fmaf(A.qf[j * DH + e], A.kw[wk * DH + e], dsum);
+                    }
+                    dsum = warp_sum(dsum);
+                    const float mn = fmaxf(m, dsum), corr = exp2f(m - mn), pw = exp2f(dsum - mn);
+                    l = l * corr + pw;
+#pragma unroll
+                    for (int i = 0; i < EPL; ++i) {
+                        const int e = lane + 32 * i;
+                        if (e < DH) acc[i] = acc[i] * corr + pw * A.vw[wk * DH + e];
+                    }
+                    m = mn;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) {
+                const int e = lane + 32 * i;
+                if (e < DH) wst[j * (DH + 2) + e] = acc[i];
+            }
+            if (lane == 0) { wst[j * (DH + 2) + DH] = m; wst[j * (DH + 2) + DH + 1] = l; }
+        }
+    }
+    csync();
+    // 6. merge the warps (and the window state); one thread per (query row, element); element DH = denominator
+    float *mg = A.raw;    // [K1][DH + 2] merged (O, m, l); raw q/k/v are no longer needed
+    for (int i = tid; i < K1 * (DH + 1); i += kConsumerThreads) {
+        const int j = i / (DH + 1), e = i - j * (DH + 1);
+        float m = kNegBig;
+        for (int w = 0; w <= kConsumerWarps; ++w) m = fmaxf(m, A.st[((size_t)w * K1 + j) * (DH + 2) + DH]);
+        float o = 0.f;
+        for (int w = 0; w <= kConsumerWarps; ++w) {
+            const float *sw = A.st + ((size_t)w * K1 + j) * (DH + 2);
+            o += exp2f(sw[DH] - m) * (e < DH ? sw[e] : sw[DH + 1]);
+        }
+        mg[j * (DH + 2) + (e < DH ? e : DH + 1)] = o;
+        if (e == DH) mg[j * (DH + 2) + DH] = m;
+    }
+    csync();
+    if (!merger) {
+        // leave the partial for the last split
+        float *pr = part + ((size_t)(b * D.H + h) * D.S_max + it.s) * K1 * (DH + 2);
+        for (int i = tid; i < K1 * (DH + 2); i += kConsumerThreads) st_relaxed_u32(pr + i, tagged(mg[i], tag_part));
+        return;
+    }
+    if (it.S > 1) {
+        // wait for the other splits and fold them in (fixed order)
+        for (int i = tid; i < K1 * (DH + 1); i += kConsumerThreads) {
+            const int j = i / (DH + 1), e = i - j * (DH + 1);
+            float m = mg[j * (DH + 2) + DH];
+            const float *pb = part + ((size_t)(b * D.H + h) * D.S_max) * K1 * (DH + 2) + (size_t)j * (DH + 2);
+            for (int ss = 0; ss < it.S - 1; ++ss)
+                m = fmaxf(m, untag(poll_u32(D, S.ctl, pb + (size_t)ss * K1 * (DH + 2) + DH, tag_part)));
+            float o = exp2f(mg[j * (DH + 2) + DH] - m) * mg[j * (DH + 2) + (e < DH ? e : DH + 1)];
+            for (int ss = 0; ss < it.S - 1; ++ss) {
+                const float *ps = pb + (size_t)ss * K1 * (DH + 2);
+                const float pm = untag(ld_relaxed_u32(ps + DH));
+                o += exp2f(pm - m) * untag(poll_u32(D, S.ctl, ps + (e < DH ? e : DH + 1), tag_part));
+            }
+            A.st[j * (DH + 2) + (e < DH ? e : DH + 1)] = o;   // st is free again: final numerators and denominator
+        }
+        csync();
+        mg = A.st;
+    }
+    for (int i = tid; i < K1 * DH; i += kConsumerThreads) {
+        const int j = i / DH, e = i - j * DH;
+        st_relaxed_u32(out + (size_t)(b * K1 + j) * d + h * DH + e, publish_word<KVT>(mg[j * (DH + 2) + e] / mg[j * (DH + 2) + DH + 1], tag_out, false));
+    }
+}
+
+template <typename KVT, int DH>
+static __device__ void consume_attn(const Dev &D, const Smem &S, Ring &ring, const Stage &st, uint32_t serial) {
+    const bool cross = st.kind == ST_ATTN_CROSS;
+    AttnItem it;
+    for (int idx = blockIdx.x; attn_item_at(D, S.ctl, cross, idx, it); idx += gridDim.x)
+        attn_item<KVT, DH>(D, S, ring, st, it, serial);
+}
+
+// ----------------------------------------------------------------- verify / accept length / resample
+
+// is (va, ia) ranked before (vb, ib): larger logit first, then smaller index
+__device__ __forceinline__ bool ranked_before(float va, int ia, float vb, int ib) {
+    return va > vb || (va == vb && ia < ib);
+}
+
+static __device__ float block_sum(float v, float *sh) {
+    v = warp_sum(v);
+    csync();
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+    csync();
+    float s = 0.f;
+    for (int w = 0; w < kConsumerWarps; ++w) s += sh[w];
+    return s;
+}
+static __device__ float block_max(float v, float *sh) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    csync();
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+    csync();
+    float s = -INFINITY;
+    for (int w = 0; w < kConsumerWarps; ++w) s = fmaxf(s, sh[w]);
+    return s;
+}
+// best (value, index) over the block under ranked_before; threads without a candidate pass idx = INT_MAX
+static __device__ void block_best(float &v, int &idx, float *shv, int *shi) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+        if (oi != 0x7fffffff && (idx == 0x7fffffff || ranked_before(ov, oi, v, idx))) { v = ov; idx = oi; }
+    }
+    csync();
+    if ((threadIdx.x & 31) == 0) { shv[threadIdx.x >> 5] = v; shi[threadIdx.x >> 5] = idx; }
+    csync();
+    v = shv[0]; idx = shi[0];
+    for (int w = 1; w < kConsumerWarps; ++w)
+        if (shi[w] != 0x7fffffff && (idx == 0x7fffffff || ranked_before(shv[w], shi[w], v, idx))) { v = shv[w]; idx = shi[w]; }
+}
+
+// copies one tagged logits row into shared memory (waiting for it), tags stripped
+static __device__ void fetch_row(const Dev &D, const Smem &S, const float *z, float *row, uint32_t tag) {
+    const int V = D.V;
+    csync();
+    if ((V & 3) == 0) {   // rows start on 16-byte boundaries
+        const int n4 = V >> 2;
+        for (int i0 = 0; i0 < n4; i0 += kConsumerThreads * kPollBatch) {
+            uint4 w[kPollBatch];
+#pragma unroll
+            for (int u = 0; u < kPollBatch; ++u) {
+                const int i = i0 + u * kConsumerThreads + threadIdx.x;
+                if (i < n4) w[u] = ld_relaxed_u4(z + 4 * i);
+            }
+#pragma unroll
+            for (int u = 0; u < kPollBatch; ++u) {
+                const int i = i0 + u * kConsumerThreads + threadIdx.x;
+                if (i < n4) {
+                    if (!tags_ok(w[u], tag)) w[u] = poll_u4(D, S.ctl, z + 4 * i, tag);
+                    *reinterpret_cast<float4 *>(row + 4 * i) = make_float4(untag(w[u].x), untag(w[u].y), untag(w[u].z), untag(w[u].w));
+                }
+            }
+        }
+    } else {
+        for (int i = threadIdx.x; i < V; i += kConsumerThreads) row[i] = untag(poll_u32(D, S.ctl, z + i, tag));
+    }
+    csync();
+}
+
+// acceptance of token x under backbone logits z (shared memory), block-wide; every thread returns the same answer
+static __device__ bool accept_token(const Dev &D, const float *z, int x, float *sh) {
+    const int V = D.V;
+    if (x < 0 || x >= V) return false;
+    if (D.verify_mode == 2) {     // p0(x) > delta
+        float m = -INFINITY;
+        for (int v = threadIdx.x; v < V; v += kConsumerThreads) m = fmaxf(m, z[v]);
+        m = block_max(m, sh);
+        float sum = 0.f;
+        for (int v = threadIdx.x; v < V; v += kConsumerThreads) sum += expf(z[v] - m);
+        sum = block_sum(sum, sh);
+        return expf(z[x] - m) / sum > D.delta;
+    }
+    const int ka = D.verify_mode == 0 ? 1 : D.k_accept;
+    const float zx = z[x];
+    float cnt = 0.f;
+    for (int v = threadIdx.x; v < V; v += kConsumerThreads)
+        if (v != x && ranked_before(z[v], v, zx, x)) cnt += 1.f;
+    cnt = block_sum(cnt, sh);
+    return (int)cnt < ka;
+}
+
+static __device__ int sample_token(const Dev &D, const float *z, uint32_t r24, float *sh) {
+    const int V = D.V;
+    float *shv = sh;
+    int *shi = reinterpret_cast<int *>(sh + kConsumerWarps);
+    float *cv = sh + 2 * kConsumerWarps;               // candidates (value, index), up to 64
+    int *ci = reinterpret_cast<int *>(cv + 64);
+    int *pick_s = ci + 64;
+    const int k = D.sample_mode == 0 ? 1 : min(max(D.k_sample, 1), min(V, 64));
+    float pv = INFINITY;
+    int pi = -1;
+    for (int j = 0; j < k; ++j) {      // j-th candidate: best among those ranked after the previous one
+        float bv = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int v = threadIdx.x; v < V; v += kConsumerThreads) {
+            const float zv = z[v];
+            if (j > 0 && !ranked_before(pv, pi, zv, v)) continue;
+            if (bi == 0x7fffffff || ranked_before(zv, v, bv, bi)) { bv = zv; bi = v; }
+        }
+        block_best(bv, bi, shv, shi);
+        if (threadIdx.x == 0) { cv[j] = bv; ci[j] = bi; }
+        pv = bv; pi = bi;
+        csync();
+    }
+    if (threadIdx.x == 0) {
+        int pick = ci[0];
+        if (D.sample_mode != 0) {
+            float total = 0.f;      // the weights are evaluated twice rather than kept in a local array
+            for (int j = 0; j < k; ++j) total += expf((cv[j] - cv[0]) / D.temperature);
+            const float u = (float)r24 * (1.0f / 16777216.0f);
+            float cum = 0.f;
+            pick = ci[k - 1];
+            for (int j = 0; j < k; ++j) {
+                cum += expf((cv[j] - cv[0]) / D.temperature);
+                if (cum > u * total) { pick = ci[j]; break; }
+            }
+        }
+        *pick_s = pick;
+    }
+    csync();
+    return *pick_s;
+}
+
+// item (sequence b, slot): slot 0 resamples x_{s*} from the backbone row of the first rejection, slot i
+// from head i's logits of the same row (independent sampling).  Every item recomputes the accept length.
+// (not inlined, and handed nothing whose address would pin the caller's registers to memory: the shared-memory
+// plan is derived again from the kernel's parameters)
+static __device__ __noinline__ void sample_stage(const Dev &D, uint32_t serial) {
+    extern __shared__ __align__(1024) char smem[];
+    const Smem S = carve(smem, D);
+    const int K1 = D.K1, K = D.K, V = D.V;
+    const TagRef once = {1, 0};
+    const uint32_t tag = tag_of(serial, once);
+    float *row = reinterpret_cast<float *>(S.acts);
+    float *sh = row + ((V + 3) & ~3);
+    for (int it = blockIdx.x; it < D.B * K1; it += gridDim.x) {
+        const int b = it / K1, slot = it % K1;
+        if (S.ctl->flags[b] & 3) continue;
+        int a = 0;
+        while (a < K) {
+            const int x = __ldcg(D.window + b * K1 + a + 1);
+            fetch_row(D, S, D.logits0 + (size_t)(b * K1 + a) * V, row, tag);
+            if (!accept_token(D, row, x, sh)) break;
+            ++a;
+        }
+        const float *z = slot == 0 ? D.logits0 + (size_t)(b * K1 + a) * V
+                                   : D.hlogits + ((size_t)(slot - 1) * D.M + b * K1 + a) * V;
+        fetch_row(D, S, z, row, tag);
+        const uint32_t r = rand24(D, b, __ldcg(D.step_idx + b), (uint32_t)slot, 0u);
+        const int tok = sample_token(D, row, r, sh);
+        if (threadIdx.x == 0) {
+            st_relaxed_u32(D.candx + (size_t)b * (K1 + 1) + slot, tagged_int(tok, tag));
+            if (slot == 0) st_relaxed_u32(D.candx + (size_t)b * (K1 + 1) + K1, tagged_int(a, tag));
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------- commit / next window
+
+// After the length and the window of sequence b are final: reserve cache pages for positions < len + K + 1,
+// gather the embeddings of the window into the residual stream (master copy and tagged copy for the step
+// `serial`), and tabulate cos/sin of the window rows' positions.  Threads 0..nthr-1 take part; `win` may point to
+// shared or global memory; nb_held = pages the sequence holds already.
+template <typename WT> __device__ void prepare_window(const Dev &D, int b, uint32_t serial, int len, int nb_held, const int *win, int nthr) {
+    const int K1 = D.K1, d = D.d, half = D.dh / 2;
+    const TagRef hemb = {3 * D.L + 1, 0};
+    const uint32_t tag = tag_of(serial, hemb);
+    if (threadIdx.x == 0) {
+        const int need = (len + K1 + D.P - 1) / D.P;
+        int nb = nb_held;
+        while (nb < need) {
+            const int idx = atomicSub(D.n_free, 1) - 1;
+            if (idx < 0 || nb >= D.max_blocks) {
+                atomicAdd(D.n_free, 1);
+                atomicExch(D.status, XSM_STATUS_CAPACITY);
+                break;
+            }
+            __stcg(D.block_table + (size_t)b * D.max_blocks + nb, __ldcg(D.free_stack + idx));
+            ++nb;
+        }
+        if (nb != nb_held) __stcg(D.n_blocks + b, nb);
+    }
+    const WT *E = reinterpret_cast<const WT *>(D.E);
+    const WT *g0 = reinterpret_cast<const WT *>(D.gain_first);
+    // one warp per window row: embedding -> master copy and published copy (bf16 models: times the gain of the
+    // step's first RMSNorm, with the row's sum of squares as this writer's share and zero shares for the rest)
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = nthr >> 5;
+    for (int j = warp; j < K1; j += nwarps) {
+        const int tok = min(max(win[j], 0), D.V - 1), row = b * K1 + j;
+        float ssq = 0.f;
+        for (int e = lane; e < d; e += 32) {
+            const float v = to_f(E[(size_t)tok * d + e]);
+            __stcg(D.h + (size_t)row * d + e, v);
+            ssq = fmaf(v, v, ssq);
+            const float pub = sizeof(WT) == 2 ? v * to_f(g0[e]) : v;
+            st_relaxed_u32(D.hpub + (size_t)row * d + e, publish_word<WT>(pub, tag, false));
+        }
+        if (sizeof(WT) == 2) {
+            ssq = warp_sum(ssq);
+            for (int c = lane; c < D.grid; c += 32) st_relaxed_u32(D.sspub + (size_t)c * D.M + row, tagged(c == 0 ? ssq : 0.f, tag));
+        }
+    }
+    for (int i = threadIdx.x; i < K1 * half; i += nthr) {
+        const int j = i / half, f = i % half;
+        double sn, cs;
+        sincos((double)(len + j) * D.inv_freq[f], &sn, &cs);
+        __stcg(D.rope_cs + (size_t)(b * K1 + j) * half + f, make_float2((float)cs, (float)sn));
+    }
+}
+
+// publishes the header of sequence b for step `serial` (after everything else of the sequence is written);
+// threads 0..3 of the block write one word each
+static __device__ void publish_header(const Dev &D, int b, uint32_t serial, int len, int flags) {
+    const TagRef once = {1, 0};
+    const uint32_t tag = tag_of(serial, once);
+    uint32_t *hd = D.header + (size_t)b * kHeaderWords;
+    if (threadIdx.x < kHeaderWords)
+        st_relaxed_u32(hd + threadIdx.x, tagged_int(threadIdx.x == 0 ? len : threadIdx.x == 1 ? flags : 0, tag));
+}
+
+static __device__ void draw_initial_drafts(const Dev &D, int b, int *win) {
+    for (int i = 1; i <= D.K; ++i) {
+        const unsigned long long m = rand24(D, b, 0u, (uint32_t)i, 1u);
+        win[i] = (int)((m * (unsigned long long)D.V) >> 24);
+    }
+}
+
+// Algorithm 1 line 12 and the loop guard: commit x_{s+1..s*}, s <- s*, next window <- candidates.
+template <typename WT> __device__ __noinline__ void commit_stage(const Dev &D, uint32_t serial) {
+    extern __shared__ __align__(1024) char smem[];
+    const Smem S = carve(smem, D);
+    const int K1 = D.K1, tid = threadIdx.x;
+    const TagRef once = {1, 0};
+    const uint32_t tag = tag_of(serial, once);
+    // scratch words in shared memory
+    int *sm = reinterpret_cast<int *>(S.acts);
+    int *s_cand = sm + 8;                 // [K1] resampled tokens, [K1] accept length
+    int *s_state = sm + 40;               // len, ingest_left, n_gen, step_idx, n_blocks
+    int *s_win = sm + 64;                 // [K1] window before, then after
+    enum { O_LEN = 0, O_FLAGS = 1 };      // sm[0], sm[1]: new length and flags
+    if ((int)blockIdx.x < D.B) {
+        for (int c = tid; c < (int)gridDim.x; c += kConsumerThreads) poll_u32(D, S.ctl, D.done + c, tag);
+        __threadfence();
+    }
+    for (int b = blockIdx.x; b < D.B; b += gridDim.x) {
+        csync();
+        const int fl = S.ctl->flags[b];
+        // every word the commit needs, fetched side by side
+        if (!(fl & 1)) {
+            if (tid <= K1 && !(fl & 2)) s_cand[tid] = untag_int(poll_u32(D, S.ctl, D.candx + (size_t)b * (K1 + 1) + tid, tag));
+            if (tid == 32) s_state[0] = __ldcg(D.len + b);
+            if (tid == 33) s_state[1] = __ldcg(D.ingest_left + b);
+            if (tid == 34) s_state[2] = __ldcg(D.n_gen + b);
+            if (tid == 35) s_state[3] = (int)__ldcg(D.step_idx + b);
+            if (tid == 36) s_state[4] = __ldcg(D.n_blocks + b);
+            if (tid >= 64 && tid < 64 + K1) s_win[tid - 64] = __ldcg(D.window + b * K1 + tid - 64);
+        }
+        csync();
+        if (tid == 0) {
+            int len = S.ctl->len[b], flags = fl;
+            if (!(fl & 1)) {
+                len = s_state[0];
+                const int left = s_state[1];
+                if (left > 0) {
+                    // prompt ingestion: the window held prompt tokens; all of them that are prompt enter the cache
+                    const int n = min(K1, left);
+                    len += n;
+                    __stcg(D.ingest_left + b, left - n);
+                    __stcg(D.step_n_new + b, 0);
+                    const int *pr = D.prompt + (size_t)b * D.prompt_len;
+                    if (left - n > 0) {
+                        for (int j = 0; j < K1; ++j) s_win[j] = len + j < D.prompt_len ? pr[len + j] : 0;
+                        flags = 2;
+                    } else {
+                        s_win[0] = pr[D.prompt_len - 1];
+                        draw_initial_drafts(D, b, s_win);
+                        flags = 0;
+                    }
+                } else {
+                    const int a = min(max(s_cand[K1], 0), D.K);
+                    __stcg(D.acc_len + b, a);
+                    int n_gen = s_state[2], fin = 0, n_out = 0;
+                    for (int j = 0; j <= a; ++j) {
+                        const int tok = j < a ? s_win[j + 1] : s_cand[0];
+                        if (n_gen >= D.max_new) break;
+                        __stcg(D.tok_log + (size_t)b * D.tok_ld + n_gen, tok);
+                        __stcg(D.step_tokens + b * K1 + n_out, tok);
+                        ++n_gen; ++n_out;
+                        if (D.eos >= 0 && tok == D.eos) { fin = 1; break; }
+                    }
+                    for (int j = n_out; j < K1; ++j) __stcg(D.step_tokens + b * K1 + j, -1);
+                    __stcg(D.step_n_new + b, n_out);
+                    len += a + 1;
+                    if (n_gen >= D.max_new || len > D.max_seq_len) fin = 1;
+                    __stcg(D.n_gen + b, n_gen);
+                    for (int j = 0; j < K1; ++j) {
+                        s_win[j] = s_cand[j];
+                        __stcg(D.cand + b * K1 + j, s_cand[j]);
+                    }
+                    __stcg(D.step_idx + b, (uint32_t)s_state[3] + 1u);
+                    atomicAdd(D.hist + (size_t)b * (kMaxDraft + 1) + a, 1ull);
+                    atomicAdd(D.steps + b, 1ull);
+                    if (fin) {
+                        __stcg(D.finished + b, 1);
+                        atomicSub(D.n_active, 1);
+                        flags = 1;
+                    }
+                }
+                __stcg(D.len + b, len);
+                for (int j = 0; j < K1; ++j) __stcg(D.window + b * K1 + j, s_win[j]);
+            } else {
+                __stcg(D.step_n_new + b, 0);
+            }
+            sm[O_LEN] = len;
+            sm[O_FLAGS] = flags;
+        }
+        csync();
+        if (!(sm[O_FLAGS] & 1)) prepare_window<WT>(D, b, serial + 1u, sm[O_LEN], s_state[4], s_win, kConsumerThreads);
+        __threadfence();
+        csync();
+        publish_header(D, b, serial + 1u, sm[O_LEN], sm[O_FLAGS]);
+    }
+}
+
+// ------------------------------------------------------------------------------------ step kernel
+
+// 9 warps are allocated as 12 (warps come in fours), which leaves 168 registers per thread
+// The projection and attention stages [p_lo, p_hi) of one step, consumer side.  A function of its own that
+// calls nothing: the register allocation of the hot loops is then not disturbed by values that must survive
+// the calls of the rare stages.  Returns the ring position.
+template <typename WT, int NTM>
+static __device__ __forceinline__ uint32_t consume_gemv_stage(const Dev &D, const Stage *st, uint32_t serial, uint32_t ring_pos) {
+    extern __shared__ __align__(1024) char smem[];
+    const Smem S = carve(smem, D);
+    Ring ring;
+    ring.pos = ring_pos;
+    gemv_stage<WT, NTM, false>(D, S, ring, *st, serial);
+    return ring.pos;
+}
+template <typename WT, int DH>
+static __device__ __forceinline__ uint32_t consume_attn_stage(const Dev &D, const Stage *st, uint32_t serial, uint32_t ring_pos) {
+    extern __shared__ __align__(1024) char smem[];
+    const Smem S = carve(smem, D);
+    Ring ring;
+    ring.pos = ring_pos;
+    consume_attn<WT, DH>(D, S, ring, *st, serial);
+    return ring.pos;
+}
+
+// The projection and attention stages [p_lo, p_hi) of one step, consumer side.  Returns the ring position.
+template <typename WT, int NTM, int DH>
+static __device__ __forceinline__ uint32_t consume_stages(const Dev &D, uint32_t serial, uint32_t ring_pos, int p_lo, int p_hi,
+                                                          int tracing) {
+    extern __shared__ __align__(1024) char smem[];
+    Ctl *ctl = reinterpret_cast<Ctl *>(smem + 256);
+    for (int p = p_lo; p < p_hi; ++p) {
+        const Stage *st = D.stages + p;
+        const int kind = st->kind;
+        if (threadIdx.x == 0) ctl->trace_row = tracing ? 1 + 2 * p : 0;
+        if (kind == ST_GEMV) ring_pos = consume_gemv_stage<WT, NTM>(D, st, serial, ring_pos);
+        else if (kind == ST_ATTN_SELF || kind == ST_ATTN_CROSS) ring_pos = consume_attn_stage<WT, DH>(D, st, serial, ring_pos);
+        if (tracing) trace_mark(D, 2 + 2 * p);
+    }
+    return ring_pos;
+}
+
+// the same stages seen by the producer warp
+template <typename WT, int NTM>
+static __device__ __forceinline__ uint32_t produce_stages(const Dev &D, uint32_t ring_pos, int p_lo, int p_hi) {
+    extern __shared__ __align__(1024) char smem[];
+    const Smem S = carve(smem, D);
+    Ring ring;
+    ring.pos = ring_pos;
+    for (int p = p_lo; p < p_hi; ++p) {
+        const Stage &st = D.stages[p];
+        if (st.kind == ST_GEMV) gemv_stage<WT, NTM, true>(D, S, ring, st, 0u);
+        else if (st.kind == ST_ATTN_SELF || st.kind == ST_ATTN_CROSS) produce_attn<WT>(D, S, ring, st);
+    }
+    return ring.pos;
+}
+
+// One instance per (weight type, token capacity, head width): each carries only its own code path.
+// The last two stages of a step are verify/resample and commit; all stages before them stream through the ring.
+template <typename WT, int NTM, int DH>
+__global__ void __launch_bounds__(kThreads, 1)
+step_kernel(const __grid_constant__ Dev D, int st_lo, int st_hi, int n_steps, uint32_t serial0) {
+    extern __shared__ __align__(1024) char smem[];
+    const Smem S = carve(smem, D);
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (tid == 0) {
+        for (int i = 0; i < S.n_slots; ++i) {
+            mbar_init(S.full0 + 8u * i, 1u);
+            mbar_init(S.empty0 + 8u * i, (uint32_t)kConsumerWarps);
+        }
+        mbar_init(S.go_bar, 1u);
+        S.ctl->dead = 0;
+        S.ctl->go = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    __syncthreads();
+    uint32_t ring_pos = 0;
+    const TagRef once = {1, 0};
+    const int p_sample = D.n_stages - 2, p_commit = D.n_stages - 1;
+    const int ring_hi = min(st_hi, p_sample);          // stages [st_lo, ring_hi) use the ring
+    if (warp == kConsumerWarps) {
+        // ---- producer warp
+        for (int t = 0; t < n_steps; ++t) {
+            mbar_wait(D, S.ctl, S.go_bar, (uint32_t)t & 1u);
+            if (!S.ctl->go) break;
+            fence_proxy_async();   // cache rows written by other CTAs in the previous step, read below by bulk copies
+            ring_pos = produce_stages<WT, NTM>(D, ring_pos, st_lo, ring_hi);
+        }
+        return;
+    }
+    // ---- consumer warps
+    for (int t = 0; t < n_steps; ++t) {
+        const uint32_t serial = serial0 + (uint32_t)t;
+        // the step header: length and flags of every sequence, published by the previous commit (or by prefill)
+        csync();
+        int any = 0;
+        {
+            const uint32_t tag = tag_of(serial, once);
+            for (int b = tid; b < D.B; b += kConsumerThreads) {
+                const uint32_t *hd = D.header + (size_t)b * kHeaderWords;
+                S.ctl->len[b] = untag_int(poll_u32(D, S.ctl, hd, tag));
+                S.ctl->flags[b] = untag_int(poll_u32(D, S.ctl, hd + 1, tag));
+            }
+            __threadfence();   // what the publisher wrote before the header (pages, rope table, master h) is visible now
+            csync();
+            for (int m = tid; m < D.M; m += kConsumerThreads) S.ctl->row_dead[m] = (unsigned char)(S.ctl->flags[m / D.K1] & 1);
+            for (int b = 0; b < D.B; ++b) any |= !(S.ctl->flags[b] & 1);
+            if (S.ctl->dead) any = 0;
+        }
+        if (tid == 0) {
+            S.ctl->go = any;
+            mbar_arrive(S.go_bar);
+        }
+        if (!any) break;
+        const int tracing = D.trace != nullptr && t == 0;
+        if (tracing) trace_mark(D, 0);
+        ring_pos = consume_stages<WT, NTM, DH>(D, serial, ring_pos, st_lo, ring_hi, tracing);
+        if (st_lo <= p_sample && p_sample < st_hi) {
+            // everything this CTA wrote in the step (cache rows above all) is ordered before its mark;
+            // the commit waits for every CTA's mark before it publishes the next step's header
+            __threadfence();
+            csync();
+            if (tid == 0) st_relaxed_u32(D.done + blockIdx.x, tagged_int(0, tag_of(serial, once)));
+            sample_stage(D, serial);
+            if (tracing) trace_mark(D, 2 + 2 * p_sample);
+        }
+        if (st_lo <= p_commit && p_commit < st_hi) {
+            commit_stage<WT>(D, serial);
+            if (tracing) trace_mark(D, 2 + 2 * p_commit);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------ host side of the step kernel
+
+template <typename WT, int NTM, int DH>
+cudaError_t launch_step_instance(const Dev &D, int st_lo, int st_hi, int n_steps, uint32_t serial0, int grid, int smem_bytes,
+                                 cudaStream_t st, int *max_grid) {
+    const void *fn = (const void *)step_kernel<WT, NTM, DH>;
+    static int attr_bytes = 0;     // largest dynamic shared memory this instance has been opened for
+    cudaError_t e;
+    if (smem_bytes > attr_bytes) {
+        if ((e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes)) != cudaSuccess) return e;
+        attr_bytes = smem_bytes;
+    }
+    if (max_grid != nullptr) {     // set-up query: how many CTAs can be resident
+        int dev = 0, sms = 0, per_sm = 0;
+        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, smem_bytes)) != cudaSuccess) return e;
+        *max_grid = per_sm >= 1 ? sms : 0;
+        return cudaSuccess;
+    }
+    void *args[] = {(void *)&D, &st_lo, &st_hi, &n_steps, &serial0};
+    // cooperative: every CTA must be resident, they wait for one another's data
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), args, (size_t)smem_bytes, st);
+}
+
+// picks the instance for the weight type and the number of token rows M
+template <int DH>
+cudaError_t launch_step_dh(const Dev &D, int dtype, int st_lo, int st_hi, int n_steps, uint32_t serial0, int grid, int smem_bytes,
+                           cudaStream_t st, int *max_grid) {
+    const int M = D.M;
+#define XSM_GO(WT, NTM) return launch_step_instance<WT, NTM, DH>(D, st_lo, st_hi, n_steps, serial0, grid, smem_bytes, st, max_grid)
+    if (dtype == 1) {
+        if (M <= 8) XSM_GO(bf16, 1);
+        if (M <= 16) XSM_GO(bf16, 2);
+        if (M <= 32) XSM_GO(bf16, 4);
+        if (M <= 80) XSM_GO(bf16, 10);
+        XSM_GO(bf16, 16);
+    }
+    if (M <= 8) XSM_GO(float, 8);
+    if (M <= 16) XSM_GO(float, 16);
+    XSM_GO(float, 24);
+#undef XSM_GO
+}
+
+}  // namespace xsm

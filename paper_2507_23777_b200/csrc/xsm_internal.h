@@ -6,7 +6,7 @@
 namespace xsm {
 
 // ---- geometry of the persistent step kernel
-constexpr int kConsumerWarps = 8;                    // warps that compute
+constexpr int kConsumerWarps = 7;                    // warps that compute; with the producer warp: 8 warps, 255 registers each
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;      // + one producer warp that feeds the ring
 constexpr int kMaxDraft = 16;                        // size of the histogram rows (n_draft itself is <= 15)
@@ -48,6 +48,9 @@ struct GemvJob {
     float *hm;               // EPI_ADD: untagged fp32 master copy of the residual stream [M][out_ld]
     int rows, kdim, out_ld, epi;
     TagRef in, outt;
+    // bf16 models publish activations as bf16 hi + lo pairs (see xsm_device.cuh); then:
+    const void *gain_out;    // EPI_ADD: RMSNorm gain of the stage that reads `out`, applied to the published copy
+    int out_plain;           // 1: `out` is published as plain tagged fp32 (logits) even in a bf16 model
 };
 
 struct Stage {
@@ -60,6 +63,7 @@ struct Dev {
     // shape
     int L, d, H, dh, f, V, C, dc, K, K1, B, M, P;
     int max_blocks, n_pages, cpages, max_seq_len, tok_ld;
+    int grid;                      // CTAs of the step kernel
     int S_max, S_cross;            // most key splits of a self-attention item; splits of a cross-attention item
     float eps, scale;
     int bos, eos;
@@ -88,6 +92,8 @@ struct Dev {
     float *hpub, *qkv, *attn, *qc, *cattn, *act, *y, *logits0, *hlogits, *part, *cpart;
     uint32_t *candx, *header;      // [B][K1 + 1] resampled tokens and accept length; [B][4] len, flags
     uint32_t *done;                // [grid] "this CTA has finished the projections of the step"
+    float *sspub;                  // [grid][M] bf16 models: each CTA's share of the sum of squares of the rows of hpub
+    const void *gain_first;        // RMSNorm gain that the first stage of a step applies to the embeddings
     unsigned long long *trace;     // null, or [1 + 2 * n_stages][grid] nanosecond timestamps of the launch's first step
     // untagged
     float *h;                      // master copy of the residual stream (each column range has one owner CTA)
@@ -109,6 +115,6 @@ cudaError_t launch_embed(const Dev &D, int dtype, uint32_t serial, cudaStream_t 
 cudaError_t launch_gather_kv(const Dev &D, int dtype, int layer, int seq, int pos0, int n, float *out_k,
                              float *out_v, cudaStream_t st);
 cudaError_t launch_export(const Dev &D, int max_new, int *d_tokens, int *d_lengths, cudaStream_t st);
-cudaError_t step_kernel_setup(int dtype, int smem_bytes, int *max_grid);
+cudaError_t step_kernel_setup(const Dev &D, int dtype, int smem_bytes, int *max_grid);
 
 }  // namespace xsm
