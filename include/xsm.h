@@ -122,6 +122,20 @@ XSM_API xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, cons
  * [batch] (0 for a finished sequence).  Either may be NULL.  Asynchronous. */
 XSM_API xsm_status xsm_spec_step(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_n_new);
 
+/* The paper has no counterpart of this call; it serves hosts that cannot give the library scratch memory of
+ * their own.  xsm_spec_step with one difference: the partial results that the key splits of an attention
+ * stage hand to one another (scratch that xsm_spec_step keeps in the caller's workspace) live in a 1 MiB
+ * array that is part of the library image, so the call needs no allocation by anyone: not by the library
+ * (it calls no allocator) and not by a caller that runs where cudaMalloc is not available, e.g. inside a
+ * host process that handed out all device memory at start-up, or on a path that must not synchronise the
+ * device.  Every GPU that loads the library holds the 1 MiB until the process exits.  The first call on a
+ * device looks up the array's device address; make that call before any stream capture.  A batch whose
+ * partials exceed the array (batch * n_heads * splits * (K+1) * (d_head+2) floats, twice) is refused with
+ * XSM_ERR_CAPACITY.  All contexts of a process share the array and it keeps the last call's contents; the
+ * call clears the part it uses first, so calls must not overlap on the GPU (same stream, or otherwise
+ * ordered): overlapping calls race.  Arguments and results as xsm_spec_step.  Asynchronous. */
+XSM_API xsm_status xsm_spec_step_static(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_n_new);
+
 /* Runs steps until every sequence has committed max_new_tokens tokens since
  * xsm_prefill, met EOS, or reached max_seq_len.  d_tokens: DEVICE int32
  * [batch, max_new_tokens] (x_1, x_2, ...; unused tail -1); d_lengths: DEVICE

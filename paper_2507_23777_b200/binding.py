@@ -22,7 +22,7 @@ EXPORTS = [
     "xsm_weights_bytes", "xsm_workspace_bytes", "xsm_create", "xsm_prefill", "xsm_spec_step", "xsm_generate",
     "xsm_generate_host", "xsm_destroy", "xsm_last_error", "xsm_kernel_launches", "xsm_debug_get_logits",
     "xsm_debug_get_kv", "xsm_debug_set_drafts", "xsm_debug_get_state", "xsm_debug_set_phase_launch",
-    "xsm_debug_trace_step",
+    "xsm_debug_trace_step", "xsm_spec_step_static",
 ]
 
 
@@ -69,6 +69,7 @@ def load(path: str | None = None):
     L.xsm_create.argtypes = [C.POINTER(ModelConfig), vp, vp, C.c_size_t, vp, C.POINTER(vp)]
     L.xsm_prefill.argtypes = [vp, C.c_int, vp, ip, C.c_int, C.POINTER(DecodeConfig)]
     L.xsm_spec_step.argtypes = [vp, ip, ip]
+    L.xsm_spec_step_static.argtypes = [vp, ip, ip]
     L.xsm_generate.argtypes = [vp, C.c_int, ip, ip, C.POINTER(Stats)]
     L.xsm_generate_host.argtypes = [vp, C.c_int, vp, ip, C.c_int, C.POINTER(DecodeConfig), C.c_int, ip, ip,
                                     C.POINTER(Stats)]
@@ -169,6 +170,10 @@ class Context:
     def xsm_spec_step(self, d_new_tokens=None, d_n_new=None):
         self._check(self.lib.xsm_spec_step(self._h, d_new_tokens.data_ptr() if d_new_tokens is not None else None,
                                            d_n_new.data_ptr() if d_n_new is not None else None))
+
+    def xsm_spec_step_static(self, d_new_tokens=None, d_n_new=None):
+        self._check(self.lib.xsm_spec_step_static(self._h, d_new_tokens.data_ptr() if d_new_tokens is not None else None,
+                                                  d_n_new.data_ptr() if d_n_new is not None else None))
 
     def xsm_generate(self, max_new: int, d_tokens=None, d_lengths=None) -> Stats:
         st = Stats()

@@ -555,6 +555,51 @@ xsm_status xsm_spec_step(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_n_new) 
     return XSM_OK;
 }
 
+// ---- scratch owned by the library, for xsm_spec_step_static
+// The name below is a device symbol: host code may not use it as an address.  Its device address is asked
+// for once per device (cudaGetSymbolAddress) and kept.
+constexpr size_t kStaticScratchBytes = (size_t)1 << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+static void *g_static_scratch_addr[kMaxDevices];   // by device ordinal; null until the first call on that device
+
+xsm_status xsm_spec_step_static(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_n_new) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "xsm_spec_step_static before xsm_prefill");
+    Dev &D = ctx->dev;
+    // the split partials of self- and cross-attention: [B * H * S_max][K + 1][d_head + 2] floats each
+    const size_t one = (size_t)D.B * D.H * D.S_max * D.K1 * (D.dh + 2) * sizeof(float);
+    const size_t half = (one + 255) / 256 * 256;
+    if (2 * half > kStaticScratchBytes)
+        return fail(ctx, XSM_ERR_CAPACITY, "xsm_spec_step_static: the attention partials of this batch need " +
+                                               std::to_string(2 * half) + " bytes, the built-in scratch holds " +
+                                               std::to_string(kStaticScratchBytes));
+    int dev = 0;
+    XSM_CUDA(ctx, cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(ctx, XSM_ERR_INVALID_ARG, "device ordinal out of range");
+    if (g_static_scratch_addr[dev] == nullptr) {   // set-up, once per device, with that device current
+        void *p = nullptr;
+        XSM_CUDA(ctx, cudaGetSymbolAddress(&p, g_static_scratch));
+        g_static_scratch_addr[dev] = p;
+    }
+    char *scratch = static_cast<char *>(g_static_scratch_addr[dev]);
+    // the array keeps what the last call left; a stale tag would pass for a fresh partial, so it restarts from zero
+    XSM_CUDA(ctx, cudaMemsetAsync(scratch, 0, 2 * half, ctx->stream));
+    float *const ws_part = D.part, *const ws_cpart = D.cpart;
+    D.part = reinterpret_cast<float *>(scratch);
+    D.cpart = reinterpret_cast<float *>(scratch + half);
+    D.max_new = INT_MAX;
+    const xsm_status st = run_steps(ctx, 1);     // the kernel arguments are copied at launch
+    D.part = ws_part;
+    D.cpart = ws_cpart;
+    if (st != XSM_OK) return st;
+    if (d_new_tokens)
+        XSM_CUDA(ctx, cudaMemcpyAsync(d_new_tokens, D.step_tokens, sizeof(int32_t) * D.M, cudaMemcpyDeviceToDevice, ctx->stream));
+    if (d_n_new)
+        XSM_CUDA(ctx, cudaMemcpyAsync(d_n_new, D.step_n_new, sizeof(int32_t) * D.B, cudaMemcpyDeviceToDevice, ctx->stream));
+    return XSM_OK;
+}
+
 xsm_status xsm_generate(xsm_ctx *ctx, int max_new_tokens, int32_t *d_tokens, int32_t *d_lengths, xsm_stats *host_stats) {
     if (!ctx) return XSM_ERR_INVALID_ARG;
     if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "xsm_generate before xsm_prefill");
