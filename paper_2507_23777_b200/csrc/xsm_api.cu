@@ -52,8 +52,8 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.n_phases = c.n_layers * 8 + 3 + (c.n_draft > 0 ? 1 : 0);
     L.n_jobs = c.n_layers * 6 + 1 + 2 * c.n_draft;
     size_t cur = 0;
-    L.phases = take(cur, sizeof(Stage) * L.n_phases);
-    L.jobs = take(cur, sizeof(GemvJob) * L.n_jobs);
+    L.phases = take(cur, sizeof(Tables));
+    L.jobs = take(cur, 256);
     L.inv_freq = take(cur, sizeof(double) * (dh / 2 + 1));
     L.wkc_off = take(cur, sizeof(size_t) * c.n_layers);
     L.wvc_off = take(cur, sizeof(size_t) * c.n_layers);
@@ -197,8 +197,8 @@ struct xsm_ctx {
     uint32_t serial;          // decoding steps launched since the last xsm_prefill
     uint64_t launches;
     std::string err;
-    std::vector<Stage> h_stages;
-    std::vector<GemvJob> h_jobs;
+    Tables h_tab;
+    int n_stages;             // stages of one decoding step
     int *pinned;              // [4] n_active, status
     cudaEvent_t ev0, ev1;
     double last_wall_ms;
@@ -229,7 +229,7 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     const int K1 = c.n_draft + 1, M = batch * K1, dh = c.d_head;
     const int kmax = c.d_model > c.d_ff ? c.d_model : c.d_ff;
     const int tail = (kMaxTokens + 1536) * 4;                        // sums of squares and their partials
-    const int avail = kSmemMax - kSmemHeader - tail;
+    const int avail = kSmemMax - kSmemHeader - kSmemTables - tail;
     // what the other users of the activation area need
     const int np = c.dtype == 1 ? (M <= 8 ? 8 : M <= 16 ? 16 : M <= 32 ? 32 : M <= 80 ? 80 : 128) : 8;
     int need = kConsumerWarps * np * 16 * 4 + 2 * 16 * M * 4;         // reduction of the projections, new residual values
@@ -255,11 +255,11 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     D.kca = kca;
     D.tile_bytes = c.page_size * dh * (c.dtype == 1 ? 2 : 4);
     D.kv_one_item = 2 * D.tile_bytes <= kSlotBytes ? 1 : 0;
-    smem_bytes = kSmemHeader + slots * kSlotBytes + acts + tail;
+    smem_bytes = kSmemHeader + kSmemTables + slots * kSlotBytes + acts + tail;
     return nullptr;
 }
 
-// stage and job tables for the current batch
+// stage and job tables for the current batch: the eight stages of layer 0, then the tail of the step
 void build_tables(xsm_ctx *ctx) {
     const xsm_model_config &c = ctx->cfg;
     const Dev &D = ctx->dev;
@@ -267,68 +267,71 @@ void build_tables(xsm_ctx *ctx) {
     const int d = c.d_model, f = c.d_ff, V = c.vocab, K = c.n_draft, L = c.n_layers;
     const size_t M = D.M;
     const int hw = 3 * L + 1;      // writes of the residual stream per step: the embedding and three per layer
-    ctx->h_stages.clear();
-    ctx->h_jobs.clear();
+    Tables &T = ctx->h_tab;
+    memset(&T, 0, sizeof(T));
+    T.layer_bytes = L > 1 ? (long long)((w.wq[1] - w.wq[0]) * esize(c)) : 0;
+    T.gain_last = wptr(ctx, w.gf);
+    int n_jobs = 0, n_stages = 0;
     auto job = [&](const void *W, const void *W2, int rows, int kdim, const float *x, const void *gain, float *out,
-                   int out_ld, int epi, TagRef in, TagRef outt, const void *gain_out = nullptr, int out_plain = 0) {
-        GemvJob j;
-        memset(&j, 0, sizeof(j));
+                   int out_ld, int epi, TagRef in, int in_jinc, TagRef outt, int out_jinc, const void *gain_out = nullptr,
+                   int out_plain = 0) -> GemvJob & {
+        GemvJob &j = T.jobs[n_jobs++];
         j.W = W; j.W2 = W2; j.x = x; j.gain = gain; j.out = out; j.hm = epi == EPI_ADD ? D.h : nullptr;
         j.rows = rows; j.kdim = kdim; j.out_ld = out_ld; j.epi = epi; j.in = in; j.outt = outt;
-        j.gain_out = gain_out; j.out_plain = out_plain;
-        ctx->h_jobs.push_back(j);
-        return (int)ctx->h_jobs.size() - 1;
+        j.in_jinc = in_jinc; j.out_jinc = out_jinc; j.gain_out = gain_out; j.out_plain = out_plain;
+        return j;
     };
-    auto gemv1 = [&](int layer, int j0, int n) {
-        Stage s;
-        memset(&s, 0, sizeof(s));
-        s.kind = ST_GEMV; s.layer = layer; s.job0 = j0; s.njobs = n;
-        ctx->h_stages.push_back(s);
+    auto gemv1 = [&](int j0, int n) {
+        Stage &s = T.stages[n_stages++];
+        s.kind = ST_GEMV; s.job0 = j0; s.njobs = n;
     };
-    auto attn = [&](int kind, int layer) {
-        Stage s;
-        memset(&s, 0, sizeof(s));
-        s.kind = kind; s.layer = layer;
-        s.in = TagRef{L, layer}; s.outt = TagRef{L, layer}; s.part = TagRef{L, layer};
-        ctx->h_stages.push_back(s);
+    auto attn = [&](int kind) {
+        Stage &s = T.stages[n_stages++];
+        s.kind = kind;
+        s.in = TagRef{L, 0}; s.outt = TagRef{L, 0}; s.part = TagRef{L, 0}; s.jinc = 1;
     };
-    for (int l = 0; l < L; ++l) {
-        const TagRef per_layer{L, l};
-        gemv1(l, job(wptr(ctx, w.wq[l]), nullptr, 3 * d, d, D.hpub, wptr(ctx, w.g1[l]), D.qkv, 3 * d, EPI_STORE,
-                     TagRef{hw, 3 * l}, per_layer), 1);
-        attn(ST_ATTN_SELF, l);
-        // a stage that adds to the residual stream publishes it with the gain of the RMSNorm that reads it next
-        gemv1(l, job(wptr(ctx, w.wo[l]), nullptr, d, d, D.attn, nullptr, D.hpub, d, EPI_ADD, per_layer,
-                     TagRef{hw, 3 * l + 1}, wptr(ctx, w.g2[l])), 1);
-        gemv1(l, job(wptr(ctx, w.wqc[l]), nullptr, d, d, D.hpub, wptr(ctx, w.g2[l]), D.qc, d, EPI_STORE,
-                     TagRef{hw, 3 * l + 1}, per_layer), 1);
-        attn(ST_ATTN_CROSS, l);
-        gemv1(l, job(wptr(ctx, w.woc[l]), nullptr, d, d, D.cattn, nullptr, D.hpub, d, EPI_ADD, per_layer,
-                     TagRef{hw, 3 * l + 2}, wptr(ctx, w.g3[l])), 1);
-        gemv1(l, job(wptr(ctx, w.wgate[l]), wptr(ctx, w.wup[l]), f, d, D.hpub, wptr(ctx, w.g3[l]), D.act, f, EPI_GATEUP,
-                     TagRef{hw, 3 * l + 2}, per_layer), 1);
-        gemv1(l, job(wptr(ctx, w.wdown[l]), nullptr, d, f, D.act, nullptr, D.hpub, d, EPI_ADD, per_layer,
-                     TagRef{hw, 3 * l + 3}, l + 1 < L ? wptr(ctx, w.g1[l + 1]) : wptr(ctx, w.gf)), 1);
+    // layer 0.  Buffers written once per layer have write index serial * L + l, the residual stream 3 l + which.
+    // A stage that adds to the residual stream publishes it with the gain of the RMSNorm that reads it next.
+    const TagRef per_layer{L, 0};
+    job(wptr(ctx, w.wq[0]), nullptr, 3 * d, d, D.hpub, wptr(ctx, w.g1[0]), D.qkv, 3 * d, EPI_STORE, TagRef{hw, 0}, 3, per_layer, 1);
+    gemv1(0, 1);
+    attn(ST_ATTN_SELF);
+    job(wptr(ctx, w.wo[0]), nullptr, d, d, D.attn, nullptr, D.hpub, d, EPI_ADD, per_layer, 1, TagRef{hw, 1}, 3, wptr(ctx, w.g2[0]));
+    gemv1(1, 1);
+    job(wptr(ctx, w.wqc[0]), nullptr, d, d, D.hpub, wptr(ctx, w.g2[0]), D.qc, d, EPI_STORE, TagRef{hw, 1}, 3, per_layer, 1);
+    gemv1(2, 1);
+    attn(ST_ATTN_CROSS);
+    job(wptr(ctx, w.woc[0]), nullptr, d, d, D.cattn, nullptr, D.hpub, d, EPI_ADD, per_layer, 1, TagRef{hw, 2}, 3, wptr(ctx, w.g3[0]));
+    gemv1(3, 1);
+    job(wptr(ctx, w.wgate[0]), wptr(ctx, w.wup[0]), f, d, D.hpub, wptr(ctx, w.g3[0]), D.act, f, EPI_GATEUP, TagRef{hw, 2}, 3,
+        per_layer, 1);
+    gemv1(4, 1);
+    {   // the down projection's published copy is read through the first RMSNorm of the NEXT layer (or the final one)
+        GemvJob &j = job(wptr(ctx, w.wdown[0]), nullptr, d, f, D.act, nullptr, D.hpub, d, EPI_ADD, per_layer, 1, TagRef{hw, 3}, 3,
+                         wptr(ctx, w.g1[0]));
+        j.gain_out_step = T.layer_bytes != 0 ? T.layer_bytes : 1;
+        gemv1(5, 1);
     }
+    // tail
     const TagRef once{1, 0};
-    int j0 = job(wptr(ctx, w.W0), nullptr, V, d, D.hpub, wptr(ctx, w.gf), D.logits0, V, EPI_STORE, TagRef{hw, 3 * L}, once, nullptr, 1);
+    int j0 = n_jobs;
+    job(wptr(ctx, w.W0), nullptr, V, d, D.hpub, wptr(ctx, w.gf), D.logits0, V, EPI_STORE, TagRef{hw, 3 * L}, 0, once, 0, nullptr, 1);
     for (int i = 0; i < K; ++i)
         job(wptr(ctx, w.W1[i]), nullptr, d, d, D.hpub, wptr(ctx, w.gf), D.y + (size_t)i * M * d, d, EPI_HEADY,
-            TagRef{hw, 3 * L}, once);
-    gemv1(-1, j0, 1 + K);
+            TagRef{hw, 3 * L}, 0, once, 0);
+    gemv1(j0, 1 + K);
     if (K > 0) {
-        j0 = (int)ctx->h_jobs.size();
+        j0 = n_jobs;
         for (int i = 0; i < K; ++i)
             job(wptr(ctx, w.Wout[i]), nullptr, V, d, D.y + (size_t)i * M * d, nullptr, D.hlogits + (size_t)i * M * V, V,
-                EPI_STORE, once, once, nullptr, 1);
-        gemv1(-1, j0, K);
+                EPI_STORE, once, 0, once, 0, nullptr, 1);
+        gemv1(j0, K);
     }
-    Stage s;
-    memset(&s, 0, sizeof(s));
-    s.kind = ST_SAMPLE; s.layer = -1;
-    ctx->h_stages.push_back(s);
-    s.kind = ST_COMMIT;
-    ctx->h_stages.push_back(s);
+    T.stages[n_stages++].kind = ST_SAMPLE;
+    T.stages[n_stages++].kind = ST_COMMIT;
+    T.n_tail_stages = n_stages - kLayerStages;
+    T.n_tail_jobs = n_jobs - kLayerJobs;
+    ctx->n_stages = kLayerStages * L + T.n_tail_stages;
 }
 
 xsm_status check_device_status(xsm_ctx *ctx) {
@@ -343,7 +346,7 @@ xsm_status check_device_status(xsm_ctx *ctx) {
 
 // n_steps decoding steps on the stream
 xsm_status run_steps(xsm_ctx *ctx, int n_steps) {
-    const int np = (int)ctx->h_stages.size();
+    const int np = ctx->n_stages;
     if (!ctx->phase_launch) {
         XSM_CUDA(ctx, launch_step(ctx->dev, ctx->cfg.dtype, 0, np, n_steps, ctx->serial, ctx->grid, ctx->smem_bytes, ctx->stream));
         ctx->launches += 1;
@@ -446,7 +449,7 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     D.max_seq_len = cfg->max_seq_len; D.tok_ld = L.tok_ld;
     D.eps = cfg->rms_eps; D.scale = (float)(1.0 / sqrt((double)cfg->d_head)); D.bos = cfg->bos_id; D.eos = cfg->eos_id;
     D.max_new = INT_MAX;
-    D.stages = at<Stage>(ctx, L.phases); D.jobs = at<GemvJob>(ctx, L.jobs);
+    D.tables = at<Tables>(ctx, L.phases);
     D.E = wptr(ctx, ctx->wo.E); D.inv_freq = at<double>(ctx, L.inv_freq);
     D.len = at<int>(ctx, L.len); D.window = at<int>(ctx, L.window); D.cand = at<int>(ctx, L.cand);
     D.acc_len = at<int>(ctx, L.acc_len); D.finished = at<int>(ctx, L.finished); D.n_gen = at<int>(ctx, L.n_gen);
@@ -513,20 +516,15 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
     }
     D.S_cross = s_cross;
     build_tables(ctx);
-    D.n_stages = (int)ctx->h_stages.size();
-    if ((int)ctx->h_stages.size() > ctx->lay.n_phases || (int)ctx->h_jobs.size() > ctx->lay.n_jobs)
-        return fail(ctx, XSM_ERR_STATE, "internal: stage table overflow");
-    XSM_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->lay.phases, ctx->h_stages.data(), sizeof(Stage) * ctx->h_stages.size(),
-                                  cudaMemcpyHostToDevice, ctx->stream));
-    XSM_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->lay.jobs, ctx->h_jobs.data(), sizeof(GemvJob) * ctx->h_jobs.size(),
-                                  cudaMemcpyHostToDevice, ctx->stream));
+    D.n_stages = ctx->n_stages;
+    XSM_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->lay.phases, &ctx->h_tab, sizeof(Tables), cudaMemcpyHostToDevice, ctx->stream));
     if ((const void *)d_prompt != (const void *)D.prompt)
         XSM_CUDA(ctx, cudaMemcpyAsync((void *)D.prompt, d_prompt, sizeof(int32_t) * batch * prompt_len,
                                       cudaMemcpyDeviceToDevice, ctx->stream));
     // no tag of an earlier generation may survive: the exchange buffers restart from "never written"
     XSM_CUDA(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.xchg_begin, 0, ctx->lay.xchg_end - ctx->lay.xchg_begin, ctx->stream));
     ctx->serial = 0;
-    // the tables above are read from host vectors that may be rebuilt by the next prefill
+    // the table above is read from host memory that the next prefill rewrites
     XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     XSM_CUDA(ctx, launch_cross_kv(D, c.dtype, ctx->weights, at<size_t>(ctx, ctx->lay.wkc_off),
                                   at<size_t>(ctx, ctx->lay.wvc_off), d_cond, ctx->stream));
@@ -766,7 +764,7 @@ xsm_status xsm_debug_trace_step(xsm_ctx *ctx, uint64_t *h_times, size_t capacity
     if (!ctx || !h_times || !n_rows || !n_ctas) return XSM_ERR_INVALID_ARG;
     if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "xsm_debug_trace_step before xsm_prefill");
     if (ctx->phase_launch) return fail(ctx, XSM_ERR_STATE, "the timeline is taken from the persistent kernel");
-    const int rows = 1 + 2 * (int)ctx->h_stages.size();
+    const int rows = 1 + 2 * ctx->n_stages;
     const size_t words = (size_t)rows * ctx->grid;
     if (capacity < words) return fail(ctx, XSM_ERR_CAPACITY, "h_times is too small");
     unsigned long long *d_trace = at<unsigned long long>(ctx, ctx->lay.trace);

@@ -202,6 +202,7 @@ struct Ctl {
 struct Smem {
     uint32_t full0, empty0, go_bar;   // shared-space addresses of full[0], empty[0], go
     Ctl *ctl;
+    const Tables *tab;                // shared-memory copy of the stage and job tables
     char *ring;
     char *acts;
     float *ss;                        // [kMaxTokens] sum of squares / 1 / rms
@@ -216,7 +217,8 @@ __device__ __forceinline__ Smem carve(char *smem, const Dev &D) {
     s.empty0 = s.full0 + 8u * kMaxSlots;
     s.go_bar = s.empty0 + 8u * kMaxSlots;
     s.ctl = reinterpret_cast<Ctl *>(smem + 256);   // 2 * 12 * 8 + 8 = 200 bytes of barriers before it
-    s.ring = smem + kSmemHeader;
+    s.tab = reinterpret_cast<const Tables *>(smem + kSmemHeader);
+    s.ring = smem + kSmemHeader + kSmemTables;
     s.n_slots = D.n_slots;
     s.acts = s.ring + (size_t)D.n_slots * kSlotBytes;
     s.ss = reinterpret_cast<float *>(s.acts + D.acts_bytes);
@@ -291,6 +293,42 @@ __device__ __forceinline__ void ring_claim(const Dev &D, const Smem &S, const Ri
         mbar_arrive_expect_tx(bar, bytes);
     }
     __syncwarp();
+}
+
+// ------------------------------------------------------------------------------------ tables
+
+// stage p of the step: layers first (eight stages each), then the tail
+__device__ __forceinline__ Stage stage_at(const Dev &D, const Smem &S, int p) {
+    const int n_layer = kLayerStages * D.L;
+    if (p < n_layer) {
+        const int l = p / kLayerStages;
+        Stage st = S.tab->stages[p - l * kLayerStages];
+        st.layer = l;
+        st.in.j += l * st.jinc; st.outt.j += l * st.jinc; st.part.j += l * st.jinc;
+        return st;
+    }
+    Stage st = S.tab->stages[kLayerStages + p - n_layer];
+    st.layer = -1;
+    return st;
+}
+// job `idx` of a stage of layer `layer` (< 0: a job of the tail), by value: its fields then live in registers
+__device__ __forceinline__ GemvJob job_at(const Dev &D, const Smem &S, int idx, int layer) {
+    GemvJob J = S.tab->jobs[idx];
+    if (layer > 0) {
+        const long long off = S.tab->layer_bytes * layer;
+        J.W = reinterpret_cast<const char *>(J.W) + off;
+        if (J.W2 != nullptr) J.W2 = reinterpret_cast<const char *>(J.W2) + off;
+        if (J.gain != nullptr) J.gain = reinterpret_cast<const char *>(J.gain) + off;
+        if (J.gain_out != nullptr) J.gain_out = reinterpret_cast<const char *>(J.gain_out) + off;
+        J.in.j += layer * J.in_jinc;
+        J.outt.j += layer * J.out_jinc;
+    }
+    // the down projection's published copy carries the gain of the next layer's first RMSNorm, or the final one
+    if (layer >= 0 && J.gain_out_step != 0) {
+        if (layer == D.L - 1) J.gain_out = S.tab->gain_last;
+        else J.gain_out = reinterpret_cast<const char *>(J.gain_out) + J.gain_out_step;
+    }
+    return J;
 }
 
 // ------------------------------------------------------------------------------ projection: plan
@@ -745,18 +783,19 @@ template <int NTM> struct ConsumeSegment<float, NTM> {
 // A projection stage, seen by the producer warp (PRODUCER) or by the consumer warps.
 template <typename WT, int NTM, bool PRODUCER>
 static __device__ void gemv_stage(const Dev &D, const Smem &S, Ring &ring, const Stage &st, uint32_t serial) {
-    long long total = 0;
-    for (int j = 0; j < st.njobs; ++j) total += D.jobs[st.job0 + j].rows;
-    const long long u_lo = total * blockIdx.x / gridDim.x, u_hi = total * (blockIdx.x + 1) / gridDim.x;
-    long long base = 0;
+    unsigned total = 0;      // rows of all jobs (a few tens of thousands at most)
+    for (int j = 0; j < st.njobs; ++j) total += (unsigned)S.tab->jobs[st.job0 + j].rows;
+    const int u_lo = (int)(total * blockIdx.x / gridDim.x), u_hi = (int)(total * (blockIdx.x + 1) / gridDim.x);
+    int base = 0;
     for (int j = 0; j < st.njobs; ++j) {
-        const GemvJob &J = D.jobs[st.job0 + j];
-        const long long lo = max(u_lo - base, 0LL), hi = min(u_hi - base, (long long)J.rows);
+        const int rows = S.tab->jobs[st.job0 + j].rows;
+        const int lo = max(u_lo - base, 0), hi = min(u_hi - base, rows);
         if (lo < hi) {
-            if (PRODUCER) produce_segment<WT>(D, S, ring, J, (int)lo, (int)hi);
-            else ConsumeSegment<WT, NTM>::run(D, S, ring, J, (int)lo, (int)hi, serial);
+            const GemvJob J = job_at(D, S, st.job0 + j, st.layer);
+            if (PRODUCER) produce_segment<WT>(D, S, ring, J, lo, hi);
+            else ConsumeSegment<WT, NTM>::run(D, S, ring, J, lo, hi, serial);
         }
-        base += J.rows;
+        base += rows;
     }
 }
 
@@ -1567,55 +1606,29 @@ template <typename WT> __device__ __noinline__ void commit_stage(const Dev &D, u
 
 // ------------------------------------------------------------------------------------ step kernel
 
-// 9 warps are allocated as 12 (warps come in fours), which leaves 168 registers per thread
-// The projection and attention stages [p_lo, p_hi) of one step, consumer side.  A function of its own that
-// calls nothing: the register allocation of the hot loops is then not disturbed by values that must survive
-// the calls of the rare stages.  Returns the ring position.
-template <typename WT, int NTM>
-static __device__ __forceinline__ uint32_t consume_gemv_stage(const Dev &D, const Stage *st, uint32_t serial, uint32_t ring_pos) {
-    extern __shared__ __align__(1024) char smem[];
-    const Smem S = carve(smem, D);
-    Ring ring;
-    ring.pos = ring_pos;
-    gemv_stage<WT, NTM, false>(D, S, ring, *st, serial);
-    return ring.pos;
-}
-template <typename WT, int DH>
-static __device__ __forceinline__ uint32_t consume_attn_stage(const Dev &D, const Stage *st, uint32_t serial, uint32_t ring_pos) {
-    extern __shared__ __align__(1024) char smem[];
-    const Smem S = carve(smem, D);
-    Ring ring;
-    ring.pos = ring_pos;
-    consume_attn<WT, DH>(D, S, ring, *st, serial);
-    return ring.pos;
-}
-
 // The projection and attention stages [p_lo, p_hi) of one step, consumer side.  Returns the ring position.
 template <typename WT, int NTM, int DH>
-static __device__ __forceinline__ uint32_t consume_stages(const Dev &D, uint32_t serial, uint32_t ring_pos, int p_lo, int p_hi,
-                                                          int tracing) {
-    extern __shared__ __align__(1024) char smem[];
-    Ctl *ctl = reinterpret_cast<Ctl *>(smem + 256);
+static __device__ __forceinline__ uint32_t consume_stages(const Dev &D, const Smem &S, uint32_t serial, uint32_t ring_pos,
+                                                          int p_lo, int p_hi, int tracing) {
+    Ring ring;
+    ring.pos = ring_pos;
     for (int p = p_lo; p < p_hi; ++p) {
-        const Stage *st = D.stages + p;
-        const int kind = st->kind;
-        if (threadIdx.x == 0) ctl->trace_row = tracing ? 1 + 2 * p : 0;
-        if (kind == ST_GEMV) ring_pos = consume_gemv_stage<WT, NTM>(D, st, serial, ring_pos);
-        else if (kind == ST_ATTN_SELF || kind == ST_ATTN_CROSS) ring_pos = consume_attn_stage<WT, DH>(D, st, serial, ring_pos);
+        const Stage st = stage_at(D, S, p);
+        if (threadIdx.x == 0) S.ctl->trace_row = tracing ? 1 + 2 * p : 0;
+        if (st.kind == ST_GEMV) gemv_stage<WT, NTM, false>(D, S, ring, st, serial);
+        else if (st.kind == ST_ATTN_SELF || st.kind == ST_ATTN_CROSS) consume_attn<WT, DH>(D, S, ring, st, serial);
         if (tracing) trace_mark(D, 2 + 2 * p);
     }
-    return ring_pos;
+    return ring.pos;
 }
 
 // the same stages seen by the producer warp
 template <typename WT, int NTM>
-static __device__ __forceinline__ uint32_t produce_stages(const Dev &D, uint32_t ring_pos, int p_lo, int p_hi) {
-    extern __shared__ __align__(1024) char smem[];
-    const Smem S = carve(smem, D);
+static __device__ __forceinline__ uint32_t produce_stages(const Dev &D, const Smem &S, uint32_t ring_pos, int p_lo, int p_hi) {
     Ring ring;
     ring.pos = ring_pos;
     for (int p = p_lo; p < p_hi; ++p) {
-        const Stage &st = D.stages[p];
+        const Stage st = stage_at(D, S, p);
         if (st.kind == ST_GEMV) gemv_stage<WT, NTM, true>(D, S, ring, st, 0u);
         else if (st.kind == ST_ATTN_SELF || st.kind == ST_ATTN_CROSS) produce_attn<WT>(D, S, ring, st);
     }
@@ -1641,6 +1654,11 @@ step_kernel(const __grid_constant__ Dev D, int st_lo, int st_hi, int n_steps, ui
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
+    {   // the tables move to shared memory once per launch
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(D.tables);
+        uint32_t *dst = reinterpret_cast<uint32_t *>(smem + kSmemHeader);
+        for (int i = tid; i < (int)(sizeof(Tables) / 4); i += kThreads) dst[i] = __ldg(src + i);
+    }
     __syncthreads();
     uint32_t ring_pos = 0;
     const TagRef once = {1, 0};
@@ -1652,7 +1670,7 @@ step_kernel(const __grid_constant__ Dev D, int st_lo, int st_hi, int n_steps, ui
             mbar_wait(D, S.ctl, S.go_bar, (uint32_t)t & 1u);
             if (!S.ctl->go) break;
             fence_proxy_async();   // cache rows written by other CTAs in the previous step, read below by bulk copies
-            ring_pos = produce_stages<WT, NTM>(D, ring_pos, st_lo, ring_hi);
+            ring_pos = produce_stages<WT, NTM>(D, S, ring_pos, st_lo, ring_hi);
         }
         return;
     }
@@ -1682,7 +1700,7 @@ step_kernel(const __grid_constant__ Dev D, int st_lo, int st_hi, int n_steps, ui
         if (!any) break;
         const int tracing = D.trace != nullptr && t == 0;
         if (tracing) trace_mark(D, 0);
-        ring_pos = consume_stages<WT, NTM, DH>(D, serial, ring_pos, st_lo, ring_hi, tracing);
+        ring_pos = consume_stages<WT, NTM, DH>(D, S, serial, ring_pos, st_lo, ring_hi, tracing);
         if (st_lo <= p_sample && p_sample < st_hi) {
             // everything this CTA wrote in the step (cache rows above all) is ordered before its mark;
             // the commit waits for every CTA's mark before it publishes the next step's header

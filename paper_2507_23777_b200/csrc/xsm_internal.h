@@ -51,12 +51,28 @@ struct GemvJob {
     // bf16 models publish activations as bf16 hi + lo pairs (see xsm_device.cuh); then:
     const void *gain_out;    // EPI_ADD: RMSNorm gain of the stage that reads `out`, applied to the published copy
     int out_plain;           // 1: `out` is published as plain tagged fp32 (logits) even in a bf16 model
+    int in_jinc, out_jinc;   // a layer job: how much in.j / outt.j grow from one layer to the next
+    long long gain_out_step; // a layer job: bytes from one layer's gain_out to the next layer's
 };
 
 struct Stage {
     int kind, layer, job0, njobs;
     TagRef in, outt, part;   // attention: q/k/v (or q) in, attention rows out, split partials
+    int jinc;                // a layer stage: growth of the three j's per layer
 };
+
+// Every layer has the same eight stages and the same weight layout, so the tables describe layer 0 (the
+// weights of layer l lie l * layer_bytes further) and the tail of the step (LM head and decoding heads, their
+// output projections, verify/resample, commit).  The step kernel works from a copy in shared memory.
+constexpr int kLayerStages = 8, kMaxTailStages = 4, kLayerJobs = 6, kMaxTailJobs = 2 * kMaxDraft + 1;
+struct Tables {
+    Stage stages[kLayerStages + kMaxTailStages];
+    GemvJob jobs[kLayerJobs + kMaxTailJobs];
+    long long layer_bytes;
+    const void *gain_last;   // gain_out of the last layer's down projection (the final RMSNorm)
+    int n_tail_stages, n_tail_jobs;
+};
+constexpr int kSmemTables = (sizeof(Tables) + 127) / 128 * 128;
 
 // Everything a kernel needs; passed by value.
 struct Dev {
@@ -73,9 +89,8 @@ struct Dev {
     uint32_t key0, key1;
     int max_new;
     // stage tables
-    const Stage *stages;
-    const GemvJob *jobs;
-    int n_stages;
+    const Tables *tables;
+    int n_stages;                  // 8 L + stages of the tail
     const void *E;                 // embedding table
     const double *inv_freq;        // [dh/2] theta^(-2i/dh)
     // shared-memory plan of the step kernel
