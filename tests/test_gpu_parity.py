@@ -119,6 +119,53 @@ def test_config1_small_bf16_prefix(P):
     ls.close()
 
 
+def test_config2_medium_bf16_prefix(P):
+    """Config 2 (24 layers, d=1024, K=4, top-5 acceptance, top-5 / T=0.5 resampling, output projections x4):
+    logits within the bf16 bound, decisions identical under teacher forcing except at small margins."""
+    cfg = inputs.config(2)
+    ls = P.LockStep(cfg)
+    ls.begin()
+    for _ in range(12):
+        ls.step(**BF16_TOL)
+    assert ls.excused <= 3
+    ls.compare_cache(layers=[0, 23], **BF16_TOL)
+    ls.close()
+
+
+def test_config2_k0_baseline_path(P):
+    """Config 2 with n_draft = 0 (the non-speculative baseline of the same library): one token per step."""
+    cfg = inputs.config(2, n_draft=0)
+    ls = P.LockStep(cfg)
+    ls.begin()
+    for _ in range(6):
+        _, acc = ls.step(**BF16_TOL)
+        assert acc == [0]
+    ls.close()
+
+
+def test_config3_batched_bf16_prefix(P):
+    """Config 3: 16 meshes with their own condition and Philox stream in one paged pool, ragged accept lengths."""
+    cfg = inputs.config(3)
+    ls = P.LockStep(cfg, batch=16)
+    ls.begin()
+    for _ in range(3):
+        ls.step(**BF16_TOL)
+    assert ls.excused <= 4
+    ls.compare_cache(layers=[11], **BF16_TOL)
+    ls.close()
+
+
+def test_config4_large_bf16_prefix(P):
+    """Config 4: 32 layers, d=2048, heads of 128, K=6, batch 4, top-8 acceptance at T=0.7."""
+    cfg = inputs.config(4)
+    ls = P.LockStep(cfg, batch=4)
+    ls.begin()
+    for _ in range(2):
+        ls.step(**BF16_TOL)
+    assert ls.excused <= 2
+    ls.close()
+
+
 def test_sampling_modes_lockstep(P):
     """Top-k acceptance with top-k / temperature resampling and threshold acceptance on the unit model."""
     for over in (dict(verify_mode=1, k_accept=3, sample_mode=1, k_sample=4, temperature=0.7, sigma=0.3),
