@@ -24,6 +24,7 @@
 #include "xsm_internal.h"
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <math.h>
 
 namespace xsm {
@@ -97,9 +98,17 @@ __device__ __forceinline__ void csync() { asm volatile("bar.sync 1, %0;" :: "n"(
 
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_f(__half v) { return __half2float(v); }
 template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ __half from_f<__half>(float v) { return __float2half_rn(fminf(fmaxf(v, -65504.f), 65504.f)); }
+
+// Element type of the key/value caches.  bf16 models keep them in fp16: the same two bytes, eleven bits of
+// mantissa instead of eight (cached keys and values are normalised activations times small weights, far
+// inside the fp16 range; stores saturate).  Rounding of the cache is the largest error of the whole path.
+template <typename WT> struct CacheT { typedef WT type; };
+template <> struct CacheT<bf16> { typedef __half type; };
 
 __device__ __forceinline__ float silu_f(float v) { return v / (1.0f + expf(-v)); }
 
@@ -116,6 +125,13 @@ __device__ __forceinline__ void split_bf16(float x, unsigned &hi, unsigned &lo) 
     hi = __bfloat16_as_ushort(h);
     lo = __bfloat16_as_ushort(l);
 }
+// x = hi + lo with hi, lo fp16 (operands of the attention products)
+__device__ __forceinline__ void split_f16(float x, unsigned &hi, unsigned &lo) {
+    const __half h = __float2half_rn(x);
+    const __half l = __float2half_rn(x - __half2float(h));
+    hi = __half_as_ushort(h);
+    lo = __half_as_ushort(l);
+}
 // four values -> {hi01, hi23, lo01, lo23}
 __device__ __forceinline__ uint4 split4(float a, float b, float c, float d) {
     unsigned h0, l0, h1, l1, h2, l2, h3, l3;
@@ -128,6 +144,14 @@ __device__ __forceinline__ void mma16816(float (&c)[4], unsigned a0, unsigned a1
                                          unsigned b0, unsigned b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma16816_f16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
+                                             unsigned b0, unsigned b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
         "{%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
@@ -561,6 +585,57 @@ __device__ __forceinline__ void mma_item_bf16(const char *slot, const char *acts
     }
 }
 
+// The same products for all items of one tile at once: the warp's column blocks (32 columns each) are spread
+// over the items of the tile, which sit in consecutive ring slots from position pos_tile; U blocks are in
+// flight together, each with accumulators of its own.
+template <int NT, int U>
+__device__ __forceinline__ void mma_tile_bf16(const Smem &S, uint32_t pos_tile, const char *acts, int pitch, int total_kb, int part,
+                                              int parts, int M, float (&acc)[NT][2][4]) {
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const uint32_t ring0 = smem_u32(S.ring), lane_off = (uint32_t)g * kRowPitch + (uint32_t)t * 16u;
+    const uint32_t x_base = smem_u32(acts) + (uint32_t)t * 32u;
+    const int ns = S.n_slots, s0 = (int)(pos_tile % (uint32_t)ns);
+    float au[U][NT][2][4];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) au[u][nt][0][q] = au[u][nt][1][q] = 0.f;
+    for (int q0 = part; q0 < total_kb; q0 += parts * U) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int kbg = q0 + u * parts;
+            if (kbg < total_kb) {
+                int slot = s0 + (kbg >> 4);
+                if (slot >= ns) slot -= ns;
+                const uint32_t wa_addr = ring0 + (uint32_t)slot * kSlotBytes + lane_off + (uint32_t)(kbg & 15) * 64u;
+                const uint4 wa = lds_u4(wa_addr), wb = lds_u4(wa_addr + 8u * kRowPitch);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int m = nt * 8 + g;
+                    uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = xa;
+                    if (m < M) {
+                        const uint32_t a = x_base + (uint32_t)m * (uint32_t)pitch + (uint32_t)kbg * 128u;
+                        xa = lds_u4(a);
+                        xb = lds_u4(a + 16u);
+                    }
+                    mma16816(au[u][nt][0], wa.x, wb.x, wa.y, wb.y, xa.x, xa.y);
+                    mma16816(au[u][nt][1], wa.x, wb.x, wa.y, wb.y, xa.z, xa.w);
+                    mma16816(au[u][nt][0], wa.z, wb.z, wa.w, wb.w, xb.x, xb.y);
+                    mma16816(au[u][nt][1], wa.z, wb.z, wa.w, wb.w, xb.z, xb.w);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { acc[nt][0][q] += au[u][nt][0][q]; acc[nt][1][q] += au[u][nt][1][q]; }
+}
+
 // What one output element becomes (after the dot product v, already scaled by 1/rms when the job has a gain).
 // hprev: the residual stream's value when the caller has fetched it ahead (have_prev), EPI_ADD only.
 // Returns the value before any gain of the next stage is applied (the residual stream's new value for EPI_ADD).
@@ -629,12 +704,31 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
                 staged = true;
                 if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
             }
-            for (int tl = 0; tl < tg; ++tl) {
-                for (int sc = 0; sc < acw; sc += p.ksub) {
-                    const int kw = min(p.ksub, acw - sc);
-                    const char *slot = ring_wait(D, S, ring);
-                    if (tl == my_tile) mma_item_bf16<NT>(slot, S.acts, pitch, sc, kw, my_part, parts, M, acc);
-                    ring_release(S, ring);
+            const int nsub = (acw + p.ksub - 1) / p.ksub;
+            if (one_chunk && tg * nsub <= S.n_slots) {
+                // All items of the stage are in the ring at once (each in a slot of its own).  A warp waits only
+                // for the items of its tile and multiplies them in one sweep.  A warp that does not read an item
+                // frees it at once: the previous item of that slot was freed by every warp before the barrier at
+                // the start of this stage, so no arrival can fall into the wrong phase.
+                constexpr int U = NT == 1 ? 4 : (NT == 2 ? 2 : 1);
+                const uint32_t pos0 = ring.pos;
+                if (my_tile < tg) {
+                    Ring r;
+                    for (int i = 0; i < nsub; ++i) { r.pos = pos0 + (uint32_t)(my_tile * nsub + i); ring_wait(D, S, r); }
+                    mma_tile_bf16<NT, U>(S, pos0 + (uint32_t)(my_tile * nsub), S.acts, pitch, acw >> 5, my_part, parts, M, acc);
+                }
+                __syncwarp();
+                if (lane == 0)
+                    for (int i = 0; i < tg * nsub; ++i) mbar_arrive(S.empty0 + 8u * ring_slot(S, pos0 + (uint32_t)i));
+                ring.pos = pos0 + (uint32_t)(tg * nsub);
+            } else {
+                for (int tl = 0; tl < tg; ++tl) {
+                    for (int sc = 0; sc < acw; sc += p.ksub) {
+                        const int kw = min(p.ksub, acw - sc);
+                        const char *slot = ring_wait(D, S, ring);
+                        if (tl == my_tile) mma_item_bf16<NT>(slot, S.acts, pitch, sc, kw, my_part, parts, M, acc);
+                        ring_release(S, ring);
+                    }
                 }
             }
         }
@@ -801,7 +895,7 @@ static __device__ void gemv_stage(const Dev &D, const Smem &S, Ring &ring, const
 
 // -------------------------------------------------------------------------------- attention: plan
 
-// Cache tiles.  One (page, head) tile holds P rows (positions) of dh elements.  bf16 tiles are stored with
+// Cache tiles.  One (page, head) tile holds P rows (positions) of dh elements.  16-bit tiles are stored with
 // their 16-byte chunks permuted so that ldmatrix over 8 consecutive rows touches every bank once; fp32
 // tiles are stored plain.
 template <typename KVT>
@@ -815,7 +909,7 @@ __device__ __forceinline__ int swz(int r, int c, int row_bytes) {
 // element offset of (row r, element e) inside a tile
 template <typename KVT> __device__ __forceinline__ size_t tile_off(int r, int e, int dh);
 template <> __device__ __forceinline__ size_t tile_off<float>(int r, int e, int dh) { return (size_t)r * dh + e; }
-template <> __device__ __forceinline__ size_t tile_off<bf16>(int r, int e, int dh) {
+template <> __device__ __forceinline__ size_t tile_off<__half>(int r, int e, int dh) {
     return (size_t)r * dh + (size_t)swz(r, e >> 3, dh * 2) * 8 + (e & 7);
 }
 
@@ -846,8 +940,9 @@ __device__ __forceinline__ void split_pages(int n_keys, int P, int s, int S, int
 
 // ---------------------------------------------------------------------------- attention: producer
 
-template <typename KVT>
+template <typename WT>
 static __device__ void produce_attn(const Dev &D, const Smem &S, Ring &ring, const Stage &st) {
+    typedef typename CacheT<WT>::type KVT;
     if (sizeof(KVT) != 2) return;   // the fp32 cache is read straight from global memory
     const bool cross = st.kind == ST_ATTN_CROSS;
     const int lane = threadIdx.x & 31;
@@ -926,10 +1021,10 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
             const int chunk = 2 * ks + ((lane >> 3) & 1);
             unsigned kb[4];
             ldmatrix_x4(kb, k_tile + (uint32_t)row * RB + (uint32_t)swz(row, chunk, RB) * 16u);
-            mma16816(s[2 * np], qh[0], qh[1], qh[2], qh[3], kb[0], kb[1]);
-            mma16816(s[2 * np], ql[0], ql[1], ql[2], ql[3], kb[0], kb[1]);
-            mma16816(s[2 * np + 1], qh[0], qh[1], qh[2], qh[3], kb[2], kb[3]);
-            mma16816(s[2 * np + 1], ql[0], ql[1], ql[2], ql[3], kb[2], kb[3]);
+            mma16816_f16(s[2 * np], qh[0], qh[1], qh[2], qh[3], kb[0], kb[1]);
+            mma16816_f16(s[2 * np], ql[0], ql[1], ql[2], ql[3], kb[0], kb[1]);
+            mma16816_f16(s[2 * np + 1], qh[0], qh[1], qh[2], qh[3], kb[2], kb[3]);
+            mma16816_f16(s[2 * np + 1], ql[0], ql[1], ql[2], ql[3], kb[2], kb[3]);
         }
     }
     // mask the keys past the end, row maxima over the 32 keys
@@ -955,7 +1050,7 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
         const float p2 = exp2f(s[nt][2] - m1), p3 = exp2f(s[nt][3] - m1);
         l0 += p0 + p1; l1 += p2 + p3;
         unsigned h0, h1, h2, h3, e0, e1, e2, e3;
-        split_bf16(p0, h0, e0); split_bf16(p1, h1, e1); split_bf16(p2, h2, e2); split_bf16(p3, h3, e3);
+        split_f16(p0, h0, e0); split_f16(p1, h1, e1); split_f16(p2, h2, e2); split_f16(p3, h3, e3);
         const int kk = nt >> 1, hi2 = (nt & 1) * 2;     // a0,a1 from the even key tile, a2,a3 from the odd one
         ph[kk][hi2] = h0 | (h1 << 16); ph[kk][hi2 + 1] = h2 | (h3 << 16);
         pl[kk][hi2] = e0 | (e1 << 16); pl[kk][hi2 + 1] = e2 | (e3 << 16);
@@ -972,10 +1067,10 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
             const int chunk = 2 * dp + (lane >> 4);
             unsigned vb[4];
             ldmatrix_x4_trans(vb, v_tile + (uint32_t)row * RB + (uint32_t)swz(row, chunk, RB) * 16u);
-            mma16816(ws.o[2 * dp], ph[kk][0], ph[kk][1], ph[kk][2], ph[kk][3], vb[0], vb[1]);
-            mma16816(ws.o[2 * dp], pl[kk][0], pl[kk][1], pl[kk][2], pl[kk][3], vb[0], vb[1]);
-            mma16816(ws.o[2 * dp + 1], ph[kk][0], ph[kk][1], ph[kk][2], ph[kk][3], vb[2], vb[3]);
-            mma16816(ws.o[2 * dp + 1], pl[kk][0], pl[kk][1], pl[kk][2], pl[kk][3], vb[2], vb[3]);
+            mma16816_f16(ws.o[2 * dp], ph[kk][0], ph[kk][1], ph[kk][2], ph[kk][3], vb[0], vb[1]);
+            mma16816_f16(ws.o[2 * dp], pl[kk][0], pl[kk][1], pl[kk][2], pl[kk][3], vb[0], vb[1]);
+            mma16816_f16(ws.o[2 * dp + 1], ph[kk][0], ph[kk][1], ph[kk][2], ph[kk][3], vb[2], vb[3]);
+            mma16816_f16(ws.o[2 * dp + 1], pl[kk][0], pl[kk][1], pl[kk][2], pl[kk][3], vb[2], vb[3]);
         }
     }
 }
@@ -984,8 +1079,9 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
 // cached keys of this split's pages; the last split also takes the window's own keys (row j sees window
 // keys 0..j, fp32) and appends them to the cache.  Cross-attention: the same rows against the cached
 // condition keys, no mask, no rotation.  Splits leave (m, l, O) partials; the last split merges them.
-template <typename KVT, int DH>
+template <typename WT, int DH>
 static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const Stage &st, const AttnItem &it, uint32_t serial) {
+    typedef typename CacheT<WT>::type KVT;
     constexpr bool MMA = sizeof(KVT) == 2;
     const bool cross = st.kind == ST_ATTN_CROSS;
     const int K1 = D.K1, P = D.P, d = D.d, half = DH / 2, b = it.b, h = it.h;
@@ -1032,7 +1128,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
         const int which = i / (K1 * (DH / 4)), rem = i - which * K1 * (DH / 4), j = rem / (DH / 4), c4 = rem - j * (DH / 4);
         const uint4 w = poll_u4(D, S.ctl, qsrc + (size_t)(b * K1 + j) * q_ld + which * d + h * DH + c4 * 4, tag_in);
         *reinterpret_cast<float4 *>(A.raw + ((size_t)which * K1 + j) * DH + c4 * 4) =
-            make_float4(read_word<KVT>(w.x), read_word<KVT>(w.y), read_word<KVT>(w.z), read_word<KVT>(w.w));
+            make_float4(read_word<WT>(w.x), read_word<WT>(w.y), read_word<WT>(w.z), read_word<WT>(w.w));
     }
     csync();
     if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
@@ -1060,7 +1156,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
         }
         if (MMA) {
             unsigned hi, lo;
-            split_bf16(q, hi, lo);
+            split_f16(q, hi, lo);
             A.qh[j * A.QP + e] = __ushort_as_bfloat16((unsigned short)hi);
             A.ql[j * A.QP + e] = __ushort_as_bfloat16((unsigned short)lo);
         }
@@ -1088,7 +1184,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     ws.m[0] = ws.m[1] = kNegBig;
     ws.l[0] = ws.l[1] = 0.f;
     float *my_st = A.st + (size_t)warp * K1 * (DH + 2);
-    if (MMA) {
+    if constexpr (MMA) {
         const uint32_t q_hi = smem_u32(A.qh), q_lo = smem_u32(A.ql);
         const int upp = P / 32;   // 32-key units per page
         int unit = 0;
@@ -1257,16 +1353,16 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     }
     for (int i = tid; i < K1 * DH; i += kConsumerThreads) {
         const int j = i / DH, e = i - j * DH;
-        st_relaxed_u32(out + (size_t)(b * K1 + j) * d + h * DH + e, publish_word<KVT>(mg[j * (DH + 2) + e] / mg[j * (DH + 2) + DH + 1], tag_out, false));
+        st_relaxed_u32(out + (size_t)(b * K1 + j) * d + h * DH + e, publish_word<WT>(mg[j * (DH + 2) + e] / mg[j * (DH + 2) + DH + 1], tag_out, false));
     }
 }
 
-template <typename KVT, int DH>
+template <typename WT, int DH>
 static __device__ void consume_attn(const Dev &D, const Smem &S, Ring &ring, const Stage &st, uint32_t serial) {
     const bool cross = st.kind == ST_ATTN_CROSS;
     AttnItem it;
     for (int idx = blockIdx.x; attn_item_at(D, S.ctl, cross, idx, it); idx += gridDim.x)
-        attn_item<KVT, DH>(D, S, ring, st, it, serial);
+        attn_item<WT, DH>(D, S, ring, st, it, serial);
 }
 
 // ----------------------------------------------------------------- verify / accept length / resample

@@ -64,8 +64,9 @@ __global__ void __launch_bounds__(256) cross_kv_kernel(const Dev D, const WT *Wa
             const int c = c0 + ty * 4 + i, r = r0 + tx * 4 + j;
             if (c < D.C && r < D.d) {
                 const int page = b * D.cpages + c / D.P, head = r / D.dh, e = r % D.dh;
-                WT *tile = kv_tile<WT>(D, D.ckv_pool, D.B * D.cpages, layer, kv, page, head);
-                tile[tile_off<WT>(c % D.P, e, D.dh)] = from_f<WT>(acc[i][j]);
+                typedef typename CacheT<WT>::type KVT;
+                KVT *tile = kv_tile<KVT>(D, D.ckv_pool, D.B * D.cpages, layer, kv, page, head);
+                tile[tile_off<KVT>(c % D.P, e, D.dh)] = from_f<KVT>(acc[i][j]);
             }
         }
 }
@@ -144,7 +145,7 @@ __global__ void gather_kv_kernel(const Dev D, int layer, int seq, int pos0, int 
 cudaError_t launch_gather_kv(const Dev &D, int dtype, int layer, int seq, int pos0, int n, float *out_k,
                              float *out_v, cudaStream_t st) {
     const int total = n * D.d;
-    if (dtype == 1) gather_kv_kernel<bf16><<<(total + 255) / 256, 256, 0, st>>>(D, layer, seq, pos0, n, out_k, out_v);
+    if (dtype == 1) gather_kv_kernel<__half><<<(total + 255) / 256, 256, 0, st>>>(D, layer, seq, pos0, n, out_k, out_v);
     else gather_kv_kernel<float><<<(total + 255) / 256, 256, 0, st>>>(D, layer, seq, pos0, n, out_k, out_v);
     return cudaGetLastError();
 }

@@ -55,17 +55,9 @@ def sample_excused(z, dc, r24, margin):
 
 
 def assert_logits(gpu, ref, atol, rtol, what):
-    """Every logit within atol + rtol |ref|.  With bf16 storage (atol >= 1e-2) the errors of the rounded cache
-    are random (measured standard deviation about 7e-3 on the x4-scaled logits of the medium model, i.e. the
-    bound sits near three sigma) and a step compares about 1e5 logits, so the bound is read as: at most 1 logit
-    in 1000 beyond it, none beyond twice it.  fp32 comparisons stay strict."""
+    """Every logit within atol + rtol |ref| (no exceptions)."""
     ok = logits_close(gpu, ref, atol, rtol)
-    if ok.all():
-        return
-    err = float(np.abs(gpu - ref).max())
-    assert atol >= 1e-2, f"{what} off by {err}"
-    assert logits_close(gpu, ref, 2 * atol, 2 * rtol).all(), f"{what} off by {err}: beyond twice the bound"
-    assert (~ok).mean() <= 1e-3, f"{what} off by {err}: {(~ok).sum()} of {ok.size} beyond the bound"
+    assert ok.all(), f"{what} off by {float(np.abs(gpu - ref).max())} ({int((~ok).sum())} of {ok.size} beyond the bound)"
 
 
 class LockStep:
