@@ -360,50 +360,67 @@ __device__ __forceinline__ GemvJob job_at(const Dev &D, const Smem &S, int idx, 
 // The rows of a stage's jobs form one range that is cut evenly over the CTAs; a CTA's piece of one job is a
 // segment.  A segment is processed as tile groups of up to 8 tiles (a tile: 16 weight rows, or 8 gate rows
 // + 8 up rows), the activations in chunks of D.kca columns, a tile in items of at most kItemRowBytes per row.
+// A tile has up to 16 layout rows (16 weight rows, or 8 gate rows then 8 up rows; 8 or 4 rows where a row is
+// longer than 4 KB, so that a tile never exceeds four slots).  An item is `rpi` consecutive layout rows at full
+// width: consecutive weight rows are contiguous in memory, so one bulk copy brings an item.  A tile group
+// (`tpg` tiles at most) has all its items in the ring at once.
+constexpr int kItemBytes = 16384;
 struct SegPlan {
-    int tile_units;   // units (output rows) per tile: 16, or 8 for gate/up
+    int tile_units;   // units (output rows) per tile: 16, 8 or 4; 8 for gate/up
+    int tu_shift;     // log2(tile_units)
+    int tile_rows;    // layout rows per tile: tile_units, or 16 for gate/up
     int n_tiles;
-    int ksub;         // columns per item
+    int rpi_shift;    // log2 of the layout rows per item (rows per item: 1, 2, 4 or 8)
+    int ipt;          // items per tile
+    int tpg;          // tiles per group = min(consumer warps, slots / ipt), at least 1
+    int row_bytes;
 };
-template <typename WT> __device__ __forceinline__ SegPlan seg_plan(const GemvJob &J, int lo, int hi) {
+template <typename WT> __device__ __forceinline__ SegPlan seg_plan(const Smem &S, const GemvJob &J, int lo, int hi) {
     SegPlan p;
-    p.tile_units = J.epi == EPI_GATEUP ? 8 : 16;
+    p.row_bytes = J.kdim * (int)sizeof(WT);            // the host refuses rows beyond kItemBytes
+    const int fit = kItemBytes / p.row_bytes;          // whole rows per item
+    p.rpi_shift = fit >= 8 ? 3 : fit >= 4 ? 2 : fit >= 2 ? 1 : 0;
+    if (J.epi == EPI_GATEUP) { p.tile_units = 8; p.tu_shift = 3; p.tile_rows = 16; }      // rows are d_model long: <= 4 KB
+    else {
+        p.tu_shift = p.row_bytes <= 4096 ? 4 : p.row_bytes <= 8192 ? 3 : 2;
+        p.tile_units = p.tile_rows = 1 << p.tu_shift;
+    }
     p.n_tiles = (hi - lo + p.tile_units - 1) / p.tile_units;
-    p.ksub = kItemRowBytes / (int)sizeof(WT);
+    p.ipt = max(1, p.tile_rows >> p.rpi_shift);
+    p.tpg = max(1, min(kConsumerWarps, S.n_slots / p.ipt));
     return p;
+}
+// valid weight rows of item `it` of a tile that starts at unit u0 and has nu units, and where they come from
+template <typename WT>
+__device__ __forceinline__ int item_rows(const GemvJob &J, const SegPlan &p, int u0, int nu, int it, const WT *&src) {
+    const int r0 = it << p.rpi_shift, rpi = 1 << p.rpi_shift;      // first layout row
+    if (J.epi == EPI_GATEUP) {
+        const int ui = r0 & 7;                                      // unit of the first row
+        src = reinterpret_cast<const WT *>(r0 < 8 ? J.W : J.W2) + (size_t)(u0 + ui) * J.kdim;
+        return min(max(nu - ui, 0), rpi);
+    }
+    src = reinterpret_cast<const WT *>(J.W) + (size_t)(u0 + r0) * J.kdim;
+    return min(max(nu - r0, 0), rpi);
 }
 
 // ---------------------------------------------------------------------------- projection: producer
 
 template <typename WT>
 static __device__ void produce_segment(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi) {
-    const SegPlan p = seg_plan<WT>(J, lo, hi);
+    const SegPlan p = seg_plan<WT>(S, J, lo, hi);
     const int lane = threadIdx.x & 31;
-    const int kca = min(J.kdim, D.kca);
-    for (int tg0 = 0; tg0 < p.n_tiles; tg0 += kConsumerWarps) {
-        const int tg = min(kConsumerWarps, p.n_tiles - tg0);
-        for (int ac0 = 0; ac0 < J.kdim; ac0 += kca) {
-            const int acw = min(kca, J.kdim - ac0);
-            for (int t = 0; t < tg; ++t) {
-                const int u0 = lo + (tg0 + t) * p.tile_units, nu = min(p.tile_units, hi - u0);
-                for (int sc = 0; sc < acw; sc += p.ksub) {
-                    const int kw = min(p.ksub, acw - sc), k0 = ac0 + sc;
-                    const uint32_t row_bytes = (uint32_t)kw * (uint32_t)sizeof(WT);
-                    const int nrows = J.epi == EPI_GATEUP ? 2 * nu : nu;
-                    uint32_t dst, bar;
-                    ring_claim(D, S, ring, row_bytes * (uint32_t)nrows, dst, bar);
-                    if (lane < 16) {
-                        const WT *src = nullptr;
-                        if (J.epi == EPI_GATEUP) {
-                            const int i = lane & 7;
-                            if (i < nu) src = reinterpret_cast<const WT *>(lane < 8 ? J.W : J.W2) + (size_t)(u0 + i) * J.kdim + k0;
-                        } else if (lane < nu) {
-                            src = reinterpret_cast<const WT *>(J.W) + (size_t)(u0 + lane) * J.kdim + k0;
-                        }
-                        if (src) bulk_g2s(dst + (uint32_t)lane * kRowPitch, src, row_bytes, bar);
-                    }
-                    ring.pos += 1;
-                }
+    for (int tg0 = 0; tg0 < p.n_tiles; tg0 += p.tpg) {
+        const int tg = min(p.tpg, p.n_tiles - tg0);
+        for (int t = 0; t < tg; ++t) {
+            const int u0 = lo + (tg0 + t) * p.tile_units, nu = min(p.tile_units, hi - u0);
+            for (int it = 0; it < p.ipt; ++it) {
+                const WT *src;
+                const int nrows = item_rows<WT>(J, p, u0, nu, it, src);
+                const uint32_t bytes = (uint32_t)(nrows * p.row_bytes);
+                uint32_t dst, bar;
+                ring_claim(D, S, ring, bytes, dst, bar);        // an item without valid rows is only announced
+                if (lane == 0 && bytes != 0u) bulk_g2s(dst, src, bytes, bar);
+                ring.pos += 1;
             }
         }
     }
@@ -555,46 +572,26 @@ __device__ void stage_acts<bf16>(const Dev &D, const Smem &S, const GemvJob &J, 
     csync();
 }
 
-// bf16 weights.  Warp (tile, part): A = 16 weight rows x 32 columns per step out of the ring slot (lane
-// g = lane/4, t = lane%4 loads 16 bytes = 8 consecutive columns of rows g and g+8; the same column
-// permutation is applied to the activation fragments, so the products pair up), B = activations of 8 tokens.
-template <int NT>
-__device__ __forceinline__ void mma_item_bf16(const char *slot, const char *acts, int pitch, int kcol0, int kw, int part,
-                                              int parts, int M, float (&acc)[NT][2][4]) {
-    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const uint32_t wa_addr = smem_u32(slot) + (uint32_t)g * kRowPitch + (uint32_t)t * 16u;
-    const uint32_t wb_addr = wa_addr + 8u * kRowPitch;
-    const uint32_t x_addr = smem_u32(acts) + (uint32_t)(kcol0 + t * 8) * 4u;
-    const int nkb = kw >> 5;
-    for (int kb = part; kb < nkb; kb += parts) {
-        const uint4 wa = lds_u4(wa_addr + (uint32_t)kb * 64u), wb = lds_u4(wb_addr + (uint32_t)kb * 64u);
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const int m = nt * 8 + g;
-            uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = xa;
-            if (m < M) {
-                const uint32_t a = x_addr + (uint32_t)m * (uint32_t)pitch + (uint32_t)kb * 128u;
-                xa = lds_u4(a);
-                xb = lds_u4(a + 16u);
-            }
-            mma16816(acc[nt][0], wa.x, wb.x, wa.y, wb.y, xa.x, xa.y);
-            mma16816(acc[nt][1], wa.x, wb.x, wa.y, wb.y, xa.z, xa.w);
-            mma16816(acc[nt][0], wa.z, wb.z, wa.w, wb.w, xb.x, xb.y);
-            mma16816(acc[nt][1], wa.z, wb.z, wa.w, wb.w, xb.z, xb.w);
-        }
-    }
+// shared-memory address of layout row `row` of the tile whose first item sits at ring position pos_tile
+__device__ __forceinline__ uint32_t tile_row_addr(const Smem &S, const SegPlan &p, uint32_t pos_tile, int row) {
+    const int ns = S.n_slots;
+    row = min(row, p.tile_rows - 1);     // rows past a short tile read its last row; their products are never used
+    int slot = (int)(pos_tile % (uint32_t)ns) + (row >> p.rpi_shift);
+    if (slot >= ns) slot -= ns;
+    return smem_u32(S.ring) + (uint32_t)slot * kSlotBytes + (uint32_t)((row & ((1 << p.rpi_shift) - 1)) * p.row_bytes);
 }
 
-// The same products for all items of one tile at once: the warp's column blocks (32 columns each) are spread
-// over the items of the tile, which sit in consecutive ring slots from position pos_tile; U blocks are in
-// flight together, each with accumulators of its own.
+// bf16 weights.  Warp (tile, part): A = 16 weight rows x 32 columns per step out of the ring (lane g = lane/4,
+// t = lane%4 loads 16 bytes = 8 consecutive columns of rows g and g+8; the same column permutation is applied
+// to the activation fragments, so the products pair up), B = activations of 8 tokens.  The warp takes the
+// column blocks part, part + parts, ... of columns [k0, k0 + 32 * n_kb); U blocks are in flight together, each
+// with accumulators of its own.
 template <int NT, int U>
-__device__ __forceinline__ void mma_tile_bf16(const Smem &S, uint32_t pos_tile, const char *acts, int pitch, int total_kb, int part,
+__device__ __forceinline__ void mma_tile_bf16(uint32_t row_a, uint32_t row_b, const char *acts, int pitch, int k0, int n_kb, int part,
                                               int parts, int M, float (&acc)[NT][2][4]) {
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const uint32_t ring0 = smem_u32(S.ring), lane_off = (uint32_t)g * kRowPitch + (uint32_t)t * 16u;
+    const uint32_t wa0 = row_a + (uint32_t)(k0 * 2 + t * 16), wb0 = row_b + (uint32_t)(k0 * 2 + t * 16);
     const uint32_t x_base = smem_u32(acts) + (uint32_t)t * 32u;
-    const int ns = S.n_slots, s0 = (int)(pos_tile % (uint32_t)ns);
     float au[U][NT][2][4];
 #pragma unroll
     for (int u = 0; u < U; ++u)
@@ -602,21 +599,18 @@ __device__ __forceinline__ void mma_tile_bf16(const Smem &S, uint32_t pos_tile, 
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int q = 0; q < 4; ++q) au[u][nt][0][q] = au[u][nt][1][q] = 0.f;
-    for (int q0 = part; q0 < total_kb; q0 += parts * U) {
+    for (int q0 = part; q0 < n_kb; q0 += parts * U) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int kbg = q0 + u * parts;
-            if (kbg < total_kb) {
-                int slot = s0 + (kbg >> 4);
-                if (slot >= ns) slot -= ns;
-                const uint32_t wa_addr = ring0 + (uint32_t)slot * kSlotBytes + lane_off + (uint32_t)(kbg & 15) * 64u;
-                const uint4 wa = lds_u4(wa_addr), wb = lds_u4(wa_addr + 8u * kRowPitch);
+            const int kb = q0 + u * parts;
+            if (kb < n_kb) {
+                const uint4 wa = lds_u4(wa0 + (uint32_t)kb * 64u), wb = lds_u4(wb0 + (uint32_t)kb * 64u);
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const int m = nt * 8 + g;
                     uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = xa;
                     if (m < M) {
-                        const uint32_t a = x_base + (uint32_t)m * (uint32_t)pitch + (uint32_t)kbg * 128u;
+                        const uint32_t a = x_base + (uint32_t)m * (uint32_t)pitch + (uint32_t)kb * 128u;
                         xa = lds_u4(a);
                         xb = lds_u4(a + 16u);
                     }
@@ -641,7 +635,7 @@ __device__ __forceinline__ void mma_tile_bf16(const Smem &S, uint32_t pos_tile, 
 // Returns the value before any gain of the next stage is applied (the residual stream's new value for EPI_ADD).
 template <typename WT>
 __device__ __forceinline__ float epilogue_store(const GemvJob &J, int m, int u, float v, float v2, float inv, uint32_t tag_out,
-                                                bool have_prev = false, float hprev = 0.f) {
+                                                bool have_prev = false, float hprev = 0.f, float gprev = 1.f) {
     float *o = J.out + (size_t)m * J.out_ld + u;
     float r, pub;
     if (J.epi == EPI_STORE) pub = r = v;
@@ -651,7 +645,7 @@ __device__ __forceinline__ float epilogue_store(const GemvJob &J, int m, int u, 
         pub = r = (have_prev ? hprev : __ldcg(hm)) + v;
         __stcg(hm, r);
         // bf16 models: the reader's RMSNorm gain is applied here, once, instead of by every reader
-        if (sizeof(WT) == 2 && J.gain_out != nullptr) pub = r * to_f(reinterpret_cast<const WT *>(J.gain_out)[u]);
+        if (sizeof(WT) == 2 && J.gain_out != nullptr) pub = r * (have_prev ? gprev : to_f(reinterpret_cast<const WT *>(J.gain_out)[u]));
     } else {   // EPI_HEADY: residual on the normalised input (this CTA has already waited for that word);
                // inv = 1 / rms(x[m]), times gain[u] where the input is published without its gain (fp32 models)
         pub = r = read_word<WT>(ld_relaxed_u32(J.x + (size_t)m * J.kdim + u)) * inv + silu_f(v);
@@ -663,7 +657,7 @@ __device__ __forceinline__ float epilogue_store(const GemvJob &J, int m, int u, 
 template <typename WT, int NT>
 static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi,
                                      uint32_t serial) {
-    const SegPlan p = seg_plan<WT>(J, lo, hi);
+    const SegPlan p = seg_plan<WT>(S, J, lo, hi);
     const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int kca = min(J.kdim, D.kca);
     const bool one_chunk = kca >= J.kdim;
@@ -672,26 +666,40 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
     constexpr int NP = NT * 8;
     bool staged = false;
     float ss_share = 0.f;
-    for (int tg0 = 0; tg0 < p.n_tiles; tg0 += kConsumerWarps) {
-        const int tg = min(kConsumerWarps, p.n_tiles - tg0);
+    for (int tg0 = 0; tg0 < p.n_tiles; tg0 += p.tpg) {
+        const int tg = min(p.tpg, p.n_tiles - tg0);
         const int parts = kConsumerWarps / tg;
         const int my_tile = warp / parts, my_part = warp - my_tile * parts;   // my_tile >= tg: idle warp
+        const uint32_t pos0 = ring.pos;      // the group's items: tile tl at positions pos0 + tl * ipt ...
+        bool landed = false;
         float acc[NT][2][4];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int q = 0; q < 4; ++q) acc[nt][0][q] = acc[nt][1][q] = 0.f;
-        // the residual stream's old values of this group's outputs, fetched while the inputs are awaited
-        const int outs = tg * p.tile_units * M;     // (tile, token, unit)
-        float hpre[4] = {0.f, 0.f, 0.f, 0.f};
-        if (J.epi == EPI_ADD) {
+        // The static part of the epilogue is done now, while the inputs are still on their way: where this
+        // thread's first four outputs go (output i = (tile, token, unit), unit fastest), and what they need from
+        // global memory (the residual stream's old value, the gain applied to the published copy).
+        const int outs = tg * p.tile_units * M;
+        const int tu_shift = p.tu_shift, tu_mask = p.tile_units - 1;
+        const int n_out_iter = (outs + kConsumerThreads - 1) / kConsumerThreads;
+        int o_n[4], o_u[4], o_red[4];
+        float hpre[4], gpre[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int i = tid + q * kConsumerThreads;
-                if (i < outs) {
-                    const int tl = i / (p.tile_units * M), rem = i - tl * p.tile_units * M;
-                    const int n = rem / p.tile_units, u = lo + (tg0 + tl) * p.tile_units + rem - n * p.tile_units;
-                    if (u < hi) hpre[q] = __ldcg(J.hm + (size_t)n * J.out_ld + u);
+        for (int q = 0; q < 4; ++q) {
+            const int i = tid + q * kConsumerThreads;
+            o_n[q] = 0; o_u[q] = -1; o_red[q] = 0; hpre[q] = 0.f; gpre[q] = 1.f;
+            if (i < outs) {
+                const int ui = i & tu_mask, rest = i >> tu_shift, tl = rest / M, n = rest - tl * M;
+                const int u = lo + (tg0 + tl) * p.tile_units + ui;
+                o_n[q] = n;
+                o_red[q] = tl * parts * NP * 16 + n * 16 + ui;
+                if (u < hi) {
+                    o_u[q] = u;
+                    if (J.epi == EPI_ADD) {
+                        hpre[q] = __ldcg(J.hm + (size_t)n * J.out_ld + u);
+                        if (J.gain_out != nullptr) gpre[q] = to_f(reinterpret_cast<const WT *>(J.gain_out)[u]);
+                    }
                 }
             }
         }
@@ -704,34 +712,27 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
                 staged = true;
                 if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
             }
-            const int nsub = (acw + p.ksub - 1) / p.ksub;
-            if (one_chunk && tg * nsub <= S.n_slots) {
-                // All items of the stage are in the ring at once (each in a slot of its own).  A warp waits only
-                // for the items of its tile and multiplies them in one sweep.  A warp that does not read an item
-                // frees it at once: the previous item of that slot was freed by every warp before the barrier at
-                // the start of this stage, so no arrival can fall into the wrong phase.
-                constexpr int U = NT == 1 ? 4 : (NT == 2 ? 2 : 1);
-                const uint32_t pos0 = ring.pos;
-                if (my_tile < tg) {
+            // All items of the group are in the ring at once, each in a slot of its own.  A warp waits only for
+            // the items of its tile (once, before the first chunk of activations is multiplied).
+            if (my_tile < tg) {
+                if (!landed) {
                     Ring r;
-                    for (int i = 0; i < nsub; ++i) { r.pos = pos0 + (uint32_t)(my_tile * nsub + i); ring_wait(D, S, r); }
-                    mma_tile_bf16<NT, U>(S, pos0 + (uint32_t)(my_tile * nsub), S.acts, pitch, acw >> 5, my_part, parts, M, acc);
+                    for (int i = 0; i < p.ipt; ++i) { r.pos = pos0 + (uint32_t)(my_tile * p.ipt + i); ring_wait(D, S, r); }
+                    landed = true;
                 }
-                __syncwarp();
-                if (lane == 0)
-                    for (int i = 0; i < tg * nsub; ++i) mbar_arrive(S.empty0 + 8u * ring_slot(S, pos0 + (uint32_t)i));
-                ring.pos = pos0 + (uint32_t)(tg * nsub);
-            } else {
-                for (int tl = 0; tl < tg; ++tl) {
-                    for (int sc = 0; sc < acw; sc += p.ksub) {
-                        const int kw = min(p.ksub, acw - sc);
-                        const char *slot = ring_wait(D, S, ring);
-                        if (tl == my_tile) mma_item_bf16<NT>(slot, S.acts, pitch, sc, kw, my_part, parts, M, acc);
-                        ring_release(S, ring);
-                    }
-                }
+                constexpr int U = NT == 1 ? 4 : (NT == 2 ? 2 : 1);
+                const uint32_t pos_tile = pos0 + (uint32_t)(my_tile * p.ipt);
+                mma_tile_bf16<NT, U>(tile_row_addr(S, p, pos_tile, g), tile_row_addr(S, p, pos_tile, g + 8), S.acts, pitch, ac0,
+                                     acw >> 5, my_part, parts, M, acc);
             }
         }
+        // Every warp frees every item of the group; a warp that did not read an item does so without waiting
+        // for it: the previous item of that slot was freed by all warps before the barrier that opened this
+        // group's staging, so no arrival can fall into the wrong phase.
+        __syncwarp();
+        if (lane == 0)
+            for (int i = 0; i < tg * p.ipt; ++i) mbar_arrive(S.empty0 + 8u * ring_slot(S, pos0 + (uint32_t)i));
+        ring.pos = pos0 + (uint32_t)(tg * p.ipt);
         // cross-warp reduction through the activation area, then the epilogue
         csync();
         float *red = reinterpret_cast<float *>(S.acts);   // [warp][NP][16]
@@ -749,37 +750,52 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
         }
         if (gain != nullptr && tid < M) S.ss[tid] = 1.0f / sqrtf(S.ss[tid] / (float)J.kdim + D.eps);   // restaged, hence raw, in every tile group
         csync();
-        float *hv = red + (size_t)kConsumerWarps * NP * 16;    // new values of the residual stream, for their squares
+        float *ssg = red + (size_t)kConsumerWarps * NP * 16;   // [tile][token] sums of squares of the new residual values
         const bool want_ss = J.epi == EPI_ADD && J.gain_out != nullptr;
-        for (int i = tid; i < outs; i += kConsumerThreads) {
-            const int tl = i / (p.tile_units * M), rem = i - tl * p.tile_units * M;
-            const int n = rem / p.tile_units, ui = rem - n * p.tile_units;
-            const int u = lo + (tg0 + tl) * p.tile_units + ui;
+        for (int q = 0; q < n_out_iter; ++q) {
+            const int i = tid + q * kConsumerThreads;
+            int n, u, ro;
+            if (q < 4) {
+                n = q == 0 ? o_n[0] : q == 1 ? o_n[1] : q == 2 ? o_n[2] : o_n[3];
+                u = q == 0 ? o_u[0] : q == 1 ? o_u[1] : q == 2 ? o_u[2] : o_u[3];
+                ro = q == 0 ? o_red[0] : q == 1 ? o_red[1] : q == 2 ? o_red[2] : o_red[3];
+            } else {
+                const int ui = i & tu_mask, rest = i >> tu_shift, tl = rest / M;
+                n = rest - tl * M;
+                u = lo + (tg0 + tl) * p.tile_units + ui;
+                ro = tl * parts * NP * 16 + n * 16 + ui;
+                if (i >= outs || u >= hi) u = -1;
+            }
             float r = 0.f;
-            if (u < hi) {
+            if (u >= 0) {
                 float v = 0.f, v2 = 0.f;
-                for (int q = 0; q < parts; ++q) {
-                    const float *rr = red + (size_t)(tl * parts + q) * NP * 16 + n * 16;
-                    v += rr[ui];
-                    if (J.epi == EPI_GATEUP) v2 += rr[ui + 8];
+                for (int pq = 0; pq < parts; ++pq) {
+                    const float *rr = red + ro + pq * NP * 16;
+                    v += rr[0];
+                    if (J.epi == EPI_GATEUP) v2 += rr[8];
                 }
                 float inv = 1.f;
                 if (gain != nullptr) { inv = S.ss[n]; v *= inv; v2 *= inv; }
-                const int q = (i - tid) / kConsumerThreads;
-                r = epilogue_store<WT>(J, n, u, v, v2, inv, tag_out, q < 4, q == 0 ? hpre[0] : q == 1 ? hpre[1] : q == 2 ? hpre[2] : hpre[3]);
+                r = epilogue_store<WT>(J, n, u, v, v2, inv, tag_out, q < 4,
+                                       q == 0 ? hpre[0] : q == 1 ? hpre[1] : q == 2 ? hpre[2] : hpre[3],
+                                       q == 0 ? gpre[0] : q == 1 ? gpre[1] : q == 2 ? gpre[2] : gpre[3]);
             }
-            if (want_ss) hv[i] = r;
+            if (want_ss) {
+                // the units of one (tile, token) sit in adjacent lanes: a fixed tree adds their squares
+                float sq = r * r;
+                sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+                sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+                if (p.tile_units >= 8) sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+                if (p.tile_units == 16) sq += __shfl_xor_sync(0xffffffffu, sq, 8);
+                if ((i & tu_mask) == 0 && i < outs) ssg[i >> tu_shift] = sq;
+            }
         }
         if (want_ss) {
             // this CTA's share of the sum of squares of every row, in a fixed order
             csync();
             if (tid < M) {
-                for (int tl = 0; tl < tg; ++tl)
-                    for (int ui = 0; ui < p.tile_units; ++ui) {
-                        const float r = hv[(tl * M + tid) * p.tile_units + ui];
-                        ss_share = fmaf(r, r, ss_share);
-                    }
-                if (tg0 + kConsumerWarps >= p.n_tiles) st_relaxed_u32(D.sspub + (size_t)blockIdx.x * M + tid, tagged(ss_share, tag_out));
+                for (int tl = 0; tl < tg; ++tl) ss_share += ssg[tl * M + tid];
+                if (tg0 + p.tpg >= p.n_tiles) st_relaxed_u32(D.sspub + (size_t)blockIdx.x * M + tid, tagged(ss_share, tag_out));
             }
         }
     }
@@ -792,7 +808,7 @@ template <int MT>
 __device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi,
                                     uint32_t serial) {
     constexpr int PPW = (8 + kConsumerWarps - 1) / kConsumerWarps;   // pairs per warp
-    const SegPlan p = seg_plan<float>(J, lo, hi);
+    const SegPlan p = seg_plan<float>(S, J, lo, hi);
     const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t tag_in = tag_of(serial, J.in), tag_out = tag_of(serial, J.outt);
     const float *gain = reinterpret_cast<const float *>(J.gain);
@@ -802,62 +818,71 @@ __device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, con
     csync();
     if (gain != nullptr && tid < M) S.ss[tid] = 1.0f / sqrtf(S.ss[tid] / (float)J.kdim + D.eps);
     csync();
-    for (int tl = 0; tl < p.n_tiles; ++tl) {
-        float acc[PPW][2][MT];
+    if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
+    for (int tg0 = 0; tg0 < p.n_tiles; tg0 += p.tpg) {
+        const int tg = min(p.tpg, p.n_tiles - tg0);
+        const uint32_t pos0 = ring.pos;
+        for (int tl = 0; tl < tg; ++tl) {
+            const uint32_t pos_tile = pos0 + (uint32_t)(tl * p.ipt);
+            Ring r;
+            for (int i = 0; i < p.ipt; ++i) { r.pos = pos_tile + (uint32_t)i; ring_wait(D, S, r); }
+            float acc[PPW][2][MT];
 #pragma unroll
-        for (int s = 0; s < PPW; ++s)
+            for (int s2 = 0; s2 < PPW; ++s2)
 #pragma unroll
-            for (int n = 0; n < MT; ++n) acc[s][0][n] = acc[s][1][n] = 0.f;
-        for (int sc = 0; sc < J.kdim; sc += p.ksub) {
-            const int kw = min(p.ksub, J.kdim - sc);
-            const char *slot = ring_wait(D, S, ring);
+                for (int n = 0; n < MT; ++n) acc[s2][0][n] = acc[s2][1][n] = 0.f;
 #pragma unroll
-            for (int s = 0; s < PPW; ++s) {
-                const int q = warp + s * kConsumerWarps;
+            for (int s2 = 0; s2 < PPW; ++s2) {
+                const int q = warp + s2 * kConsumerWarps;
                 if (q < 8) {
-                    const float *ra = reinterpret_cast<const float *>(slot + (size_t)q * kRowPitch);
-                    const float *rb = reinterpret_cast<const float *>(slot + (size_t)(q + 8) * kRowPitch);
-                    for (int k = lane * 4; k < kw; k += 128) {
-                        const float4 wa = *reinterpret_cast<const float4 *>(ra + k), wb = *reinterpret_cast<const float4 *>(rb + k);
+                    const uint32_t ra = tile_row_addr(S, p, pos_tile, q), rb = tile_row_addr(S, p, pos_tile, q + 8);
+                    for (int k = lane * 4; k < J.kdim; k += 128) {
+                        const uint4 ua = lds_u4(ra + (uint32_t)k * 4u), ub = lds_u4(rb + (uint32_t)k * 4u);
+                        const float4 wa = make_float4(__uint_as_float(ua.x), __uint_as_float(ua.y), __uint_as_float(ua.z), __uint_as_float(ua.w));
+                        const float4 wb = make_float4(__uint_as_float(ub.x), __uint_as_float(ub.y), __uint_as_float(ub.z), __uint_as_float(ub.w));
 #pragma unroll
                         for (int n = 0; n < MT; ++n) {
                             if (n < M) {
-                                const float4 x = *reinterpret_cast<const float4 *>(S.acts + (size_t)n * pitch + (size_t)(sc + k) * 4);
-                                acc[s][0][n] = fmaf(wa.x, x.x, acc[s][0][n]); acc[s][0][n] = fmaf(wa.y, x.y, acc[s][0][n]);
-                                acc[s][0][n] = fmaf(wa.z, x.z, acc[s][0][n]); acc[s][0][n] = fmaf(wa.w, x.w, acc[s][0][n]);
-                                acc[s][1][n] = fmaf(wb.x, x.x, acc[s][1][n]); acc[s][1][n] = fmaf(wb.y, x.y, acc[s][1][n]);
-                                acc[s][1][n] = fmaf(wb.z, x.z, acc[s][1][n]); acc[s][1][n] = fmaf(wb.w, x.w, acc[s][1][n]);
+                                const float4 x = *reinterpret_cast<const float4 *>(S.acts + (size_t)n * pitch + (size_t)k * 4);
+                                acc[s2][0][n] = fmaf(wa.x, x.x, acc[s2][0][n]); acc[s2][0][n] = fmaf(wa.y, x.y, acc[s2][0][n]);
+                                acc[s2][0][n] = fmaf(wa.z, x.z, acc[s2][0][n]); acc[s2][0][n] = fmaf(wa.w, x.w, acc[s2][0][n]);
+                                acc[s2][1][n] = fmaf(wb.x, x.x, acc[s2][1][n]); acc[s2][1][n] = fmaf(wb.y, x.y, acc[s2][1][n]);
+                                acc[s2][1][n] = fmaf(wb.z, x.z, acc[s2][1][n]); acc[s2][1][n] = fmaf(wb.w, x.w, acc[s2][1][n]);
                             }
                         }
                     }
                 }
             }
-            ring_release(S, ring);
-        }
-        const int u0 = lo + tl * p.tile_units;
+            const int u0 = lo + (tg0 + tl) * p.tile_units;
 #pragma unroll
-        for (int s = 0; s < PPW; ++s) {
-            const int q = warp + s * kConsumerWarps;
-            if (q >= 8) continue;
+            for (int s2 = 0; s2 < PPW; ++s2) {
+                const int q = warp + s2 * kConsumerWarps;
+                if (q >= 8) continue;
 #pragma unroll
-            for (int n = 0; n < MT; ++n) {
-                if (n < M) {
-                    float va = warp_sum(acc[s][0][n]), vb = warp_sum(acc[s][1][n]);
-                    if (lane == 0) {
-                        const float inv = gain != nullptr ? S.ss[n] : 1.f;
-                        va *= inv; vb *= inv;
-                        if (J.epi == EPI_GATEUP) {
-                            if (u0 + q < hi) epilogue_store<float>(J, n, u0 + q, va, vb, inv, tag_out);
-                        } else {
-                            if (u0 + q < hi)
-                                epilogue_store<float>(J, n, u0 + q, va, 0.f, J.epi == EPI_HEADY ? inv * gain[u0 + q] : inv, tag_out);
-                            if (u0 + q + 8 < hi)
-                                epilogue_store<float>(J, n, u0 + q + 8, vb, 0.f, J.epi == EPI_HEADY ? inv * gain[u0 + q + 8] : inv, tag_out);
+                for (int n = 0; n < MT; ++n) {
+                    if (n < M) {
+                        float va = warp_sum(acc[s2][0][n]), vb = warp_sum(acc[s2][1][n]);
+                        if (lane == 0) {
+                            const float inv = gain != nullptr ? S.ss[n] : 1.f;
+                            va *= inv; vb *= inv;
+                            if (J.epi == EPI_GATEUP) {
+                                if (u0 + q < hi) epilogue_store<float>(J, n, u0 + q, va, vb, inv, tag_out);
+                            } else {
+                                if (q < p.tile_units && u0 + q < hi)
+                                    epilogue_store<float>(J, n, u0 + q, va, 0.f, J.epi == EPI_HEADY ? inv * gain[u0 + q] : inv, tag_out);
+                                if (q + 8 < p.tile_units && u0 + q + 8 < hi)
+                                    epilogue_store<float>(J, n, u0 + q + 8, vb, 0.f, J.epi == EPI_HEADY ? inv * gain[u0 + q + 8] : inv, tag_out);
+                            }
                         }
                     }
                 }
             }
         }
+        // every warp has read every item of the group
+        __syncwarp();
+        if (lane == 0)
+            for (int i = 0; i < tg * p.ipt; ++i) mbar_arrive(S.empty0 + 8u * ring_slot(S, pos0 + (uint32_t)i));
+        ring.pos = pos0 + (uint32_t)(tg * p.ipt);
     }
 }
 
