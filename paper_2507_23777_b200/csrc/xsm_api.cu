@@ -239,7 +239,7 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     if (attn > need) need = attn;
     const int samp = (((c.vocab + 3) & ~3) + 256) * 4;
     if (samp > need) need = samp;
-    const int full = M * (kmax * 4 + 16);                             // all activations of the widest projection
+    const int full = M * (kmax * 4 + 16) + (kConsumerWarps * np * 16 + kConsumerWarps * M) * 4;   // all activations of the widest projection, and the partial products behind them
     int acts = full > need ? full : need;
     if (acts > avail - kMinSlots * kSlotBytes) acts = avail - kMinSlots * kSlotBytes;
     if (acts < need) return "the shape needs more shared memory than one CTA has";

@@ -358,13 +358,12 @@ __device__ __forceinline__ GemvJob job_at(const Dev &D, const Smem &S, int idx, 
 // ------------------------------------------------------------------------------ projection: plan
 
 // The rows of a stage's jobs form one range that is cut evenly over the CTAs; a CTA's piece of one job is a
-// segment.  A segment is processed as tile groups of up to 8 tiles (a tile: 16 weight rows, or 8 gate rows
-// + 8 up rows), the activations in chunks of D.kca columns, a tile in items of at most kItemRowBytes per row.
+// segment.  A segment is processed as groups of tiles, the activations in chunks of D.kca columns.
 // A tile has up to 16 layout rows (16 weight rows, or 8 gate rows then 8 up rows; 8 or 4 rows where a row is
 // longer than 4 KB, so that a tile never exceeds four slots).  An item is `rpi` consecutive layout rows at full
 // width: consecutive weight rows are contiguous in memory, so one bulk copy brings an item.  A tile group
 // (`tpg` tiles at most) has all its items in the ring at once.
-constexpr int kItemBytes = 16384;
+constexpr int kItemBytes = kSlotBytes;
 struct SegPlan {
     int tile_units;   // units (output rows) per tile: 16, 8 or 4; 8 for gate/up
     int tu_shift;     // log2(tile_units)
@@ -735,8 +734,12 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
         ring.pos = pos0 + (uint32_t)(tg * p.ipt);
         // cross-warp reduction through the activation area, then the epilogue
         csync();
-        float *red = reinterpret_cast<float *>(S.acts);   // [warp][NP][16]
-        staged = false;
+        // [warp][NP][16] partial products: behind the staged activations when both fit (then a following tile
+        // group finds the activations still in place), else over them
+        const int red_bytes = (kConsumerWarps * NP * 16 + kConsumerWarps * M) * 4;
+        const bool red_apart = one_chunk && M * (J.kdim * 4 + 16) + red_bytes <= D.acts_bytes;
+        float *red = reinterpret_cast<float *>(S.acts + (red_apart ? M * (J.kdim * 4 + 16) : 0));
+        if (!red_apart) staged = false;
         if (my_tile < tg) {
             float *r = red + (size_t)warp * NP * 16;
 #pragma unroll

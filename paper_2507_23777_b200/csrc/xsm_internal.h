@@ -13,14 +13,10 @@ constexpr int kMaxDraft = 16;                        // size of the histogram ro
 constexpr int kMaxTokens = 128;                      // largest M = batch * (K + 1)
 constexpr int kMaxBatch = 128;
 
-// Ring of shared-memory slots filled by bulk copies.  A weight item is up to 16 rows of up to 1024 bytes,
-// rows kRowPitch bytes apart (1024 + 64: rows g and g+1 land in different halves of a 128-byte bank line).
-// A cache item is one (page, head) tile of keys followed by the tile of values (or one of them when both do
-// not fit).
-constexpr int kItemRows = 16;
-constexpr int kItemRowBytes = 1024;
-constexpr int kRowPitch = kItemRowBytes + 64;
-constexpr int kSlotBytes = kItemRows * kRowPitch;    // 17408
+// Ring of shared-memory slots filled by bulk copies.  A weight item is a run of consecutive weight rows at full
+// width (at most kSlotBytes, one bulk copy); a cache item is one (page, head) tile of keys followed by the tile
+// of values (or one of them when both do not fit).
+constexpr int kSlotBytes = 16384;
 constexpr int kMaxSlots = 12;
 constexpr int kSmemHeader = 2048;                    // barriers and per-step scalars
 constexpr int kSmemMax = 227 * 1024;
