@@ -226,7 +226,7 @@ def run_gpu(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 weights and cache, f32 arithmetic" if cfg["dtype"] == 1 else "f32", "data": "synthetic",
+        "dtype": "bf16 weights, fp16 cache, f32 arithmetic" if cfg["dtype"] == 1 else "f32", "data": "synthetic",
         "config": {"workload": f"config {args.config} ({cfg['name']}): batch {B}, K={K} heads, {T} tokens per mesh, "
                                f"verify_mode {cfg['verify_mode']}, k={cfg['k_accept']}, T={cfg['temperature']}",
                    "weights": "iid N(0, sigma) as configured (heads untrained)", "l2": "inputs larger than L2 "
@@ -237,9 +237,10 @@ def run_gpu(args):
                 "d2h_bytes_per_step": int(h_tokens.numel() * 4 + h_lengths.numel() * 4)},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": metrics.measured_traffic(args.config),
+                     "frac": achieved / peaks["hbm_gbs"],
+                     "traffic": metrics.measured_traffic(args.config if not args.k0 else -1, bytes_per_step * steps_total / B / n_step_launches),
                      "peak_source": f"{which} copy bandwidth (MEASURED_PEAKS.json)" if which == "measured" else "fallback",
-                     "kernel": "step_kernel (persistent; one launch = up to 64 decoding steps)",
+                     "kernel": "xsm::step_kernel (persistent, 148 CTAs; one launch = up to 64 decoding steps)",
                      "bytes_per_launch": bytes_per_step * steps_total / B / n_step_launches,
                      "avg_launch_ms": kernel_ms / n_step_launches},
         "clocks": clocks,

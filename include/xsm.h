@@ -54,15 +54,16 @@ typedef enum {
  *   per head i=1..K: W1[head_hidden,d] Wout[V,head_hidden]
  * Block (Sec. 4.1): pre-norm residual, self-attention (RoPE, causal, cached),
  * cross-attention to c, gated feed-forward network; RMSNorm gains g*.
- * Requirements: n_heads*d_head == d_model, head_hidden == d_model, d_model,
- * d_ff and d_cond multiples of 32, d_head even and <= 128, page_size == 64 or
- * another multiple of 16, n_draft <= XSM_MAX_DRAFT. */
+ * Requirements: n_heads*d_head == d_model, head_hidden == d_model, d_model and d_ff multiples of 128 with rows
+ * of at most 16 KB (d_model additionally at most 4 KB per row), d_cond a multiple of 32, d_head 32, 64 or 128,
+ * page_size a multiple of 32 with page_size*d_head <= 8192 (bf16) / 16384 (fp32), n_draft <= 15,
+ * max_batch*(n_draft+1) <= 128.  fp32 models (the parity configuration): at most 24 token rows per step. */
 typedef struct {
     int n_layers, d_model, n_heads, d_head, d_ff, vocab, n_cond, d_cond;
     int n_draft;        /* K; 0 = plain one-token-per-step decoding (Table 3 row A) */
     int head_hidden;
     int head_kind;      /* 0: MLP head, logits = Wout (g + SiLU(W1 g)) (Table 3 rows B, C) */
-    int dtype;          /* 0: fp32 weights and cache; 1: bf16 weights and cache, fp32 arithmetic */
+    int dtype;          /* 0: fp32 weights and cache; 1: bf16 weights, fp16 cache, fp32 arithmetic */
     int page_size;      /* tokens per cache page */
     int max_batch;
     int max_seq_len;    /* largest s; the cache holds max_seq_len + K + 1 positions per sequence */

@@ -132,6 +132,8 @@ const char *check_config(const xsm_model_config &c) {
     if (c.d_cond % 32) return "d_cond must be a multiple of 32";
     if ((long long)(c.d_model > c.d_ff ? c.d_model : c.d_ff) * (c.dtype == 1 ? 2 : 4) > 16384)
         return "d_model and d_ff are limited to 16 KB per weight row (8192 bf16 or 4096 fp32 elements)";
+    if ((long long)c.d_model * (c.dtype == 1 ? 2 : 4) > 4096)
+        return "d_model is limited to 4 KB per weight row (2048 bf16 or 1024 fp32 elements)";
     if (c.d_head != 32 && c.d_head != 64 && c.d_head != 128) return "d_head must be 32, 64 or 128";
     if (c.n_draft < 0 || c.n_draft >= XSM_MAX_DRAFT) return "n_draft must be in [0, 15]";
     if (c.head_hidden != c.d_model) return "head_hidden must equal d_model (the head block is residual)";

@@ -22,10 +22,13 @@ def speedup(scr: float, latency_base: float, latency_spec: float) -> float:
     return scr * latency_base / latency_spec
 
 
-# DRAM traffic of one decoding step measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum of the
-# step kernel, scaled to one step); None until a capture exists for that configuration.  See profiles/.
-_TRAFFIC_PER_LAUNCH = {}
+# DRAM traffic of the step kernel measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum of one launch of 64
+# decoding steps at contexts 0..63, see profiles/), as a ratio to the algorithmic bytes of the same launch.  Traffic
+# grows in proportion to the units processed (weights once per step plus the cache), so a launch of the benchmark is
+# its algorithmic bytes times this ratio.  None: no capture of the current kernel for that configuration.
+_TRAFFIC_RATIO = {2: (63.659044e9 + 80.542464e6) / (64 * 981.57e6 + 98304.0 * sum(range(64)))}
 
 
-def measured_traffic(config_index: int):
-    return _TRAFFIC_PER_LAUNCH.get(config_index)
+def measured_traffic(config_index: int, algorithmic_bytes_per_launch: float):
+    r = _TRAFFIC_RATIO.get(config_index)
+    return None if r is None else r * algorithmic_bytes_per_launch
