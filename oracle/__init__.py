@@ -9,6 +9,7 @@ from __future__ import annotations
 import ctypes as C
 import os
 import subprocess
+import weakref
 
 import numpy as np
 
@@ -152,6 +153,7 @@ class Oracle:
         assert weights.size == lib().orc_weight_elements(C.byref(self.mc))
         self._w = weights
         self._h = C.c_void_p()
+        self._seqs = weakref.WeakSet()
         rc = lib().orc_create(C.byref(self.mc), weights.ctypes.data_as(C.c_void_p), C.byref(self._h))
         if rc:
             raise RuntimeError(f"orc_create failed: {rc}")
@@ -160,7 +162,9 @@ class Oracle:
         return lib().orc_free_pages(self._h)
 
     def new_seq(self, cond: np.ndarray, seq_id: int = 0, max_positions: int | None = None) -> "Seq":
-        return Seq(self, cond, seq_id, max_positions)
+        s = Seq(self, cond, seq_id, max_positions)
+        self._seqs.add(s)
+        return s
 
     def head(self, i: int, g: np.ndarray) -> np.ndarray:
         g = np.ascontiguousarray(g, dtype=np.float32)
@@ -169,6 +173,9 @@ class Oracle:
         return out
 
     def close(self):
+        # sequences hand their pages back to the context: they go first, whatever order the collector picks
+        for s in list(getattr(self, "_seqs", ())):
+            s.close()
         if self._h:
             lib().orc_destroy(self._h)
             self._h = C.c_void_p()

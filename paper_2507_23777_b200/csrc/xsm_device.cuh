@@ -663,7 +663,7 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
     const uint32_t tag_in = tag_of(serial, J.in), tag_out = tag_of(serial, J.outt);
     const WT *gain = reinterpret_cast<const WT *>(J.gain);
     constexpr int NP = NT * 8;
-    bool staged = false;
+    bool staged = false, ss_raw = false;     // ss_raw: S.ss holds sums of squares that still await 1/sqrt
     float ss_share = 0.f;
     for (int tg0 = 0; tg0 < p.n_tiles; tg0 += p.tpg) {
         const int tg = min(p.tpg, p.n_tiles - tg0);
@@ -709,6 +709,7 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
                 stage_acts<WT>(D, S, J, ac0, acw, tag_in);
                 csync();
                 staged = true;
+                if (ac0 == 0) ss_raw = true;
                 if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
             }
             // All items of the group are in the ring at once, each in a slot of its own.  A warp waits only for
@@ -751,7 +752,9 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
                 r[(n0 + 1) * 16 + g + 8] = acc[nt][0][3] + acc[nt][1][3];
             }
         }
-        if (gain != nullptr && tid < M) S.ss[tid] = 1.0f / sqrtf(S.ss[tid] / (float)J.kdim + D.eps);   // restaged, hence raw, in every tile group
+        // a tile group that found the activations still staged also finds the inverse norms of the group before
+        if (gain != nullptr && ss_raw && tid < M) S.ss[tid] = 1.0f / sqrtf(S.ss[tid] / (float)J.kdim + D.eps);
+        ss_raw = false;
         csync();
         float *ssg = red + (size_t)kConsumerWarps * NP * 16;   // [tile][token] sums of squares of the new residual values
         const bool want_ss = J.epi == EPI_ADD && J.gain_out != nullptr;

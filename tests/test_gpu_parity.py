@@ -166,6 +166,57 @@ def test_config4_large_bf16_prefix(P):
     ls.close()
 
 
+@pytest.mark.parametrize("shape", ["heads of 64", "heads of 128, batch 2"])
+def test_long_context_split_attention(P, shape):
+    """Contexts of many pages: self-attention is split over several CTAs per head and merged (6 and 4 splits
+    here), on two-layer models with the widths of configurations 2 and 4.  The oracle is teacher-forced through
+    the whole run; logits and the cache are compared at the end, decisions at every step."""
+    if shape == "heads of 64":
+        cfg, batch, steps = inputs.config(2, n_layers=2, max_seq_len=2048), 1, 300
+    else:
+        cfg, batch, steps = inputs.config(4, n_layers=2, d_ff=2048, max_seq_len=2048, n_draft=3, n_cond=70), 2, 260
+    ls = P.LockStep(cfg, batch=batch)
+    ls.begin()
+    for it in range(steps):
+        ls.step(check_logits=it >= steps - 3, **BF16_TOL)
+    st = ls.ctx.xsm_debug_get_state()
+    assert st["len"].min() >= steps and ls.excused <= max(3, batch * steps // 20)
+    ls.compare_cache(layers=[1], **BF16_TOL)
+    ls.close()
+
+
+def _shape(d, H, dh, f, K, L=2, V=1500, C=40, **kw):
+    return dict(d_model=d, n_heads=H, d_head=dh, d_ff=f, d_cond=d, head_hidden=d, n_draft=K, n_layers=L, vocab=V,
+                n_cond=C, max_seq_len=256, **kw)
+
+
+SHAPES = {
+    "rows of 16 KB, two token rows": (_shape(2048, 16, 128, 8192, 1, L=1, V=1000), 1),
+    "sixteen token rows, heads of 32": (_shape(512, 16, 32, 1024, 15, V=777, C=33, page_size=32), 1),
+    "fifteen token rows": (_shape(1024, 16, 64, 4096, 4), 3),
+    "thirty-two token rows": (_shape(1024, 16, 64, 4096, 7, L=1), 4),
+    "forty token rows": (_shape(1024, 16, 64, 4096, 4, L=1), 8),
+    "a hundred and twenty token rows": (_shape(1024, 16, 64, 4096, 4, L=1), 24),
+    "rows of 3 KB and 12 KB": (_shape(1536, 12, 128, 6144, 2), 2),
+    "rows of 1280 and 3840 bytes": (_shape(640, 10, 64, 1920, 3), 1),
+    "no heads, five sequences": (_shape(768, 12, 64, 3072, 0), 5),
+    "several tile groups per projection": (_shape(2048, 16, 128, 2048, 3, V=3000), 2),
+}
+
+
+@pytest.mark.parametrize("shape", list(SHAPES))
+def test_shape_sweep_bf16(P, shape):
+    """Shapes between the five configurations: each makes the projections pick another tiling (rows per ring
+    item, tiles per group, token tiles, activation chunks).  Three steps, logits and cache against the oracle."""
+    ov, batch = SHAPES[shape]
+    ls = P.LockStep(inputs.config(2, **ov), batch=batch)
+    ls.begin()
+    for _ in range(3):
+        ls.step(**BF16_TOL)
+    ls.compare_cache(**BF16_TOL)
+    ls.close()
+
+
 def test_sampling_modes_lockstep(P):
     """Top-k acceptance with top-k / temperature resampling and threshold acceptance on the unit model."""
     for over in (dict(verify_mode=1, k_accept=3, sample_mode=1, k_sample=4, temperature=0.7, sigma=0.3),
