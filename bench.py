@@ -112,7 +112,7 @@ def run_reference(args):
     w = inputs.make_weights(cfg)
     cond = inputs.make_cond(cfg, 1)
     vals, sample = [], ""
-    per = max(4.0, min(30.0, 120.0 / max(1, args.steps + args.warmup)))
+    per = args.reference_seconds or max(4.0, min(30.0, 120.0 / max(1, args.steps + args.warmup)))
     for i in range(args.warmup + args.steps):
         v, steps, dt, cores = oracle_sample(cfg, w, cond, seconds_budget=per)
         if i >= args.warmup:
@@ -136,17 +136,15 @@ def run_reference(args):
 def run_gpu(args):
     import torch
     import torch.distributed as dist
-    from paper_2507_23777_b200 import binding, build
+    from paper_2507_23777_b200 import binding, build, replicas
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = replicas.env_ranks()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     build.build()
     cfg = workload(args)
-    cfg["seed"] = cfg["seed"] + 1000 * rank if world > 1 else cfg["seed"]   # every replica has its own meshes
+    cfg["seed"] = replicas.replica_seed(cfg["seed"], rank, world)           # every replica has its own meshes
     B, T, K = cfg["batch"], cfg["gen_tokens"], cfg["n_draft"]
     w = inputs.make_weights(dict(cfg, seed=args.config))
     cond = inputs.make_cond(cfg, B)
@@ -202,18 +200,16 @@ def run_gpu(args):
     ms_e2e = max(ev0.elapsed_time(ev1), (time.perf_counter() - e0) * 1e3)
     clocks = sampler.stop() if rank == 0 else None
     assert int(h_lengths.numpy().min()) == T
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    tokens_total = sum(s[1] for s in stats)
+    steps_total = sum(s[0] for s in stats)
+    job = replicas.reduce_totals(tokens_total, B, ms, ms_e2e, device="cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
-    tokens_total = sum(s[1] for s in stats)
-    steps_total = sum(s[0] for s in stats)
+    ms, ms_e2e = job.ms, job.ms_e2e
     scr = tokens_total / steps_total
-    value = world * tokens_total / B / (ms / 1e3)
+    value = job.tokens_per_s_per_mesh()
     e2e = world * n_e2e * T / (ms_e2e / 1e3)
     peaks, which = measured_peaks()
     # roofline of the persistent step kernel: algorithmic bytes of all its steps / time inside xsm_generate
@@ -265,6 +261,8 @@ def main():
     ap.add_argument("--k0", action="store_true", help="non-speculative path of the same library (n_draft = 0)")
     ap.add_argument("--tokens", type=int, default=0, help="override tokens per mesh")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--reference-seconds", type=float, default=0.0,
+                    help="--impl reference: CPU seconds per step (default: 120 s spread over the steps, 4 to 30 s each)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
