@@ -513,11 +513,10 @@ __device__ void stage_acts<float>(const Dev &D, const Smem &S, const GemvJob &J,
     // the next csync() of the caller orders ss before its readers
 }
 
-// bf16 models: packed hi + lo words in (gain already applied by the writer), {hi01, hi23, lo01, lo23} out; the
-// sum of squares of a normed input arrives as one partial per writer CTA.
+// bf16 models: packed hi + lo words in (gain already applied by the writer), {hi01, hi23, lo01, lo23} out.
 template <>
 __device__ void stage_acts<bf16>(const Dev &D, const Smem &S, const GemvJob &J, int ac0, int acw, uint32_t tag) {
-    const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int M = D.M, tid = threadIdx.x;
     const int v4_per_row = acw >> 2, total = M * v4_per_row;
     const int pitch = acw * 4 + 16;
     const float *x = J.x;
@@ -545,30 +544,34 @@ __device__ void stage_acts<bf16>(const Dev &D, const Smem &S, const GemvJob &J, 
             wr.next(v4_per_row);
         }
     }
-    if (J.gain != nullptr && ac0 == 0) {
-        // sum of squares of row m = sum over the writer CTAs' shares, one warp per row, fixed order
-        const int G = (int)gridDim.x;
-        for (int m = warp; m < M; m += kConsumerWarps) {
-            float s = 0.f;
-            if (!S.ctl->row_dead[m]) {
-                uint32_t v[8];            // G <= 256: at most 8 shares per lane, all requested at once
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const int c = lane + 32 * q;
-                    v[q] = c < G ? ld_relaxed_u32(D.sspub + (size_t)c * M + m) : tag;
-                }
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const int c = lane + 32 * q;
-                    if (c < G && (v[q] & 3u) != tag) v[q] = poll_u32(D, S.ctl, D.sspub + (size_t)c * M + m, tag);
-                    s += untag(v[q]);
-                }
-            }
-            s = warp_sum(s);
-            if (lane == 0) S.ss[m] = s;
-        }
-    }
     csync();
+}
+
+// bf16 models: the sum of squares of row m of a normed input = sum of the writer CTAs' shares, one warp per row,
+// fixed order; left in S.ss (the caller synchronises).  Only the epilogue needs it, so it is gathered after the
+// products, when the shares have long been published.
+static __device__ void gather_ss(const Dev &D, const Smem &S, uint32_t tag) {
+    const int M = D.M, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = (int)gridDim.x;
+    for (int m = warp; m < M; m += kConsumerWarps) {
+        float s = 0.f;
+        if (!S.ctl->row_dead[m]) {
+            uint32_t v[8];            // G <= 256: at most 8 shares per lane, all requested at once
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int c = lane + 32 * q;
+                v[q] = c < G ? ld_relaxed_u32(D.sspub + (size_t)c * M + m) : tag;
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int c = lane + 32 * q;
+                if (c < G && (v[q] & 3u) != tag) v[q] = poll_u32(D, S.ctl, D.sspub + (size_t)c * M + m, tag);
+                s += untag(v[q]);
+            }
+        }
+        s = warp_sum(s);
+        if (lane == 0) S.ss[m] = s;
+    }
 }
 
 // shared-memory address of layout row `row` of the tile whose first item sits at ring position pos_tile
@@ -733,6 +736,7 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
         if (lane == 0)
             for (int i = 0; i < tg * p.ipt; ++i) mbar_arrive(S.empty0 + 8u * ring_slot(S, pos0 + (uint32_t)i));
         ring.pos = pos0 + (uint32_t)(tg * p.ipt);
+        if (gain != nullptr && ss_raw) gather_ss(D, S, tag_in);
         // cross-warp reduction through the activation area, then the epilogue
         csync();
         // [warp][NP][16] partial products: behind the staged activations when both fit (then a following tile
