@@ -233,7 +233,7 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     const int K1 = c.n_draft + 1, M = batch * K1, dh = c.d_head;
     const int kmax = c.d_model > c.d_ff ? c.d_model : c.d_ff;
     const int tail = (kMaxTokens + 1536) * 4;                        // sums of squares and their partials
-    const int avail = kSmemMax - kSmemHeader - kSmemTables - tail;
+    const int avail = kSmemMax - kSmemHeader - kSmemTables - kSmemPlans - tail;
     // what the other users of the activation area need
     const int np = c.dtype == 1 ? (M <= 8 ? 8 : M <= 16 ? 16 : M <= 32 ? 32 : M <= 80 ? 80 : 128) : 8;
     int need = kConsumerWarps * np * 16 * 4 + 2 * 16 * M * 4;         // reduction of the projections, new residual values
@@ -259,7 +259,7 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     D.kca = kca;
     D.tile_bytes = c.page_size * dh * (c.dtype == 1 ? 2 : 4);
     D.kv_one_item = 2 * D.tile_bytes <= kSlotBytes ? 1 : 0;
-    smem_bytes = kSmemHeader + kSmemTables + slots * kSlotBytes + acts + tail;
+    smem_bytes = kSmemHeader + kSmemTables + kSmemPlans + slots * kSlotBytes + acts + tail;
     return nullptr;
 }
 
@@ -505,6 +505,7 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
     ctx->dc = *dc;
     ctx->batch = batch;
     D.B = batch; D.M = batch * D.K1;
+    D.inv_m = ((1 << 20) + D.M - 1) / D.M;
     D.verify_mode = dc->verify_mode; D.k_accept = dc->k_accept; D.delta = dc->delta;
     D.sample_mode = dc->sample_mode; D.k_sample = dc->k_sample; D.temperature = dc->temperature;
     D.key0 = (uint32_t)dc->seed; D.key1 = (uint32_t)(dc->seed >> 32);

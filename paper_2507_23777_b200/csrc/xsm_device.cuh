@@ -227,6 +227,7 @@ struct Smem {
     uint32_t full0, empty0, go_bar;   // shared-space addresses of full[0], empty[0], go
     Ctl *ctl;
     const Tables *tab;                // shared-memory copy of the stage and job tables
+    struct SegRec *seg;               // per job: this CTA's rows and their tiling
     char *ring;
     char *acts;
     float *ss;                        // [kMaxTokens] sum of squares / 1 / rms
@@ -242,7 +243,8 @@ __device__ __forceinline__ Smem carve(char *smem, const Dev &D) {
     s.go_bar = s.empty0 + 8u * kMaxSlots;
     s.ctl = reinterpret_cast<Ctl *>(smem + 256);   // 2 * 12 * 8 + 8 = 200 bytes of barriers before it
     s.tab = reinterpret_cast<const Tables *>(smem + kSmemHeader);
-    s.ring = smem + kSmemHeader + kSmemTables;
+    s.seg = reinterpret_cast<struct SegRec *>(smem + kSmemHeader + kSmemTables);
+    s.ring = smem + kSmemHeader + kSmemTables + kSmemPlans;
     s.n_slots = D.n_slots;
     s.acts = s.ring + (size_t)D.n_slots * kSlotBytes;
     s.ss = reinterpret_cast<float *>(s.acts + D.acts_bytes);
@@ -374,6 +376,8 @@ struct SegPlan {
     int tpg;          // tiles per group = min(consumer warps, slots / ipt), at least 1
     int row_bytes;
 };
+struct SegRec { int lo, hi; SegPlan p; };    // rows [lo, hi) of the job belong to this CTA
+static_assert(sizeof(SegRec) == kSegRecBytes, "size of a plan record");
 template <typename WT> __device__ __forceinline__ SegPlan seg_plan(const Smem &S, const GemvJob &J, int lo, int hi) {
     SegPlan p;
     p.row_bytes = J.kdim * (int)sizeof(WT);            // the host refuses rows beyond kItemBytes
@@ -405,8 +409,9 @@ __device__ __forceinline__ int item_rows(const GemvJob &J, const SegPlan &p, int
 // ---------------------------------------------------------------------------- projection: producer
 
 template <typename WT>
-static __device__ void produce_segment(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi) {
-    const SegPlan p = seg_plan<WT>(S, J, lo, hi);
+static __device__ void produce_segment(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R) {
+    const SegPlan p = R.p;
+    const int lo = R.lo, hi = R.hi;
     const int lane = threadIdx.x & 31;
     for (int tg0 = 0; tg0 < p.n_tiles; tg0 += p.tpg) {
         const int tg = min(p.tpg, p.n_tiles - tg0);
@@ -446,7 +451,10 @@ constexpr int kPollBatch = 8;   // tagged 16-byte loads a thread keeps in flight
 // walks the (row, 16-byte word) pairs of a staging pass without dividing: thread t starts at word t of row 0
 struct RowWalk {
     int m, c4;
-    __device__ __forceinline__ RowWalk(int tid, int v4_per_row) { m = tid / v4_per_row; c4 = tid - m * v4_per_row; }
+    __device__ __forceinline__ RowWalk(int tid, int v4_per_row) {
+        m = 0; c4 = tid;
+        while (c4 >= v4_per_row) { c4 -= v4_per_row; ++m; }      // v4_per_row >= 32: seven rounds at most
+    }
     __device__ __forceinline__ void next(int v4_per_row) {
         c4 += kConsumerThreads;
         while (c4 >= v4_per_row) { c4 -= v4_per_row; ++m; }
@@ -657,9 +665,10 @@ __device__ __forceinline__ float epilogue_store(const GemvJob &J, int m, int u, 
 }
 
 template <typename WT, int NT>
-static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi,
+static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R,
                                      uint32_t serial) {
-    const SegPlan p = seg_plan<WT>(S, J, lo, hi);
+    const SegPlan p = R.p;
+    const int lo = R.lo, hi = R.hi;
     const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int kca = min(J.kdim, D.kca);
     const bool one_chunk = kca >= J.kdim;
@@ -670,8 +679,11 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
     float ss_share = 0.f;
     for (int tg0 = 0; tg0 < p.n_tiles; tg0 += p.tpg) {
         const int tg = min(p.tpg, p.n_tiles - tg0);
-        const int parts = kConsumerWarps / tg;
-        const int my_tile = warp / parts, my_part = warp - my_tile * parts;   // my_tile >= tg: idle warp
+        // parts = 7 / tg and my_tile = warp / parts without dividing (tg in 1..7, warp in 0..6)
+        static_assert(kConsumerWarps == 7, "the two lookups below are for seven consumer warps");
+        const int parts = (0x11112370 >> (4 * tg)) & 15;
+        const int my_tile = (warp * (parts == 7 ? 5 : parts == 3 ? 11 : parts == 2 ? 16 : 32)) >> 5;
+        const int my_part = warp - my_tile * parts;                            // my_tile >= tg: idle warp
         const uint32_t pos0 = ring.pos;      // the group's items: tile tl at positions pos0 + tl * ipt ...
         bool landed = false;
         float acc[NT][2][4];
@@ -692,7 +704,7 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
             const int i = tid + q * kConsumerThreads;
             o_n[q] = 0; o_u[q] = -1; o_red[q] = 0; hpre[q] = 0.f; gpre[q] = 1.f;
             if (i < outs) {
-                const int ui = i & tu_mask, rest = i >> tu_shift, tl = rest / M, n = rest - tl * M;
+                const int ui = i & tu_mask, rest = i >> tu_shift, tl = (rest * D.inv_m) >> 20, n = rest - tl * M;
                 const int u = lo + (tg0 + tl) * p.tile_units + ui;
                 o_n[q] = n;
                 o_red[q] = tl * parts * NP * 16 + n * 16 + ui;
@@ -770,7 +782,7 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
                 u = q == 0 ? o_u[0] : q == 1 ? o_u[1] : q == 2 ? o_u[2] : o_u[3];
                 ro = q == 0 ? o_red[0] : q == 1 ? o_red[1] : q == 2 ? o_red[2] : o_red[3];
             } else {
-                const int ui = i & tu_mask, rest = i >> tu_shift, tl = rest / M;
+                const int ui = i & tu_mask, rest = i >> tu_shift, tl = (rest * D.inv_m) >> 20;
                 n = rest - tl * M;
                 u = lo + (tg0 + tl) * p.tile_units + ui;
                 ro = tl * parts * NP * 16 + n * 16 + ui;
@@ -815,10 +827,11 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
 // warp w owns pairs w, w + kConsumerWarps, ...; lanes stride over the columns; the activations of all tokens
 // must fit the staging area in one chunk.
 template <int MT>
-__device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi,
+__device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R,
                                     uint32_t serial) {
     constexpr int PPW = (8 + kConsumerWarps - 1) / kConsumerWarps;   // pairs per warp
-    const SegPlan p = seg_plan<float>(S, J, lo, hi);
+    const SegPlan p = R.p;
+    const int lo = R.lo, hi = R.hi;
     const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t tag_in = tag_of(serial, J.in), tag_out = tag_of(serial, J.outt);
     const float *gain = reinterpret_cast<const float *>(J.gain);
@@ -899,32 +912,53 @@ __device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, con
 // NTM: token tiles of 8 (bf16 weights) or token rows (fp32 weights) the kernel is compiled for
 template <typename WT, int NTM> struct ConsumeSegment;
 template <int NTM> struct ConsumeSegment<bf16, NTM> {
-    static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi, uint32_t serial) {
-        consume_segment_bf16<bf16, NTM>(D, S, ring, J, lo, hi, serial);
+    static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
+        consume_segment_bf16<bf16, NTM>(D, S, ring, J, R, serial);
     }
 };
 template <int NTM> struct ConsumeSegment<float, NTM> {
-    static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, int lo, int hi, uint32_t serial) {
-        consume_segment_f32<NTM>(D, S, ring, J, lo, hi, serial);
+    static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
+        consume_segment_f32<NTM>(D, S, ring, J, R, serial);
     }
 };
+
+// This CTA's share of every job, worked out once per launch: the rows of a stage's jobs form one range that is cut
+// evenly over the CTAs.  Thread i fills the record of job i.
+template <typename WT> static __device__ void plan_segments(const Dev &D, const Smem &S) {
+    const Tables &T = *S.tab;
+    const int n_jobs = kLayerJobs + T.n_tail_jobs, n_st = kLayerStages + T.n_tail_stages;
+    for (int i = threadIdx.x; i < n_jobs; i += blockDim.x) {
+        SegRec r;
+        r.lo = r.hi = 0;
+        r.p = seg_plan<WT>(S, T.jobs[i], 0, 0);
+        for (int s = 0; s < n_st; ++s) {
+            const Stage &st = T.stages[s];
+            if (st.kind != ST_GEMV || i < st.job0 || i >= st.job0 + st.njobs) continue;
+            unsigned total = 0;      // rows of all jobs of the stage (a few tens of thousands at most)
+            int base = 0;
+            for (int j = 0; j < st.njobs; ++j) {
+                if (st.job0 + j == i) base = (int)total;
+                total += (unsigned)T.jobs[st.job0 + j].rows;
+            }
+            const int u_lo = (int)(total * blockIdx.x / gridDim.x), u_hi = (int)(total * (blockIdx.x + 1) / gridDim.x);
+            r.lo = max(u_lo - base, 0);
+            r.hi = max(min(u_hi - base, T.jobs[i].rows), r.lo);
+            r.p = seg_plan<WT>(S, T.jobs[i], r.lo, r.hi);
+        }
+        S.seg[i] = r;
+    }
+}
 
 // A projection stage, seen by the producer warp (PRODUCER) or by the consumer warps.
 template <typename WT, int NTM, bool PRODUCER>
 static __device__ void gemv_stage(const Dev &D, const Smem &S, Ring &ring, const Stage &st, uint32_t serial) {
-    unsigned total = 0;      // rows of all jobs (a few tens of thousands at most)
-    for (int j = 0; j < st.njobs; ++j) total += (unsigned)S.tab->jobs[st.job0 + j].rows;
-    const int u_lo = (int)(total * blockIdx.x / gridDim.x), u_hi = (int)(total * (blockIdx.x + 1) / gridDim.x);
-    int base = 0;
     for (int j = 0; j < st.njobs; ++j) {
-        const int rows = S.tab->jobs[st.job0 + j].rows;
-        const int lo = max(u_lo - base, 0), hi = min(u_hi - base, rows);
-        if (lo < hi) {
+        const SegRec R = S.seg[st.job0 + j];
+        if (R.lo < R.hi) {
             const GemvJob J = job_at(D, S, st.job0 + j, st.layer);
-            if (PRODUCER) produce_segment<WT>(D, S, ring, J, lo, hi);
-            else ConsumeSegment<WT, NTM>::run(D, S, ring, J, lo, hi, serial);
+            if (PRODUCER) produce_segment<WT>(D, S, ring, J, R);
+            else ConsumeSegment<WT, NTM>::run(D, S, ring, J, R, serial);
         }
-        base += rows;
     }
 }
 
@@ -1790,6 +1824,8 @@ step_kernel(const __grid_constant__ Dev D, int st_lo, int st_hi, int n_steps, ui
         uint32_t *dst = reinterpret_cast<uint32_t *>(smem + kSmemHeader);
         for (int i = tid; i < (int)(sizeof(Tables) / 4); i += kThreads) dst[i] = __ldg(src + i);
     }
+    __syncthreads();
+    plan_segments<WT>(D, S);
     __syncthreads();
     uint32_t ring_pos = 0;
     const TagRef once = {1, 0};

@@ -69,6 +69,9 @@ struct Tables {
     int n_tail_stages, n_tail_jobs;
 };
 constexpr int kSmemTables = (sizeof(Tables) + 127) / 128 * 128;
+// behind the tables: one record per job with this CTA's share of its rows and how they are tiled (fixed for a launch)
+constexpr int kSegRecBytes = 40;
+constexpr int kSmemPlans = ((kLayerJobs + kMaxTailJobs) * kSegRecBytes + 127) / 128 * 128;
 
 // Everything a kernel needs; passed by value.
 struct Dev {
@@ -76,6 +79,7 @@ struct Dev {
     int L, d, H, dh, f, V, C, dc, K, K1, B, M, P;
     int max_blocks, n_pages, cpages, max_seq_len, tok_ld;
     int grid;                      // CTAs of the step kernel
+    int inv_m;                     // ceil(2^20 / M): x / M == (x * inv_m) >> 20 for x < 8192
     int S_max, S_cross;            // most key splits of a self-attention item; splits of a cross-attention item
     float eps, scale;
     int bos, eos;
