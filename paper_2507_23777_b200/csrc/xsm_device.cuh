@@ -218,6 +218,7 @@ struct Ctl {
     volatile int dead;          // a wait ran out somewhere: stop waiting on global memory
     int go;                     // written by the consumers before they release the producer for a step
     int trace_row;              // row of the timeline that the running stage fills when its inputs are in (0: off)
+    int any_dead;               // some sequence of the batch has finished: row_dead has entries set
     int len[kMaxBatch];
     int flags[kMaxBatch];       // 1 finished, 2 ingesting
     unsigned char row_dead[kMaxTokens];   // token rows of finished sequences (not fetched, read as zeros)
@@ -284,11 +285,20 @@ __device__ __forceinline__ uint32_t poll_u32(const Dev &D, Ctl *ctl, const void 
 
 // ------------------------------------------------------------------------------------------- ring
 
+// A ring position is the slot (low byte) and the parity of the number of trips round the ring (bit 8): items passed so
+// far, modulo twice the ring, kept in a form that needs no division.  Same sequence on the producer and on every
+// consumer warp.
 struct Ring {
-    uint32_t pos;   // items passed so far (same sequence on the producer and on every consumer warp)
+    uint32_t pos;
 };
-__device__ __forceinline__ uint32_t ring_slot(const Smem &S, uint32_t pos) { return pos % (uint32_t)S.n_slots; }
-__device__ __forceinline__ uint32_t ring_parity(const Smem &S, uint32_t pos) { return (pos / (uint32_t)S.n_slots) & 1u; }
+__device__ __forceinline__ uint32_t ring_slot(const Smem &S, uint32_t pos) { return pos & 0xFFu; }
+__device__ __forceinline__ uint32_t ring_parity(const Smem &S, uint32_t pos) { return (pos >> 8) & 1u; }
+// the position k items further (k is at most a few rings)
+__device__ __forceinline__ uint32_t ring_add(const Smem &S, uint32_t pos, int k) {
+    uint32_t slot = (pos & 0xFFu) + (uint32_t)k, par = pos >> 8;
+    while (slot >= (uint32_t)S.n_slots) { slot -= (uint32_t)S.n_slots; par ^= 1u; }
+    return slot | (par << 8);
+}
 
 __device__ __forceinline__ void mbar_wait(const Dev &D, Ctl *ctl, uint32_t bar, uint32_t parity) {
     for (unsigned it = 0; it < kMbarSpinLimit; ++it)
@@ -306,7 +316,7 @@ __device__ __forceinline__ char *ring_wait(const Dev &D, const Smem &S, const Ri
 __device__ __forceinline__ void ring_release(const Smem &S, Ring &r) {
     __syncwarp();
     if ((threadIdx.x & 31) == 0) mbar_arrive(S.empty0 + 8u * ring_slot(S, r.pos));
-    r.pos += 1;
+    r.pos = ring_add(S, r.pos, 1);
 }
 // producer (lane 0 decides, the warp follows): claim the next slot, announce `bytes`
 __device__ __forceinline__ void ring_claim(const Dev &D, const Smem &S, const Ring &r, uint32_t bytes, uint32_t &dst,
@@ -424,7 +434,7 @@ static __device__ void produce_segment(const Dev &D, const Smem &S, Ring &ring, 
                 uint32_t dst, bar;
                 ring_claim(D, S, ring, bytes, dst, bar);        // an item without valid rows is only announced
                 if (lane == 0 && bytes != 0u) bulk_g2s(dst, src, bytes, bar);
-                ring.pos += 1;
+                ring.pos = ring_add(S, ring.pos, 1);
             }
         }
     }
@@ -529,13 +539,14 @@ __device__ void stage_acts<bf16>(const Dev &D, const Smem &S, const GemvJob &J, 
     const int pitch = acw * 4 + 16;
     const float *x = J.x;
     const int kdim = J.kdim;
+    const bool dead_rows = S.ctl->any_dead != 0;
     RowWalk rd(tid, v4_per_row), wr(tid, v4_per_row);
     for (int i0 = 0; i0 < total; i0 += kConsumerThreads * kPollBatch) {
         uint4 w[kPollBatch];
 #pragma unroll
         for (int u = 0; u < kPollBatch; ++u) {
             w[u] = make_uint4(tag, tag, tag, tag);
-            if (rd.m < M && !S.ctl->row_dead[rd.m]) w[u] = ld_relaxed_u4(x + (size_t)rd.m * kdim + ac0 + (rd.c4 << 2));
+            if (rd.m < M && !(dead_rows && S.ctl->row_dead[rd.m])) w[u] = ld_relaxed_u4(x + (size_t)rd.m * kdim + ac0 + (rd.c4 << 2));
             rd.next(v4_per_row);
         }
 #pragma unroll
@@ -586,7 +597,7 @@ static __device__ void gather_ss(const Dev &D, const Smem &S, uint32_t tag) {
 __device__ __forceinline__ uint32_t tile_row_addr(const Smem &S, const SegPlan &p, uint32_t pos_tile, int row) {
     const int ns = S.n_slots;
     row = min(row, p.tile_rows - 1);     // rows past a short tile read its last row; their products are never used
-    int slot = (int)(pos_tile % (uint32_t)ns) + (row >> p.rpi_shift);
+    int slot = (int)ring_slot(S, pos_tile) + (row >> p.rpi_shift);
     if (slot >= ns) slot -= ns;
     return smem_u32(S.ring) + (uint32_t)slot * kSlotBytes + (uint32_t)((row & ((1 << p.rpi_shift) - 1)) * p.row_bytes);
 }
@@ -732,11 +743,11 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
             if (my_tile < tg) {
                 if (!landed) {
                     Ring r;
-                    for (int i = 0; i < p.ipt; ++i) { r.pos = pos0 + (uint32_t)(my_tile * p.ipt + i); ring_wait(D, S, r); }
+                    for (int i = 0; i < p.ipt; ++i) { r.pos = ring_add(S, pos0, my_tile * p.ipt + i); ring_wait(D, S, r); }
                     landed = true;
                 }
                 constexpr int U = NT == 1 ? 4 : (NT == 2 ? 2 : 1);
-                const uint32_t pos_tile = pos0 + (uint32_t)(my_tile * p.ipt);
+                const uint32_t pos_tile = ring_add(S, pos0, my_tile * p.ipt);
                 mma_tile_bf16<NT, U>(tile_row_addr(S, p, pos_tile, g), tile_row_addr(S, p, pos_tile, g + 8), S.acts, pitch, ac0,
                                      acw >> 5, my_part, parts, M, acc);
             }
@@ -746,8 +757,8 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
         // group's staging, so no arrival can fall into the wrong phase.
         __syncwarp();
         if (lane == 0)
-            for (int i = 0; i < tg * p.ipt; ++i) mbar_arrive(S.empty0 + 8u * ring_slot(S, pos0 + (uint32_t)i));
-        ring.pos = pos0 + (uint32_t)(tg * p.ipt);
+            for (int i = 0; i < tg * p.ipt; ++i) mbar_arrive(S.empty0 + 8u * ring_slot(S, ring_add(S, pos0, i)));
+        ring.pos = ring_add(S, pos0, tg * p.ipt);
         if (gain != nullptr && ss_raw) gather_ss(D, S, tag_in);
         // cross-warp reduction through the activation area, then the epilogue
         csync();
@@ -846,9 +857,9 @@ __device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, con
         const int tg = min(p.tpg, p.n_tiles - tg0);
         const uint32_t pos0 = ring.pos;
         for (int tl = 0; tl < tg; ++tl) {
-            const uint32_t pos_tile = pos0 + (uint32_t)(tl * p.ipt);
+            const uint32_t pos_tile = ring_add(S, pos0, tl * p.ipt);
             Ring r;
-            for (int i = 0; i < p.ipt; ++i) { r.pos = pos_tile + (uint32_t)i; ring_wait(D, S, r); }
+            for (int i = 0; i < p.ipt; ++i) { r.pos = ring_add(S, pos_tile, i); ring_wait(D, S, r); }
             float acc[PPW][2][MT];
 #pragma unroll
             for (int s2 = 0; s2 < PPW; ++s2)
@@ -904,8 +915,8 @@ __device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, con
         // every warp has read every item of the group
         __syncwarp();
         if (lane == 0)
-            for (int i = 0; i < tg * p.ipt; ++i) mbar_arrive(S.empty0 + 8u * ring_slot(S, pos0 + (uint32_t)i));
-        ring.pos = pos0 + (uint32_t)(tg * p.ipt);
+            for (int i = 0; i < tg * p.ipt; ++i) mbar_arrive(S.empty0 + 8u * ring_slot(S, ring_add(S, pos0, i)));
+        ring.pos = ring_add(S, pos0, tg * p.ipt);
     }
 }
 
@@ -1030,14 +1041,14 @@ static __device__ void produce_attn(const Dev &D, const Smem &S, Ring &ring, con
                 ring_claim(D, S, ring, 2u * (uint32_t)D.tile_bytes, dst, bar);
                 if (lane == 0) bulk_g2s(dst, kt, (uint32_t)D.tile_bytes, bar);
                 if (lane == 1) bulk_g2s(dst + (uint32_t)D.tile_bytes, vt, (uint32_t)D.tile_bytes, bar);
-                ring.pos += 1;
+                ring.pos = ring_add(S, ring.pos, 1);
             } else {
                 ring_claim(D, S, ring, (uint32_t)D.tile_bytes, dst, bar);
                 if (lane == 0) bulk_g2s(dst, kt, (uint32_t)D.tile_bytes, bar);
-                ring.pos += 1;
+                ring.pos = ring_add(S, ring.pos, 1);
                 ring_claim(D, S, ring, (uint32_t)D.tile_bytes, dst, bar);
                 if (lane == 0) bulk_g2s(dst, vt, (uint32_t)D.tile_bytes, bar);
-                ring.pos += 1;
+                ring.pos = ring_add(S, ring.pos, 1);
             }
         }
     }
@@ -1261,7 +1272,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
             const char *ks = ring_wait(D, S, ring);
             const char *vs = ks + D.tile_bytes;
             Ring r2 = ring;
-            if (!D.kv_one_item) { r2.pos += 1; vs = ring_wait(D, S, r2); }
+            if (!D.kv_one_item) { r2.pos = ring_add(S, r2.pos, 1); vs = ring_wait(D, S, r2); }
             const int nv_page = min(P, n - pg * P);
             for (int u = 0; u < upp; ++u, ++unit) {
                 const int nv = min(32, nv_page - u * 32);
@@ -1857,7 +1868,9 @@ step_kernel(const __grid_constant__ Dev D, int st_lo, int st_hi, int n_steps, ui
             __threadfence();   // what the publisher wrote before the header (pages, rope table, master h) is visible now
             csync();
             for (int m = tid; m < D.M; m += kConsumerThreads) S.ctl->row_dead[m] = (unsigned char)(S.ctl->flags[m / D.K1] & 1);
-            for (int b = 0; b < D.B; ++b) any |= !(S.ctl->flags[b] & 1);
+            int fin = 0;
+            for (int b = 0; b < D.B; ++b) { any |= !(S.ctl->flags[b] & 1); fin |= S.ctl->flags[b] & 1; }
+            if (tid == 0) S.ctl->any_dead = fin;
             if (S.ctl->dead) any = 0;
         }
         if (tid == 0) {
