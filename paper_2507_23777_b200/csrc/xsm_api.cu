@@ -237,7 +237,7 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     // what the other users of the activation area need
     const int np = c.dtype == 1 ? (M <= 8 ? 8 : M <= 16 ? 16 : M <= 32 ? 32 : M <= 80 ? 80 : 128) : 8;
     int need = kConsumerWarps * np * 16 * 4 + 2 * 16 * M * 4;         // reduction of the projections, new residual values
-    const int attn = 2 * 16 * (dh + 8) * 2 + 6 * K1 * dh * 4 + (kConsumerWarps + 1) * K1 * (dh + 2) * 4;
+    const int attn = 2 * 16 * (dh + 8) * 2 + 4 * K1 * dh * 4 + 128 * dh + (kConsumerWarps + 1) * K1 * (dh + 2) * 4;
     if (attn > need) need = attn;
     const int samp = (((c.vocab + 3) & ~3) + 256) * 4;
     if (samp > need) need = samp;

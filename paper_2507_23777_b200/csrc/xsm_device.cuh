@@ -1060,7 +1060,9 @@ static __device__ void produce_attn(const Dev &D, const Smem &S, Ring &ring, con
 template <int DH> struct AttnSmem {
     static constexpr int QP = DH + 8;                 // bf16 elements between query rows (16 bytes of padding)
     bf16 *qh, *ql;                                    // [16][QP] rotated, scaled queries as hi + lo (rows >= K1 zero)
-    float *qf, *kw, *vw;                              // [K1][DH] fp32: queries, window keys (rotated), window values
+    float *qf;                                        // [K1][DH] fp32 queries
+    float *kw, *vw;                                   // fp32 cache: [K1][DH] window keys (rotated), window values
+    __half *kt, *vt;                                  // 16-bit cache: the same as two cache tiles of 32 rows (same bytes as kw, vw)
     float *raw;                                       // [3][K1][DH] unrotated q, k, v; later the merged state
     float *st;                                        // [kConsumerWarps + 1][K1][DH + 2] per-warp softmax states
     __device__ AttnSmem(char *base, int K1) {
@@ -1069,7 +1071,9 @@ template <int DH> struct AttnSmem {
         qf = reinterpret_cast<float *>(ql + 16 * QP);
         kw = qf + K1 * DH;
         vw = kw + K1 * DH;
-        raw = vw + K1 * DH;
+        kt = reinterpret_cast<__half *>(kw);
+        vt = kt + 32 * DH;
+        raw = kw + 32 * DH;                           // 128 DH bytes hold either pair (K1 <= 16)
         st = raw + 3 * K1 * DH;
     }
 };
@@ -1081,11 +1085,13 @@ template <int DH> struct WarpState {
 };
 
 // 32 keys of one tile against the 16 query rows: S = Q K^T (hi + lo queries), online softmax, O += P V.
-template <int DH>
+// CAUSAL: the keys are those of the query rows themselves, row r sees keys 0..r.
+template <int DH, bool CAUSAL>
 __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t k_tile, uint32_t v_tile, int key0, int nvalid,
                                           WarpState<DH> &ws) {
     constexpr int QPB = (DH + 8) * 2, RB = DH * 2;
-    const int lane = threadIdx.x & 31, t = lane & 3;
+    constexpr int NK = CAUSAL ? 1 : 2;      // 16-key steps: the window has at most 16 rows
+    const int lane = threadIdx.x & 31, t = lane & 3, g = lane >> 2;
     float s[4][4];
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
@@ -1096,7 +1102,7 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
         ldmatrix_x4(qh, q_hi + qo);
         ldmatrix_x4(ql, q_lo + qo);
 #pragma unroll
-        for (int np = 0; np < 2; ++np) {      // key tiles 2np, 2np+1 (8 keys each)
+        for (int np = 0; np < NK; ++np) {      // key tiles 2np, 2np+1 (8 keys each)
             const int row = key0 + np * 16 + (lane & 7) + ((lane >> 4) << 3);
             const int chunk = 2 * ks + ((lane >> 3) & 1);
             unsigned kb[4];
@@ -1110,10 +1116,16 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
     // mask the keys past the end, row maxima over the 32 keys
     float mx0 = kNegBig, mx1 = kNegBig;
 #pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
+    for (int nt = 0; nt < 2 * NK; ++nt) {
         const int k0 = nt * 8 + 2 * t;
         if (k0 >= nvalid) { s[nt][0] = -INFINITY; s[nt][2] = -INFINITY; }
         if (k0 + 1 >= nvalid) { s[nt][1] = -INFINITY; s[nt][3] = -INFINITY; }
+        if (CAUSAL) {
+            if (k0 > g) s[nt][0] = -INFINITY;
+            if (k0 + 1 > g) s[nt][1] = -INFINITY;
+            if (k0 > g + 8) s[nt][2] = -INFINITY;
+            if (k0 + 1 > g + 8) s[nt][3] = -INFINITY;
+        }
         mx0 = fmaxf(mx0, fmaxf(s[nt][0], s[nt][1]));
         mx1 = fmaxf(mx1, fmaxf(s[nt][2], s[nt][3]));
     }
@@ -1125,7 +1137,7 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
     float l0 = 0.f, l1 = 0.f;
     unsigned ph[2][4], pl[2][4];   // P as A fragments of the two 16-key steps, hi and lo
 #pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
+    for (int nt = 0; nt < 2 * NK; ++nt) {
         const float p0 = exp2f(s[nt][0] - m0), p1 = exp2f(s[nt][1] - m0);
         const float p2 = exp2f(s[nt][2] - m1), p3 = exp2f(s[nt][3] - m1);
         l0 += p0 + p1; l1 += p2 + p3;
@@ -1140,7 +1152,7 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
 #pragma unroll
     for (int dn = 0; dn < DH / 8; ++dn) { ws.o[dn][0] *= c0; ws.o[dn][1] *= c0; ws.o[dn][2] *= c1; ws.o[dn][3] *= c1; }
 #pragma unroll
-    for (int kk = 0; kk < 2; ++kk) {
+    for (int kk = 0; kk < NK; ++kk) {
 #pragma unroll
         for (int dp = 0; dp < DH / 16; ++dp) {   // value columns 16dp .. 16dp+15 (chunks 2dp, 2dp+1)
             const int row = key0 + kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
@@ -1227,12 +1239,21 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
                 q = e < half ? q * cs.x - o * cs.y : o * cs.y + q * cs.x;
                 if (win) {
                     const float kr = A.raw[(K1 + j) * DH + e], ko = A.raw[(K1 + j) * DH + (e < half ? e + half : e - half)];
-                    A.kw[j * DH + e] = e < half ? kr * cs.x - ko * cs.y : ko * cs.y + kr * cs.x;
-                    A.vw[j * DH + e] = A.raw[(2 * K1 + j) * DH + e];
+                    const float kn = e < half ? kr * cs.x - ko * cs.y : ko * cs.y + kr * cs.x, vn = A.raw[(2 * K1 + j) * DH + e];
+                    if (MMA) {
+                        A.kt[tile_off<__half>(j, e, DH)] = from_f<__half>(kn);
+                        A.vt[tile_off<__half>(j, e, DH)] = from_f<__half>(vn);
+                    } else {
+                        A.kw[j * DH + e] = kn;
+                        A.vw[j * DH + e] = vn;
+                    }
                 }
             }
             q *= qscale;
             A.qf[j * DH + e] = q;
+        } else if (MMA && win) {
+            // value rows past the window are multiplied by zero weights: they must be finite
+            A.vt[tile_off<__half>(j, e, DH)] = from_f<__half>(0.f);
         }
         if (MMA) {
             unsigned hi, lo;
@@ -1250,11 +1271,16 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
             if (i >= 2 * K1 * (DH / 8)) break;
             const int kv = i / (K1 * (DH / 8)), rem = i - kv * K1 * (DH / 8), j = rem / (DH / 8), c = rem - j * (DH / 8);
             const int pos = n + j, page = page_pre[qq], r = pos % P;
-            const float *src = (kv ? A.vw : A.kw) + j * DH + c * 8;
             KVT *tile = kv_tile<KVT>(D, pool, pool_pages, st.layer, kv, page, h);
             KVT *dst = tile + tile_off<KVT>(r, c * 8, DH);
+            if constexpr (MMA) {
+                // the window tiles hold the rows in the cache's own format: chunk c of row j goes to chunk c of row r
+                *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>((kv ? A.vt : A.kt) + tile_off<__half>(j, c * 8, DH));
+            } else {
+                const float *src = (kv ? A.vw : A.kw) + j * DH + c * 8;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) dst[q] = from_f<KVT>(src[q]);
+                for (int q = 0; q < 8; ++q) dst[q] = from_f<KVT>(src[q]);
+            }
         }
     }
     // 4. the cached keys of this split
@@ -1277,11 +1303,14 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
             for (int u = 0; u < upp; ++u, ++unit) {
                 const int nv = min(32, nv_page - u * 32);
                 if (nv > 0 && (unit % kConsumerWarps) == warp)
-                    attn_unit<DH>(q_hi, q_lo, smem_u32(ks), smem_u32(vs), u * 32, nv, ws);
+                    attn_unit<DH, false>(q_hi, q_lo, smem_u32(ks), smem_u32(vs), u * 32, nv, ws);
             }
             ring_release(S, ring);
             if (!D.kv_one_item) ring_release(S, ring);
         }
+        // the window's own keys, under the causal mask, as one more unit
+        if (win && (unit % kConsumerWarps) == warp)
+            attn_unit<DH, true>(q_hi, q_lo, smem_u32(A.kt), smem_u32(A.vt), 0, K1, ws);
         // quad-reduce the denominators, park the state in shared memory
         const int g = lane >> 2, t = lane & 3;
         ws.l[0] += __shfl_xor_sync(0xffffffffu, ws.l[0], 1); ws.l[0] += __shfl_xor_sync(0xffffffffu, ws.l[0], 2);
@@ -1363,7 +1392,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
             float m = kNegBig, l = 0.f, acc[EPL];
 #pragma unroll
             for (int i = 0; i < EPL; ++i) acc[i] = 0.f;
-            if (win) {
+            if (win && !MMA) {
                 for (int wk = 0; wk <= j; ++wk) {
                     float dsum = 0.f;
 #pragma unroll
