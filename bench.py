@@ -133,6 +133,38 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def fitted_heads_arm(args, cfg, w, cond, T):
+    """The same mesh decoded twice more: by the library's K = 0 path, and by the K-head path with heads fitted to
+    the backbone (fit_heads: first training stage of Sec. 4.3 on sequences the backbone generated for other
+    meshes).  The configured heads are drawn independently of the backbone, so they show the cost of a step but
+    accept nothing; the paper's speedup is SCR / latency ratio with trained heads."""
+    from paper_2507_23777_b200 import binding, fit_heads
+    gdc = binding.decode_config(cfg)
+
+    def timed(c, ww):
+        ctx = binding.Context(c, ww, max_batch=1)
+        ctx.prefill(cond[:1], [c["bos_id"]], gdc)
+        ctx.generate(min(T, 256))                           # warm-up
+        ctx.prefill(cond[:1], [c["bos_id"]], gdc)
+        _, lens, st = ctx.generate(T)
+        assert int(lens[0]) == T
+        ctx.xsm_destroy()
+        return {"value": T / st.wall_ms * 1e3, "unit": UNIT, "scr": st.scr, "step_latency_us": st.wall_ms * 1e3 / st.steps,
+                "accept_hist": [int(x) for x in list(st.accept_hist)[:c["n_draft"] + 1]]}
+
+    cfg0 = dict(cfg, n_draft=0)
+    k0 = timed(cfg0, np.ascontiguousarray(w[:inputs.n_weight_elements(cfg0)]))
+    fitted, report = fit_heads.fit(cfg, w, n_meshes=args.fit_meshes, n_tokens=512)
+    report.pop("curve")
+    fh = timed(cfg, fitted)
+    fh["speedup_vs_k0"] = fh["value"] / k0["value"]
+    fh["fit"] = report
+    fh["note"] = ("heads = copies of the LM head fine-tuned on the frozen backbone's own sequences of other meshes "
+                  "(stage-1 loss, w(d) = 0.8^d, best held-out checkpoint); backbone and K = 0 path unchanged; the "
+                  "synthetic backbone's token dynamics are far more repetitive than a trained mesh model's")
+    return {"k0": k0, "fitted_heads": fh}
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -241,6 +273,8 @@ def run_gpu(args):
                      "avg_launch_ms": kernel_ms / n_step_launches},
         "clocks": clocks,
     }
+    if world == 1 and K >= 1 and not args.k0 and not args.no_fitted_heads:
+        line.update(fitted_heads_arm(args, cfg, w, cond, T))
     if not args.no_cpu_baseline and world == 1:
         v, steps, dt, cores = oracle_sample(cfg, w, cond, seconds_budget=15.0)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -261,6 +295,8 @@ def main():
     ap.add_argument("--k0", action="store_true", help="non-speculative path of the same library (n_draft = 0)")
     ap.add_argument("--tokens", type=int, default=0, help="override tokens per mesh")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-fitted-heads", action="store_true", help="skip the K = 0 and fitted-heads runs of the same mesh")
+    ap.add_argument("--fit-meshes", type=int, default=64, help="meshes of 512 tokens the heads are fitted on")
     ap.add_argument("--reference-seconds", type=float, default=0.0,
                     help="--impl reference: CPU seconds per step (default: 120 s spread over the steps, 4 to 30 s each)")
     args = ap.parse_args()
