@@ -24,7 +24,7 @@ thread_local std::string g_create_error;
 
 struct Layout {
     size_t total = 0;
-    size_t phases, jobs, inv_freq, wkc_off, wvc_off;
+    size_t phases, jobs, wkc_off, wvc_off;
     size_t len, window, cand, acc_len, finished, n_gen, n_blocks, ingest_left, step_idx, block_table, free_stack,
         scalars, hist, steps, tok_log, step_tokens, step_n_new, prompt;
     size_t h, rope_cs;
@@ -54,7 +54,6 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     size_t cur = 0;
     L.phases = take(cur, sizeof(Tables));
     L.jobs = take(cur, 256);
-    L.inv_freq = take(cur, sizeof(double) * (dh / 2 + 1));
     L.wkc_off = take(cur, sizeof(size_t) * c.n_layers);
     L.wvc_off = take(cur, sizeof(size_t) * c.n_layers);
     L.len = take(cur, 4 * B);
@@ -75,7 +74,7 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.step_n_new = take(cur, 4 * B);
     L.prompt = take(cur, 4 * B * (c.max_seq_len + 1));
     L.h = take(cur, 4 * M * d);
-    L.rope_cs = take(cur, 8 * M * (dh / 2));
+    L.rope_cs = take(cur, 8 * (size_t)(c.max_seq_len + K1 + 1) * (dh / 2));
     // tagged exchange buffers, cleared together at every xsm_prefill
     L.xchg_begin = cur;
     L.hpub = take(cur, 4 * M * d);
@@ -241,6 +240,8 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     if (attn > need) need = attn;
     const int samp = (((c.vocab + 3) & ~3) + 256) * 4;
     if (samp > need) need = samp;
+    const int emb = 512 + K1 * (c.d_model / (c.dtype == 1 ? 8 : 4)) * 4;   // commit: scalars, partial sums of the new window's rows
+    if (emb > need) need = emb;
     const int full = M * (kmax * 4 + 16) + (kConsumerWarps * np * 16 + kConsumerWarps * M) * 4;   // all activations of the widest projection, and the partial products behind them
     int acts = full > need ? full : need;
     if (acts > avail - kMinSlots * kSlotBytes) acts = avail - kMinSlots * kSlotBytes;
@@ -433,9 +434,17 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     if ((e = cudaEventCreate(&ctx->ev1)) != cudaSuccess) return bail(e, "cudaEventCreate");
 
     // constant tables
-    std::vector<double> inv_freq(cfg->d_head / 2 + 1);
-    for (int i = 0; i < cfg->d_head / 2; ++i) inv_freq[i] = pow((double)cfg->rope_theta, -2.0 * i / cfg->d_head);
-    if ((e = cudaMemcpyAsync(ctx->ws + L.inv_freq, inv_freq.data(), sizeof(double) * (cfg->d_head / 2),
+    // cos and sin of position * theta^(-2i/dh) for every position a window row can take
+    const int half = cfg->d_head / 2, n_pos = cfg->max_seq_len + cfg->n_draft + 2;
+    std::vector<float> rope((size_t)n_pos * half * 2);
+    for (int i = 0; i < half; ++i) {
+        const double inv_freq = pow((double)cfg->rope_theta, -2.0 * i / cfg->d_head);
+        for (int p = 0; p < n_pos; ++p) {
+            rope[((size_t)p * half + i) * 2] = (float)cos((double)p * inv_freq);
+            rope[((size_t)p * half + i) * 2 + 1] = (float)sin((double)p * inv_freq);
+        }
+    }
+    if ((e = cudaMemcpyAsync(ctx->ws + L.rope_cs, rope.data(), sizeof(float) * rope.size(),
                              cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) return bail(e, "upload");
     if ((e = cudaMemcpyAsync(ctx->ws + L.wkc_off, ctx->wo.wkc.data(), sizeof(size_t) * cfg->n_layers,
                              cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) return bail(e, "upload");
@@ -454,7 +463,7 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     D.eps = cfg->rms_eps; D.scale = (float)(1.0 / sqrt((double)cfg->d_head)); D.bos = cfg->bos_id; D.eos = cfg->eos_id;
     D.max_new = INT_MAX;
     D.tables = at<Tables>(ctx, L.phases);
-    D.E = wptr(ctx, ctx->wo.E); D.inv_freq = at<double>(ctx, L.inv_freq);
+    D.E = wptr(ctx, ctx->wo.E);
     D.len = at<int>(ctx, L.len); D.window = at<int>(ctx, L.window); D.cand = at<int>(ctx, L.cand);
     D.acc_len = at<int>(ctx, L.acc_len); D.finished = at<int>(ctx, L.finished); D.n_gen = at<int>(ctx, L.n_gen);
     D.n_blocks = at<int>(ctx, L.n_blocks); D.block_table = at<int>(ctx, L.block_table);

@@ -1201,7 +1201,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     for (int q = 0; q < kRot; ++q) {
         const int i = tid + q * kConsumerThreads, j = i / DH, e = i - j * DH;
         cs_pre[q] = make_float2(1.f, 0.f);
-        if (!cross && j < K1) cs_pre[q] = __ldcg(D.rope_cs + (size_t)(b * K1 + j) * half + (e % half));
+        if (!cross && j < K1) cs_pre[q] = __ldcg(D.rope_cs + (n + j) * half + (e % half));
     }
     int page_pre[2] = {0, 0};
     if (win) {
@@ -1648,8 +1648,9 @@ static __device__ __noinline__ void sample_stage(const Dev &D, uint32_t serial) 
 // gather the embeddings of the window into the residual stream (master copy and tagged copy for the step
 // `serial`), and tabulate cos/sin of the window rows' positions.  Threads 0..nthr-1 take part; `win` may point to
 // shared or global memory; nb_held = pages the sequence holds already.
-template <typename WT> __device__ void prepare_window(const Dev &D, int b, uint32_t serial, int len, int nb_held, const int *win, int nthr) {
-    const int K1 = D.K1, d = D.d, half = D.dh / 2;
+template <typename WT> __device__ void prepare_window(const Dev &D, int b, uint32_t serial, int len, int nb_held, const int *win, int nthr,
+                                                      float *scratch) {
+    const int K1 = D.K1, d = D.d;
     const TagRef hemb = {3 * D.L + 1, 0};
     const uint32_t tag = tag_of(serial, hemb);
     if (threadIdx.x == 0) {
@@ -1669,29 +1670,70 @@ template <typename WT> __device__ void prepare_window(const Dev &D, int b, uint3
     }
     const WT *E = reinterpret_cast<const WT *>(D.E);
     const WT *g0 = reinterpret_cast<const WT *>(D.gain_first);
-    // one warp per window row: embedding -> master copy and published copy (bf16 models: times the gain of the
-    // step's first RMSNorm, with the row's sum of squares as this writer's share and zero shares for the rest)
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = nthr >> 5;
-    for (int j = warp; j < K1; j += nwarps) {
-        const int tok = min(max(win[j], 0), D.V - 1), row = b * K1 + j;
-        float ssq = 0.f;
-        for (int e = lane; e < d; e += 32) {
-            const float v = to_f(E[(size_t)tok * d + e]);
-            __stcg(D.h + (size_t)row * d + e, v);
-            ssq = fmaf(v, v, ssq);
-            const float pub = sizeof(WT) == 2 ? v * to_f(g0[e]) : v;
-            st_relaxed_u32(D.hpub + (size_t)row * d + e, publish_word<WT>(pub, tag, false));
+    // Embedding -> master copy and published copy (bf16 models: times the gain of the step's first RMSNorm, with
+    // the row's sum of squares as this writer's share and zero shares for the rest).  A task is 16 bytes of one
+    // embedding row; every thread keeps two of them in flight (more would raise the
+    // register demand of the whole kernel).
+    constexpr int EPC = 16 / (int)sizeof(WT);       // elements per task
+    const int nch = d / EPC, total = K1 * nch;
+    for (int t0 = threadIdx.x; t0 < total; t0 += 2 * nthr) {
+        uint4 ev[2], gv[2];
+        int tj[2], tc[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int t = t0 + u * nthr;
+            tj[u] = -1; tc[u] = 0;
+            if (t < total) {
+                tj[u] = t / nch; tc[u] = t - tj[u] * nch;
+                const int tok = min(max(win[tj[u]], 0), D.V - 1);
+                ev[u] = __ldg(reinterpret_cast<const uint4 *>(E + (size_t)tok * d) + tc[u]);
+                if (sizeof(WT) == 2) gv[u] = __ldg(reinterpret_cast<const uint4 *>(g0) + tc[u]);
+            }
         }
-        if (sizeof(WT) == 2) {
-            ssq = warp_sum(ssq);
-            for (int c = lane; c < D.grid; c += 32) st_relaxed_u32(D.sspub + (size_t)c * D.M + row, tagged(c == 0 ? ssq : 0.f, tag));
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (tj[u] < 0) continue;
+            const int row = b * K1 + tj[u];
+            float v[EPC], gn[EPC];
+            if (sizeof(WT) == 2) {
+                const uint32_t ew[4] = {ev[u].x, ev[u].y, ev[u].z, ev[u].w}, gw[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    v[2 * q] = __uint_as_float(ew[q] << 16); v[2 * q + 1] = __uint_as_float(ew[q] & 0xFFFF0000u);
+                    gn[2 * q] = __uint_as_float(gw[q] << 16); gn[2 * q + 1] = __uint_as_float(gw[q] & 0xFFFF0000u);
+                }
+            } else {
+                v[0] = __uint_as_float(ev[u].x); v[1] = __uint_as_float(ev[u].y);
+                v[2] = __uint_as_float(ev[u].z); v[3] = __uint_as_float(ev[u].w);
+#pragma unroll
+                for (int q = 0; q < EPC; ++q) gn[q] = 1.f;
+            }
+            float ssq = 0.f;
+            float *hm = D.h + (size_t)row * d + tc[u] * EPC;
+            float *hp = D.hpub + (size_t)row * d + tc[u] * EPC;
+#pragma unroll
+            for (int q = 0; q < EPC; q += 4) {
+                __stcg(reinterpret_cast<float4 *>(hm + q), make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]));
+                uint4 pw;
+                pw.x = publish_word<WT>(v[q] * gn[q], tag, false); pw.y = publish_word<WT>(v[q + 1] * gn[q + 1], tag, false);
+                pw.z = publish_word<WT>(v[q + 2] * gn[q + 2], tag, false); pw.w = publish_word<WT>(v[q + 3] * gn[q + 3], tag, false);
+                __stcg(reinterpret_cast<uint4 *>(hp + q), pw);
+                ssq += v[q] * v[q] + v[q + 1] * v[q + 1] + v[q + 2] * v[q + 2] + v[q + 3] * v[q + 3];
+            }
+            if (sizeof(WT) == 2) scratch[tj[u] * nch + tc[u]] = ssq;
         }
     }
-    for (int i = threadIdx.x; i < K1 * half; i += nthr) {
-        const int j = i / half, f = i % half;
-        double sn, cs;
-        sincos((double)(len + j) * D.inv_freq[f], &sn, &cs);
-        __stcg(D.rope_cs + (size_t)(b * K1 + j) * half + f, make_float2((float)cs, (float)sn));
+    if (sizeof(WT) == 2) {
+        if (nthr == kConsumerThreads) csync(); else __syncthreads();
+        // the partial sums of a row are added in one fixed order
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = nthr >> 5;
+        for (int j = warp; j < K1; j += nwarps) {
+            float ssq = 0.f;
+            for (int c = lane; c < nch; c += 32) ssq += scratch[j * nch + c];
+            ssq = warp_sum(ssq);
+            const int row = b * K1 + j;
+            for (int c = lane; c < D.grid; c += 32) st_relaxed_u32(D.sspub + (size_t)c * D.M + row, tagged(c == 0 ? ssq : 0.f, tag));
+        }
     }
 }
 
@@ -1802,7 +1844,8 @@ template <typename WT> __device__ __noinline__ void commit_stage(const Dev &D, u
             sm[O_FLAGS] = flags;
         }
         csync();
-        if (!(sm[O_FLAGS] & 1)) prepare_window<WT>(D, b, serial + 1u, sm[O_LEN], s_state[4], s_win, kConsumerThreads);
+        if (!(sm[O_FLAGS] & 1))
+            prepare_window<WT>(D, b, serial + 1u, sm[O_LEN], s_state[4], s_win, kConsumerThreads, reinterpret_cast<float *>(sm + 128));
         __threadfence();
         csync();
         publish_header(D, b, serial + 1u, sm[O_LEN], sm[O_FLAGS]);

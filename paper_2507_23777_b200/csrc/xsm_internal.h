@@ -92,7 +92,6 @@ struct Dev {
     const Tables *tables;
     int n_stages;                  // 8 L + stages of the tail
     const void *E;                 // embedding table
-    const double *inv_freq;        // [dh/2] theta^(-2i/dh)
     // shared-memory plan of the step kernel
     int n_slots, acts_bytes, kca, tile_bytes, kv_one_item;
     // per-sequence state (plain words, read by other CTAs only after they have seen the step header)
@@ -112,7 +111,7 @@ struct Dev {
     unsigned long long *trace;     // null, or [1 + 2 * n_stages][grid] nanosecond timestamps of the launch's first step
     // untagged
     float *h;                      // master copy of the residual stream (each column range has one owner CTA)
-    float2 *rope_cs;               // [M][dh/2] cos, sin of the window rows' positions
+    float2 *rope_cs;               // [max_seq_len + K + 2][dh/2] cos, sin of position * theta^(-2i/dh)
     // caches
     void *kv_pool;                 // [L][2][n_pages][H] tiles of P x dh
     void *ckv_pool;                // [L][2][B*cpages][H] tiles of P x dh

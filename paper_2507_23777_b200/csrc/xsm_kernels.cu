@@ -81,6 +81,9 @@ cudaError_t launch_cross_kv(const Dev &D, int dtype, const void *W, const size_t
     return cudaGetLastError();
 }
 
+// shared memory of prepare_window's partial sums: one float per 16 bytes of the window's embedding rows
+static size_t window_scratch_bytes(const Dev &D, int elem_bytes) { return (size_t)D.K1 * (D.d / (16 / elem_bytes)) * sizeof(float); }
+
 // Algorithm 1 line 1: pool reset, then per-sequence state, first window and its pages.
 __global__ void init_pool_kernel(const Dev D) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -90,6 +93,7 @@ __global__ void init_pool_kernel(const Dev D) {
 
 template <typename WT> __global__ void __launch_bounds__(256) init_seq_kernel(const Dev D, uint32_t serial) {
     const int b = blockIdx.x, K1 = D.K1;
+    extern __shared__ float s_scratch[];      // K1 * d_model / (elements per 16 bytes) floats
     __shared__ int s_win[kMaxDraft + 1];
     if (threadIdx.x == 0) {
         D.len[b] = 0; D.finished[b] = 0; D.n_gen[b] = 0; D.n_blocks[b] = 0; D.step_idx[b] = 0u;
@@ -106,7 +110,7 @@ template <typename WT> __global__ void __launch_bounds__(256) init_seq_kernel(co
         for (int j = 0; j < K1; ++j) D.window[b * K1 + j] = s_win[j];
     }
     __syncthreads();
-    prepare_window<WT>(D, b, serial, 0, 0, s_win, 256);
+    prepare_window<WT>(D, b, serial, 0, 0, s_win, 256, s_scratch);
     __threadfence();
     __syncthreads();
     publish_header(D, b, serial, 0, D.prompt_len > 1 ? 2 : 0);
@@ -115,19 +119,20 @@ template <typename WT> __global__ void __launch_bounds__(256) init_seq_kernel(co
 cudaError_t launch_init(const Dev &D, int dtype, uint32_t serial, cudaStream_t st) {
     const int n = max(D.n_pages, 1);
     init_pool_kernel<<<(n + 255) / 256, 256, 0, st>>>(D);
-    if (dtype == 1) init_seq_kernel<bf16><<<D.B, 256, 0, st>>>(D, serial);
-    else init_seq_kernel<float><<<D.B, 256, 0, st>>>(D, serial);
+    if (dtype == 1) init_seq_kernel<bf16><<<D.B, 256, window_scratch_bytes(D, 2), st>>>(D, serial);
+    else init_seq_kernel<float><<<D.B, 256, window_scratch_bytes(D, 4), st>>>(D, serial);
     return cudaGetLastError();
 }
 
 // re-gather the window embeddings after the drafts were replaced from outside
 template <typename WT> __global__ void __launch_bounds__(256) embed_kernel(const Dev D, uint32_t serial) {
     const int b = blockIdx.x;
-    if (!D.finished[b]) prepare_window<WT>(D, b, serial, D.len[b], D.n_blocks[b], D.window + b * D.K1, 256);
+    extern __shared__ float s_scratch[];
+    if (!D.finished[b]) prepare_window<WT>(D, b, serial, D.len[b], D.n_blocks[b], D.window + b * D.K1, 256, s_scratch);
 }
 cudaError_t launch_embed(const Dev &D, int dtype, uint32_t serial, cudaStream_t st) {
-    if (dtype == 1) embed_kernel<bf16><<<D.B, 256, 0, st>>>(D, serial);
-    else embed_kernel<float><<<D.B, 256, 0, st>>>(D, serial);
+    if (dtype == 1) embed_kernel<bf16><<<D.B, 256, window_scratch_bytes(D, 2), st>>>(D, serial);
+    else embed_kernel<float><<<D.B, 256, window_scratch_bytes(D, 4), st>>>(D, serial);
     return cudaGetLastError();
 }
 
