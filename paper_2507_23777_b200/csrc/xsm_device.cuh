@@ -1574,20 +1574,27 @@ static __device__ int sample_token(const Dev &D, const float *z, uint32_t r24, f
     int *ci = reinterpret_cast<int *>(cv + 64);
     int *pick_s = ci + 64;
     const int k = D.sample_mode == 0 ? 1 : min(max(D.k_sample, 1), min(V, 64));
-    float pv = INFINITY;
-    int pi = -1;
-    for (int j = 0; j < k; ++j) {      // j-th candidate: best among those ranked after the previous one
-        float bv = -INFINITY;
-        int bi = 0x7fffffff;
-        for (int v = threadIdx.x; v < V; v += kConsumerThreads) {
-            const float zv = z[v];
-            if (j > 0 && !ranked_before(pv, pi, zv, v)) continue;
-            if (bi == 0x7fffffff || ranked_before(zv, v, bv, bi)) { bv = zv; bi = v; }
+    // every thread keeps the best of its own elements; after each pick only the thread that owned the winner
+    // looks for its next best (among its elements ranked after the winner)
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int v = threadIdx.x; v < V; v += kConsumerThreads) {
+        const float zv = z[v];
+        if (bi == 0x7fffffff || ranked_before(zv, v, bv, bi)) { bv = zv; bi = v; }
+    }
+    for (int j = 0; j < k; ++j) {
+        float wv = bv;
+        int wi = bi;
+        block_best(wv, wi, shv, shi);
+        if (threadIdx.x == 0) { cv[j] = wv; ci[j] = wi; }
+        if (wi == bi && j + 1 < k) {      // mine was picked
+            bv = -INFINITY; bi = 0x7fffffff;
+            for (int v = threadIdx.x; v < V; v += kConsumerThreads) {
+                const float zv = z[v];
+                if (!ranked_before(wv, wi, zv, v)) continue;
+                if (bi == 0x7fffffff || ranked_before(zv, v, bv, bi)) { bv = zv; bi = v; }
+            }
         }
-        block_best(bv, bi, shv, shi);
-        if (threadIdx.x == 0) { cv[j] = bv; ci[j] = bi; }
-        pv = bv; pi = bi;
-        csync();
     }
     if (threadIdx.x == 0) {
         int pick = ci[0];
@@ -1632,7 +1639,7 @@ static __device__ __noinline__ void sample_stage(const Dev &D, uint32_t serial) 
         }
         const float *z = slot == 0 ? D.logits0 + (size_t)(b * K1 + a) * V
                                    : D.hlogits + ((size_t)(slot - 1) * D.M + b * K1 + a) * V;
-        fetch_row(D, S, z, row, tag);
+        if (!(slot == 0 && a < K)) fetch_row(D, S, z, row, tag);      // slot 0: the row that rejected its draft is still staged
         const uint32_t r = rand24(D, b, __ldcg(D.step_idx + b), (uint32_t)slot, 0u);
         const int tok = sample_token(D, row, r, sh);
         if (threadIdx.x == 0) {
