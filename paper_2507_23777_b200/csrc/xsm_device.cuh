@@ -1476,11 +1476,6 @@ static __device__ void consume_attn(const Dev &D, const Smem &S, Ring &ring, con
 
 // ----------------------------------------------------------------- verify / accept length / resample
 
-// is (va, ia) ranked before (vb, ib): larger logit first, then smaller index
-__device__ __forceinline__ bool ranked_before(float va, int ia, float vb, int ib) {
-    return va > vb || (va == vb && ia < ib);
-}
-
 static __device__ float block_sum(float v, float *sh) {
     v = warp_sum(v);
     csync();
@@ -1500,20 +1495,33 @@ static __device__ float block_max(float v, float *sh) {
     for (int w = 0; w < kConsumerWarps; ++w) s = fmaxf(s, sh[w]);
     return s;
 }
-// best (value, index) over the block under ranked_before; threads without a candidate pass idx = INT_MAX
-static __device__ void block_best(float &v, int &idx, float *shv, int *shi) {
+// (logit, token) as one 64-bit key whose unsigned order is the ranking: larger logit first, then smaller token.
+// 0 is below every key ("no candidate").  -0.0 ranks with +0.0.
+__device__ __forceinline__ unsigned long long rank_key(float z, int idx) {
+    uint32_t u = __float_as_uint(z + 0.0f);
+    u ^= (u & 0x80000000u) ? 0xFFFFFFFFu : 0x80000000u;
+    return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)idx);
+}
+__device__ __forceinline__ float key_logit(unsigned long long k) {
+    uint32_t u = (uint32_t)(k >> 32);
+    u ^= (u & 0x80000000u) ? 0x80000000u : 0xFFFFFFFFu;
+    return __uint_as_float(u);
+}
+__device__ __forceinline__ int key_token(unsigned long long k) { return (int)(0xFFFFFFFFu - (uint32_t)k); }
+// largest key over the block; every thread gets it
+static __device__ unsigned long long block_best(unsigned long long k, unsigned long long *sh) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-        if (oi != 0x7fffffff && (idx == 0x7fffffff || ranked_before(ov, oi, v, idx))) { v = ov; idx = oi; }
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, k, o);
+        k = other > k ? other : k;
     }
     csync();
-    if ((threadIdx.x & 31) == 0) { shv[threadIdx.x >> 5] = v; shi[threadIdx.x >> 5] = idx; }
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = k;
     csync();
-    v = shv[0]; idx = shi[0];
-    for (int w = 1; w < kConsumerWarps; ++w)
-        if (shi[w] != 0x7fffffff && (idx == 0x7fffffff || ranked_before(shv[w], shi[w], v, idx))) { v = shv[w]; idx = shi[w]; }
+    k = sh[0];
+#pragma unroll
+    for (int w = 1; w < kConsumerWarps; ++w) k = sh[w] > k ? sh[w] : k;
+    return k;
 }
 
 // copies one tagged logits row into shared memory (waiting for it), tags stripped
@@ -1558,41 +1566,35 @@ static __device__ bool accept_token(const Dev &D, const float *z, int x, float *
         return expf(z[x] - m) / sum > D.delta;
     }
     const int ka = D.verify_mode == 0 ? 1 : D.k_accept;
-    const float zx = z[x];
+    const unsigned long long kx = rank_key(z[x], x);
     float cnt = 0.f;
-    for (int v = threadIdx.x; v < V; v += kConsumerThreads)
-        if (v != x && ranked_before(z[v], v, zx, x)) cnt += 1.f;
+    for (int v = threadIdx.x; v < V; v += kConsumerThreads) cnt += rank_key(z[v], v) > kx ? 1.f : 0.f;
     cnt = block_sum(cnt, sh);
     return (int)cnt < ka;
 }
 
 static __device__ int sample_token(const Dev &D, const float *z, uint32_t r24, float *sh) {
     const int V = D.V;
-    float *shv = sh;
-    int *shi = reinterpret_cast<int *>(sh + kConsumerWarps);
-    float *cv = sh + 2 * kConsumerWarps;               // candidates (value, index), up to 64
+    unsigned long long *shk = reinterpret_cast<unsigned long long *>(sh);   // [kConsumerWarps], 8-byte aligned
+    float *cv = sh + 2 * kConsumerWarps + 2;           // candidates (value, index), up to 64
     int *ci = reinterpret_cast<int *>(cv + 64);
     int *pick_s = ci + 64;
     const int k = D.sample_mode == 0 ? 1 : min(max(D.k_sample, 1), min(V, 64));
     // every thread keeps the best of its own elements; after each pick only the thread that owned the winner
     // looks for its next best (among its elements ranked after the winner)
-    float bv = -INFINITY;
-    int bi = 0x7fffffff;
+    unsigned long long mine = 0ull;
     for (int v = threadIdx.x; v < V; v += kConsumerThreads) {
-        const float zv = z[v];
-        if (bi == 0x7fffffff || ranked_before(zv, v, bv, bi)) { bv = zv; bi = v; }
+        const unsigned long long kv = rank_key(z[v], v);
+        mine = kv > mine ? kv : mine;
     }
     for (int j = 0; j < k; ++j) {
-        float wv = bv;
-        int wi = bi;
-        block_best(wv, wi, shv, shi);
-        if (threadIdx.x == 0) { cv[j] = wv; ci[j] = wi; }
-        if (wi == bi && j + 1 < k) {      // mine was picked
-            bv = -INFINITY; bi = 0x7fffffff;
+        const unsigned long long win = block_best(mine, shk);
+        if (threadIdx.x == 0) { cv[j] = key_logit(win); ci[j] = key_token(win); }
+        if (win == mine && j + 1 < k) {      // mine was picked
+            mine = 0ull;
             for (int v = threadIdx.x; v < V; v += kConsumerThreads) {
-                const float zv = z[v];
-                if (!ranked_before(wv, wi, zv, v)) continue;
-                if (bi == 0x7fffffff || ranked_before(zv, v, bv, bi)) { bv = zv; bi = v; }
+                const unsigned long long kv = rank_key(z[v], v);
+                if (kv < win && kv > mine) mine = kv;
             }
         }
     }
