@@ -24,6 +24,39 @@ def test_philox_known_answers(oracle_mod):
         assert oracle_mod.philox4x32_10(v[0:4], v[4:6]) == v[6:10]
 
 
+def test_philox_agrees_with_curand_host_generator(oracle_mod):
+    """cuRAND's Philox4_32_10 host generator, called as a library: with seed s and offset 0 it emits the four words
+    of counter (n, 0, t, 0), key (s_lo, s_hi), for t = 0 .. T-1 (one block per generator thread), then n + 1.  The
+    oracle's block function must give the same words (round function, key schedule, word order)."""
+    import ctypes as C
+    try:
+        lib = C.CDLL("libcurand.so")
+    except OSError:
+        try:
+            lib = C.CDLL("/usr/local/cuda/lib64/libcurand.so")
+        except OSError:
+            pytest.skip("libcurand not found")
+    PHILOX4_32_10 = 161
+    gen = C.c_void_p()
+    if lib.curandCreateGeneratorHost(C.byref(gen), PHILOX4_32_10) != 0:
+        pytest.skip("no cuRAND host generator")
+    seed = 0x0123_4567_89AB_CDEF
+    key = [seed & 0xFFFFFFFF, seed >> 32]
+    assert lib.curandSetPseudoRandomGeneratorSeed(gen, C.c_ulonglong(seed)) == 0
+    assert lib.curandSetGeneratorOffset(gen, C.c_ulonglong(0)) == 0
+    n = 4 * 70000
+    out = np.zeros(n, dtype=np.uint32)
+    assert lib.curandGenerate(gen, out.ctypes.data_as(C.c_void_p), C.c_size_t(n)) == 0
+    lib.curandDestroyGenerator(gen)
+    blocks = out.reshape(-1, 4)
+    for t in (0, 1, 2, 63, 1000):
+        assert list(blocks[t]) == oracle_mod.philox4x32_10([0, 0, t, 0], key), t
+    nxt = oracle_mod.philox4x32_10([1, 0, 0, 0], key)
+    T = next(i for i in range(1, len(blocks)) if list(blocks[i]) == nxt)       # generator threads
+    assert list(blocks[T + 5]) == oracle_mod.philox4x32_10([1, 0, 5, 0], key)
+    assert list(blocks[T - 1]) == oracle_mod.philox4x32_10([0, 0, T - 1, 0], key)
+
+
 def test_rand24_addressing(oracle_mod):
     """key = (seed_lo ^ seq_id, seed_hi), counter = (step, slot, purpose, 0), top 24 bits of word 0."""
     seed = 0x1234_5678_9ABC_DEF0
