@@ -250,6 +250,12 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     if (acts > avail - kMinSlots * kSlotBytes) acts -= 128;
     int kca = ((acts / M - 16) / 4) / 128 * 128;
     if (kca > kmax) kca = kmax;
+    if (kca < kmax && c.dtype == 1) {
+        // the widest projection is staged in chunks: room for the accumulators and the per-token partial sums behind
+        // a chunk, and chunks of at most 2048 columns (four rows of a chunk fit one ring slot)
+        kca = (((acts - kAccumBytes - kAccumBytes / 16) / M - 16) / 4) / 128 * 128;
+        if (kca > 2048) kca = 2048;
+    }
     if (kca < 128) return "batch * (n_draft + 1) is too large for the activation staging area";
     if (c.dtype == 0 && kca < kmax) return "fp32 models need all activations of a projection in shared memory: reduce the batch";
     if (c.dtype == 0 && M > 24) return "fp32 models support at most 24 token rows per step";

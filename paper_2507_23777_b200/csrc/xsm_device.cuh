@@ -440,6 +440,54 @@ static __device__ void produce_segment(const Dev &D, const Smem &S, Ring &ring, 
     }
 }
 
+// ---- projections whose activations do not fit the staging area at once (many token rows, or very long rows).
+// The activations are staged in chunks of D.kca columns, each chunk once per round of tiles, and the weights follow
+// the same order: an item holds the columns of one chunk for `rpi` rows of one tile (one bulk copy per row).  A
+// round is as many tiles as have their accumulators ([tile][token][16] floats) in kAccumBytes of shared memory.
+__device__ __forceinline__ int chunk_tiles_per_round(const SegPlan &p, int M) {
+    return max(1, min(p.n_tiles, kAccumBytes / (M * 64)));
+}
+// log2 of the rows of a tile that share one item when a row contributes seg_bytes (<= 4096) to it
+__device__ __forceinline__ int chunk_rpi_shift(const SegPlan &p, int seg_bytes) {
+    const int fit = min(kSlotBytes / seg_bytes, p.tile_rows);
+    return fit >= 16 ? 4 : fit >= 8 ? 3 : fit >= 4 ? 2 : fit >= 2 ? 1 : 0;
+}
+
+template <typename WT>
+static __device__ void produce_segment_chunked(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R) {
+    const SegPlan p = R.p;
+    const int lo = R.lo, hi = R.hi, lane = threadIdx.x & 31;
+    const int tr = chunk_tiles_per_round(p, D.M);
+    for (int r0 = 0; r0 < p.n_tiles; r0 += tr) {
+        const int nr = min(tr, p.n_tiles - r0);
+        for (int ac0 = 0; ac0 < J.kdim; ac0 += D.kca) {
+            const int acw = min(D.kca, J.kdim - ac0), seg = acw * (int)sizeof(WT);
+            const int sh = chunk_rpi_shift(p, seg), ipt = p.tile_rows >> sh;
+            for (int tl = 0; tl < nr; ++tl) {
+                const int u0 = lo + (r0 + tl) * p.tile_units, nu = min(p.tile_units, hi - u0);
+                for (int it = 0; it < ipt; ++it) {
+                    const int row = (it << sh) + lane;          // layout row of the tile that this lane copies
+                    bool valid = lane < (1 << sh);
+                    const WT *src;
+                    if (J.epi == EPI_GATEUP) {
+                        const int unit = row & 7;
+                        valid = valid && unit < nu;
+                        src = reinterpret_cast<const WT *>(row < 8 ? J.W : J.W2) + (size_t)(u0 + unit) * J.kdim + ac0;
+                    } else {
+                        valid = valid && row < nu;
+                        src = reinterpret_cast<const WT *>(J.W) + (size_t)(u0 + row) * J.kdim + ac0;
+                    }
+                    const uint32_t bytes = (uint32_t)(__popc(__ballot_sync(0xffffffffu, valid)) * seg);
+                    uint32_t dst, bar;
+                    ring_claim(D, S, ring, bytes, dst, bar);
+                    if (valid) bulk_g2s(dst + (uint32_t)(lane * seg), src, (uint32_t)seg, bar);
+                    ring.pos = ring_add(S, ring.pos, 1);
+                }
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------- projection: consumer
 
 // Stages columns [ac0, ac0+acw) of the tagged input of job J into shared memory: polls the words, strips the
@@ -834,6 +882,94 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
     }
 }
 
+// Consumer side of produce_segment_chunked.  Every warp waits for every item (so every warp frees every item it has
+// seen land); a warp multiplies the token tiles warp, warp + 7, ... of each tile and adds its products to the
+// accumulators in shared memory, which it alone touches for those tokens.
+template <typename WT>
+static __device__ void consume_segment_chunked(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R,
+                                               uint32_t serial) {
+    const SegPlan p = R.p;
+    const int lo = R.lo, hi = R.hi;
+    const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const uint32_t tag_in = tag_of(serial, J.in), tag_out = tag_of(serial, J.outt);
+    const WT *gain = reinterpret_cast<const WT *>(J.gain);
+    const int tr = chunk_tiles_per_round(p, M);
+    float *accum = reinterpret_cast<float *>(S.acts + (size_t)M * (D.kca * 4 + 16));   // [tile][token][16]
+    float *ssg = accum + kAccumBytes / 4;                                              // [tile][token]
+    const int tu_shift = p.tu_shift, tu_mask = p.tile_units - 1;
+    const bool want_ss = J.epi == EPI_ADD && J.gain_out != nullptr;
+    float ss_share = 0.f;
+    for (int r0 = 0; r0 < p.n_tiles; r0 += tr) {
+        const int nr = min(tr, p.n_tiles - r0);
+        csync();                               // the previous round's epilogue has read the accumulators
+        for (int i = tid; i < nr * M * 16; i += kConsumerThreads) accum[i] = 0.f;
+        for (int ac0 = 0; ac0 < J.kdim; ac0 += D.kca) {
+            const int acw = min(D.kca, J.kdim - ac0), seg = acw * (int)sizeof(WT), pitch = acw * 4 + 16;
+            const int sh = chunk_rpi_shift(p, seg), ipt = p.tile_rows >> sh;
+            csync();                           // everyone is done with the previous chunk
+            stage_acts<WT>(D, S, J, ac0, acw, tag_in);
+            if (ac0 == 0 && S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
+            for (int tl = 0; tl < nr; ++tl) {
+                const uint32_t pos_tile = ring.pos;
+                Ring r;
+                for (int i = 0; i < ipt; ++i) { r.pos = ring_add(S, pos_tile, i); ring_wait(D, S, r); }
+                // rows g and g + 8 of the tile (rows past a short tile read its last row; their products are not used)
+                const int ra = min(g, p.tile_rows - 1), rb = min(g + 8, p.tile_rows - 1);
+                const uint32_t base = smem_u32(S.ring);
+                const uint32_t row_a = base + ring_slot(S, ring_add(S, pos_tile, ra >> sh)) * kSlotBytes + (uint32_t)((ra & ((1 << sh) - 1)) * seg);
+                const uint32_t row_b = base + ring_slot(S, ring_add(S, pos_tile, rb >> sh)) * kSlotBytes + (uint32_t)((rb & ((1 << sh) - 1)) * seg);
+                for (int nt = warp; nt * 8 < M; nt += kConsumerWarps) {
+                    float acc[1][2][4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) acc[0][0][q] = acc[0][1][q] = 0.f;
+                    mma_tile_bf16<1, 4>(row_a, row_b, S.acts + (size_t)nt * 8 * pitch, pitch, 0, acw >> 5, 0, 1, M - nt * 8, acc);
+                    const int n0 = nt * 8 + 2 * t;
+                    float *a = accum + ((size_t)tl * M + n0) * 16;
+                    if (n0 < M) { a[g] += acc[0][0][0] + acc[0][1][0]; a[g + 8] += acc[0][0][2] + acc[0][1][2]; }
+                    if (n0 + 1 < M) { a[16 + g] += acc[0][0][1] + acc[0][1][1]; a[16 + g + 8] += acc[0][0][3] + acc[0][1][3]; }
+                }
+                __syncwarp();
+                if (lane == 0)
+                    for (int i = 0; i < ipt; ++i) mbar_arrive(S.empty0 + 8u * ring_slot(S, ring_add(S, pos_tile, i)));
+                ring.pos = ring_add(S, pos_tile, ipt);
+            }
+        }
+        if (gain != nullptr && r0 == 0) gather_ss(D, S, tag_in);
+        csync();
+        if (gain != nullptr && r0 == 0 && tid < M) S.ss[tid] = 1.0f / sqrtf(S.ss[tid] / (float)J.kdim + D.eps);
+        csync();
+        const int outs = nr * p.tile_units * M;
+        for (int i0 = 0; i0 < outs; i0 += kConsumerThreads) {
+            const int i = i0 + tid;
+            const int ui = i & tu_mask, rest = i >> tu_shift, tl = (rest * D.inv_m) >> 20, n = rest - tl * M;
+            const int u = lo + (r0 + tl) * p.tile_units + ui;
+            float r = 0.f;
+            if (i < outs && u < hi) {
+                const float *a = accum + ((size_t)tl * M + n) * 16;
+                float v = a[ui], v2 = J.epi == EPI_GATEUP ? a[ui + 8] : 0.f, inv = 1.f;
+                if (gain != nullptr) { inv = S.ss[n]; v *= inv; v2 *= inv; }
+                r = epilogue_store<WT>(J, n, u, v, v2, inv, tag_out);
+            }
+            if (want_ss) {
+                // the units of one (tile, token) sit in adjacent lanes: a fixed tree adds their squares
+                float sq = r * r;
+                sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+                sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+                if (p.tile_units >= 8) sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+                if (p.tile_units == 16) sq += __shfl_xor_sync(0xffffffffu, sq, 8);
+                if ((i & tu_mask) == 0 && i < outs) ssg[i >> tu_shift] = sq;
+            }
+        }
+        if (want_ss) {
+            csync();
+            if (tid < M) {
+                for (int tl = 0; tl < nr; ++tl) ss_share += ssg[tl * M + tid];
+                if (r0 + tr >= p.n_tiles) st_relaxed_u32(D.sspub + (size_t)blockIdx.x * M + tid, tagged(ss_share, tag_out));
+            }
+        }
+    }
+}
+
 // fp32 weights: the 16 rows of a tile form 8 pairs (q, q+8) (for gate/up: the gate and the up row of unit q);
 // warp w owns pairs w, w + kConsumerWarps, ...; lanes stride over the columns; the activations of all tokens
 // must fit the staging area in one chunk.
@@ -924,6 +1060,7 @@ __device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, con
 template <typename WT, int NTM> struct ConsumeSegment;
 template <int NTM> struct ConsumeSegment<bf16, NTM> {
     static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
+        if (D.kca < J.kdim) { consume_segment_chunked<bf16>(D, S, ring, J, R, serial); return; }
         consume_segment_bf16<bf16, NTM>(D, S, ring, J, R, serial);
     }
 };
@@ -967,7 +1104,10 @@ static __device__ void gemv_stage(const Dev &D, const Smem &S, Ring &ring, const
         const SegRec R = S.seg[st.job0 + j];
         if (R.lo < R.hi) {
             const GemvJob J = job_at(D, S, st.job0 + j, st.layer);
-            if (PRODUCER) produce_segment<WT>(D, S, ring, J, R);
+            if (PRODUCER) {
+                if (sizeof(WT) == 2 && D.kca < J.kdim) produce_segment_chunked<WT>(D, S, ring, J, R);
+                else produce_segment<WT>(D, S, ring, J, R);
+            }
             else ConsumeSegment<WT, NTM>::run(D, S, ring, J, R, serial);
         }
     }

@@ -19,6 +19,7 @@ constexpr int kMaxBatch = 128;
 constexpr int kSlotBytes = 16384;
 constexpr int kMaxSlots = 12;
 constexpr int kSmemHeader = 2048;                    // barriers and per-step scalars
+constexpr int kAccumBytes = 16384;                   // accumulators of the projections that stage their activations in chunks
 constexpr int kSmemMax = 227 * 1024;
 
 // One step of Algorithm 1 is a fixed list of stages.  A stage's output is published in global memory as
