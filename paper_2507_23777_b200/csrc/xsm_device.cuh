@@ -125,6 +125,17 @@ __device__ __forceinline__ void split_bf16(float x, unsigned &hi, unsigned &lo) 
     hi = __bfloat16_as_ushort(h);
     lo = __bfloat16_as_ushort(l);
 }
+// 2^x for the online softmax (x <= 0 or -inf): the hardware approximation, 2 ulp
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// two values rounded to fp16, first in the low half
+__device__ __forceinline__ unsigned pack_f16x2(float a, float b) {
+    const __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<const unsigned *>(&h);
+}
 // x = hi + lo with hi, lo fp16 (operands of the attention products)
 __device__ __forceinline__ void split_f16(float x, unsigned &hi, unsigned &lo) {
     const __half h = __float2half_rn(x);
@@ -1272,25 +1283,25 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
     mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
     mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
     const float m0 = fmaxf(ws.m[0], mx0), m1 = fmaxf(ws.m[1], mx1);
-    const float c0 = exp2f(ws.m[0] - m0), c1 = exp2f(ws.m[1] - m1);
+    const float c0 = ex2(ws.m[0] - m0), c1 = ex2(ws.m[1] - m1);
     ws.m[0] = m0; ws.m[1] = m1;
     float l0 = 0.f, l1 = 0.f;
-    unsigned ph[2][4], pl[2][4];   // P as A fragments of the two 16-key steps, hi and lo
+    unsigned ph[2][4];             // P as A fragments of the two 16-key steps (fp16: weights in [0, 1])
 #pragma unroll
     for (int nt = 0; nt < 2 * NK; ++nt) {
-        const float p0 = exp2f(s[nt][0] - m0), p1 = exp2f(s[nt][1] - m0);
-        const float p2 = exp2f(s[nt][2] - m1), p3 = exp2f(s[nt][3] - m1);
+        const float p0 = ex2(s[nt][0] - m0), p1 = ex2(s[nt][1] - m0);
+        const float p2 = ex2(s[nt][2] - m1), p3 = ex2(s[nt][3] - m1);
         l0 += p0 + p1; l1 += p2 + p3;
-        unsigned h0, h1, h2, h3, e0, e1, e2, e3;
-        split_f16(p0, h0, e0); split_f16(p1, h1, e1); split_f16(p2, h2, e2); split_f16(p3, h3, e3);
         const int kk = nt >> 1, hi2 = (nt & 1) * 2;     // a0,a1 from the even key tile, a2,a3 from the odd one
-        ph[kk][hi2] = h0 | (h1 << 16); ph[kk][hi2 + 1] = h2 | (h3 << 16);
-        pl[kk][hi2] = e0 | (e1 << 16); pl[kk][hi2 + 1] = e2 | (e3 << 16);
+        ph[kk][hi2] = pack_f16x2(p0, p1); ph[kk][hi2 + 1] = pack_f16x2(p2, p3);
     }
     ws.l[0] = ws.l[0] * c0 + l0;
     ws.l[1] = ws.l[1] * c1 + l1;
 #pragma unroll
-    for (int dn = 0; dn < DH / 8; ++dn) { ws.o[dn][0] *= c0; ws.o[dn][1] *= c0; ws.o[dn][2] *= c1; ws.o[dn][3] *= c1; }
+    if (__any_sync(0xffffffffu, c0 != 1.f || c1 != 1.f)) {     // a new maximum somewhere in the warp's rows
+#pragma unroll
+        for (int dn = 0; dn < DH / 8; ++dn) { ws.o[dn][0] *= c0; ws.o[dn][1] *= c0; ws.o[dn][2] *= c1; ws.o[dn][3] *= c1; }
+    }
 #pragma unroll
     for (int kk = 0; kk < NK; ++kk) {
 #pragma unroll
@@ -1300,9 +1311,7 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
             unsigned vb[4];
             ldmatrix_x4_trans(vb, v_tile + (uint32_t)row * RB + (uint32_t)swz(row, chunk, RB) * 16u);
             mma16816_f16(ws.o[2 * dp], ph[kk][0], ph[kk][1], ph[kk][2], ph[kk][3], vb[0], vb[1]);
-            mma16816_f16(ws.o[2 * dp], pl[kk][0], pl[kk][1], pl[kk][2], pl[kk][3], vb[0], vb[1]);
             mma16816_f16(ws.o[2 * dp + 1], ph[kk][0], ph[kk][1], ph[kk][2], ph[kk][3], vb[2], vb[3]);
-            mma16816_f16(ws.o[2 * dp + 1], pl[kk][0], pl[kk][1], pl[kk][2], pl[kk][3], vb[2], vb[3]);
         }
     }
 }
