@@ -230,6 +230,7 @@ struct Ctl {
     int go;                     // written by the consumers before they release the producer for a step
     int trace_row;              // row of the timeline that the running stage fills when its inputs are in (0: off)
     int any_dead;               // some sequence of the batch has finished: row_dead has entries set
+    volatile unsigned char landed[16];   // attention: parity of the latest fill of each ring slot that is known to have landed
     int len[kMaxBatch];
     int flags[kMaxBatch];       // 1 finished, 2 ingesting
     unsigned char row_dead[kMaxTokens];   // token rows of finished sequences (not fetched, read as zeros)
@@ -1342,6 +1343,11 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     int p_lo, p_hi;
     split_pages(n, P, it.s, it.S, p_lo, p_hi);
 
+    if (MMA && tid < S.n_slots) {
+        // the fill of slot `tid` that precedes this item's first position has landed (a barrier of the CTA lies between)
+        const uint32_t slot0 = ring_slot(S, ring.pos), par0 = ring_parity(S, ring.pos);
+        S.ctl->landed[tid] = (unsigned char)((uint32_t)tid < slot0 ? par0 : par0 ^ 1u);
+    }
     csync();
     // the rotation table and the pages of the appended rows are fetched while q is awaited
     constexpr int kRot = (16 * DH + kConsumerThreads - 1) / kConsumerThreads;
@@ -1442,23 +1448,52 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     if constexpr (MMA) {
         const uint32_t q_hi = smem_u32(A.qh), q_lo = smem_u32(A.ql);
         const int upp = P / 32;   // 32-key units per page
-        int unit = 0;
-        for (int pg = p_lo; pg < p_hi; ++pg) {
-            const char *ks = ring_wait(D, S, ring);
+        // Who touches a page.  Where a page is one ring item and the ring has a slot per consumer warp, page i of the
+        // item belongs to warp i mod 7 alone: it waits for the page, multiplies both units and frees the slot with
+        // seven arrivals of its own, and the other warps never look at that page (their per-page bookkeeping would
+        // cost more than the units).  A warp that skips pages skips phases of a slot's barrier, and a parity wait
+        // cannot tell "the fill before mine is still on its way" from "mine has landed".  So every owner records the
+        // parity of the fill it has seen land (ctl->landed), and an owner waits for its slot's previous fill to be
+        // recorded before it tests the barrier; with at least seven slots the fill before that one had completed when
+        // the owner's previous page landed, so one bit is enough.  Otherwise every warp passes every page and the
+        // 32-key units go round the warps.
+        const bool own = D.kv_one_item && S.n_slots >= kConsumerWarps;
+        const int n_it = D.kv_one_item ? 1 : 2, n_pages = p_hi - p_lo;
+        uint32_t pos = ring.pos;
+        for (int pg = p_lo; pg < p_hi; ++pg, pos = ring_add(S, pos, n_it)) {
+            const int rel = pg - p_lo;
+            if (own && (rel % kConsumerWarps) != warp) continue;
+            Ring r;
+            r.pos = pos;
+            if (own) {
+                if (lane == 0) {
+                    unsigned it2 = 0;
+                    while (S.ctl->landed[ring_slot(S, pos)] != (unsigned char)(ring_parity(S, pos) ^ 1u) && !S.ctl->dead)
+                        if (++it2 > kMbarSpinLimit) { raise_timeout(D, S.ctl); break; }
+                }
+                __syncwarp();
+            }
+            const char *ks = ring_wait(D, S, r);
+            if (own && lane == 0) S.ctl->landed[ring_slot(S, pos)] = (unsigned char)ring_parity(S, pos);
             const char *vs = ks + D.tile_bytes;
-            Ring r2 = ring;
-            if (!D.kv_one_item) { r2.pos = ring_add(S, r2.pos, 1); vs = ring_wait(D, S, r2); }
+            if (n_it == 2) { r.pos = ring_add(S, pos, 1); vs = ring_wait(D, S, r); }
             const int nv_page = min(P, n - pg * P);
-            for (int u = 0; u < upp; ++u, ++unit) {
+            for (int u = 0; u < upp; ++u) {
                 const int nv = min(32, nv_page - u * 32);
-                if (nv > 0 && (unit % kConsumerWarps) == warp)
+                if (nv > 0 && (own || ((rel * upp + u) % kConsumerWarps) == warp))
                     attn_unit<DH, false>(q_hi, q_lo, smem_u32(ks), smem_u32(vs), u * 32, nv, ws);
             }
-            ring_release(S, ring);
-            if (!D.kv_one_item) ring_release(S, ring);
+            __syncwarp();
+            if (own) {
+                if (lane < kConsumerWarps) mbar_arrive(S.empty0 + 8u * ring_slot(S, pos));
+            } else if (lane == 0) {
+                mbar_arrive(S.empty0 + 8u * ring_slot(S, pos));
+                if (n_it == 2) mbar_arrive(S.empty0 + 8u * ring_slot(S, r.pos));
+            }
         }
-        // the window's own keys, under the causal mask, as one more unit
-        if (win && (unit % kConsumerWarps) == warp)
+        ring.pos = pos;
+        // the window's own keys, under the causal mask, as one more unit for the warp whose turn is next
+        if (win && ((own ? n_pages : n_pages * upp) % kConsumerWarps) == warp)
             attn_unit<DH, true>(q_hi, q_lo, smem_u32(A.kt), smem_u32(A.vt), 0, K1, ws);
         // quad-reduce the denominators, park the state in shared memory
         const int g = lane >> 2, t = lane & 3;
