@@ -1626,18 +1626,41 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
         return;
     }
     if (it.S > 1) {
-        // wait for the other splits and fold them in (fixed order)
+        // wait for the other splits and fold them in (fixed order).  The maximum and one numerator (or the
+        // denominator) of up to eight splits are requested together, and the whole batch is requested again until
+        // every word carries the tag: the cost is the arrival of the slowest split plus one round trip.
         for (int i = tid; i < K1 * (DH + 1); i += kConsumerThreads) {
             const int j = i / (DH + 1), e = i - j * (DH + 1);
-            float m = mg[j * (DH + 2) + DH];
+            const int col = e < DH ? e : DH + 1;
             const float *pb = part + ((size_t)(b * D.H + h) * D.S_max) * K1 * (DH + 2) + (size_t)j * (DH + 2);
-            for (int ss = 0; ss < it.S - 1; ++ss)
-                m = fmaxf(m, untag(poll_u32(D, S.ctl, pb + (size_t)ss * K1 * (DH + 2) + DH, tag_part)));
-            float o = exp2f(mg[j * (DH + 2) + DH] - m) * mg[j * (DH + 2) + (e < DH ? e : DH + 1)];
-            for (int ss = 0; ss < it.S - 1; ++ss) {
-                const float *ps = pb + (size_t)ss * K1 * (DH + 2);
-                const float pm = untag(ld_relaxed_u32(ps + DH));
-                o += exp2f(pm - m) * untag(poll_u32(D, S.ctl, ps + (e < DH ? e : DH + 1), tag_part));
+            const size_t sstride = (size_t)K1 * (DH + 2);
+            const int nsp = it.S - 1;
+            float m = mg[j * (DH + 2) + DH], o = mg[j * (DH + 2) + col];      // running maximum, sum scaled to it
+            for (int s0 = 0; s0 < nsp; s0 += 8) {
+                uint32_t wm[8], wo[8];
+                for (unsigned tries = 0;; ++tries) {
+                    bool ok = true;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        wm[q] = wo[q] = tag_part;
+                        if (s0 + q < nsp) {
+                            wm[q] = ld_relaxed_u32(pb + (size_t)(s0 + q) * sstride + DH);
+                            wo[q] = ld_relaxed_u32(pb + (size_t)(s0 + q) * sstride + col);
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) ok = ok && (wm[q] & 3u) == tag_part && (wo[q] & 3u) == tag_part;
+                    if (ok || S.ctl->dead) break;
+                    if (tries > kSpinLimit) { raise_timeout(D, S.ctl); break; }
+                }
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (s0 + q < nsp) {
+                        const float pm = untag(wm[q]), mn = fmaxf(m, pm);
+                        o = o * exp2f(m - mn) + exp2f(pm - mn) * untag(wo[q]);
+                        m = mn;
+                    }
+                }
             }
             A.st[j * (DH + 2) + (e < DH ? e : DH + 1)] = o;   // st is free again: final numerators and denominator
         }
