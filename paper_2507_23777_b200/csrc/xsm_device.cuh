@@ -1184,8 +1184,11 @@ static __device__ void produce_attn(const Dev &D, const Smem &S, Ring &ring, con
     for (int idx = blockIdx.x; attn_item_at(D, S.ctl, cross, idx, it); idx += gridDim.x) {
         int p_lo, p_hi;
         split_pages(cross ? D.C : S.ctl->len[it.b], D.P, it.s, it.S, p_lo, p_hi);
+        int table = 0;      // block-table entries of 32 consecutive pages, one per lane: one round trip per 32 pages
         for (int pg = p_lo; pg < p_hi; ++pg) {
-            const int page = cross ? it.b * D.cpages + pg : __ldcg(D.block_table + (size_t)it.b * D.max_blocks + pg);
+            const int k32 = (pg - p_lo) & 31;
+            if (!cross && k32 == 0 && pg + lane < p_hi) table = __ldcg(D.block_table + (size_t)it.b * D.max_blocks + pg + lane);
+            const int page = cross ? it.b * D.cpages + pg : __shfl_sync(0xffffffffu, table, k32);
             const KVT *kt = kv_tile<KVT>(D, pool, pool_pages, st.layer, 0, page, it.h);
             const KVT *vt = kv_tile<KVT>(D, pool, pool_pages, st.layer, 1, page, it.h);
             uint32_t dst, bar;
