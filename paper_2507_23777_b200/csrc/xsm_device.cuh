@@ -6,7 +6,7 @@
 //  * Streaming.  Every byte that must come from HBM in a step (weight rows, cached keys and values, the
 //    condition's keys and values) has an address that is known when the step starts.  A producer warp walks
 //    the CTA's share of the step in order and pulls it into a ring of shared-memory slots with bulk copies
-//    (cp.async.bulk, completion on an mbarrier); eight consumer warps compute out of the ring.  HBM stays
+//    (cp.async.bulk, completion on an mbarrier); seven consumer warps compute out of the ring.  HBM stays
 //    busy while the consumers wait for activations of the previous stage.
 //  * Exchange.  Activations travel between CTAs as fp32 words in global memory whose two lowest mantissa
 //    bits carry a tag that cycles with the write index of the buffer.  A consumer spins on the words it
@@ -16,8 +16,8 @@
 //    each buffer is enough.
 //  * Arithmetic.  bf16 weights: mma.sync.m16n8k16 with weight rows on M and the token rows on N, the
 //    fp32 activations split into bf16 hi + lo so that nothing that matters is lost; fp32 accumulation.
-//    fp32 weights: FMA.  Attention over the bf16 cache: flash-decoding with mma.sync, queries and
-//    probabilities as hi + lo pairs, base-2 online softmax, splits over keys merged by the last split.
+//    fp32 weights: FMA.  Attention over the 16-bit cache (fp16 elements): flash-decoding with mma.sync,
+//    queries as fp16 hi + lo pairs, base-2 online softmax, splits over keys merged by the last split.
 //  * Every wait is bounded.  When one runs out the CTA raises the status word; every CTA that sees it stops
 //    waiting on global memory, still drains its ring, and leaves at the end of the step.
 #pragma once
