@@ -603,16 +603,28 @@ __device__ void stage_acts<bf16>(const Dev &D, const Smem &S, const GemvJob &J, 
     RowWalk rd(tid, v4_per_row), wr(tid, v4_per_row);
     for (int i0 = 0; i0 < total; i0 += kConsumerThreads * kPollBatch) {
         uint4 w[kPollBatch];
+        const float *src[kPollBatch];      // nullptr: nothing to fetch (past the end, or a finished sequence's row)
 #pragma unroll
         for (int u = 0; u < kPollBatch; ++u) {
-            w[u] = make_uint4(tag, tag, tag, tag);
-            if (rd.m < M && !(dead_rows && S.ctl->row_dead[rd.m])) w[u] = ld_relaxed_u4(x + (size_t)rd.m * kdim + ac0 + (rd.c4 << 2));
+            src[u] = (rd.m < M && !(dead_rows && S.ctl->row_dead[rd.m])) ? x + (size_t)rd.m * kdim + ac0 + (rd.c4 << 2) : nullptr;
             rd.next(v4_per_row);
+        }
+        // The whole batch is requested at once.  Where a word has not arrived, the thread waits for the first such
+        // word alone (one spin loop in the code, one word of polling traffic) and then requests the batch again.
+        for (;;) {
+            const float *stale = nullptr;
+#pragma unroll
+            for (int u = 0; u < kPollBatch; ++u) w[u] = src[u] != nullptr ? ld_relaxed_u4(src[u]) : make_uint4(tag, tag, tag, tag);
+#pragma unroll
+            for (int u = kPollBatch - 1; u >= 0; --u)
+                if (!tags_ok(w[u], tag)) stale = src[u];
+            if (stale == nullptr) break;
+            poll_u4(D, S.ctl, stale, tag);
+            if (S.ctl->dead) break;
         }
 #pragma unroll
         for (int u = 0; u < kPollBatch; ++u) {
             if (wr.m < M) {
-                if (!tags_ok(w[u], tag)) w[u] = poll_u4(D, S.ctl, x + (size_t)wr.m * kdim + ac0 + (wr.c4 << 2), tag);
                 uint4 o;
                 o.x = __byte_perm(w[u].x, w[u].y, 0x7632);
                 o.y = __byte_perm(w[u].z, w[u].w, 0x7632);
@@ -741,8 +753,8 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
     const SegPlan p = R.p;
     const int lo = R.lo, hi = R.hi;
     const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const int kca = min(J.kdim, D.kca);
-    const bool one_chunk = kca >= J.kdim;
+    const int kca = J.kdim;               // the whole input fits the staging area (else: consume_segment_chunked)
+    constexpr bool one_chunk = true;
     const uint32_t tag_in = tag_of(serial, J.in), tag_out = tag_of(serial, J.outt);
     const WT *gain = reinterpret_cast<const WT *>(J.gain);
     constexpr int NP = NT * 8;
