@@ -647,18 +647,24 @@ static __device__ void gather_ss(const Dev &D, const Smem &S, uint32_t tag) {
     for (int m = warp; m < M; m += kConsumerWarps) {
         float s = 0.f;
         if (!S.ctl->row_dead[m]) {
-            uint32_t v[8];            // G <= 256: at most 8 shares per lane, all requested at once
+            uint32_t v[8];            // G <= 256: at most 8 shares per lane, all requested at once, and again
+                                      // after a wait for the first one that was missing
+            for (;;) {
+                const float *stale = nullptr;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const int c = lane + 32 * q;
-                v[q] = c < G ? ld_relaxed_u32(D.sspub + (size_t)c * M + m) : tag;
+                for (int q = 0; q < 8; ++q) {
+                    const int c = lane + 32 * q;
+                    v[q] = c < G ? ld_relaxed_u32(D.sspub + (size_t)c * M + m) : tag;
+                }
+#pragma unroll
+                for (int q = 7; q >= 0; --q)
+                    if ((v[q] & 3u) != tag) stale = D.sspub + (size_t)(lane + 32 * q) * M + m;
+                if (stale == nullptr) break;
+                poll_u32(D, S.ctl, stale, tag);
+                if (S.ctl->dead) break;
             }
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const int c = lane + 32 * q;
-                if (c < G && (v[q] & 3u) != tag) v[q] = poll_u32(D, S.ctl, D.sspub + (size_t)c * M + m, tag);
-                s += untag(v[q]);
-            }
+            for (int q = 0; q < 8; ++q) s += untag(v[q]);
         }
         s = warp_sum(s);
         if (lane == 0) S.ss[m] = s;
@@ -1754,18 +1760,25 @@ static __device__ void fetch_row(const Dev &D, const Smem &S, const float *z, fl
         const int n4 = V >> 2;
         for (int i0 = 0; i0 < n4; i0 += kConsumerThreads * kPollBatch) {
             uint4 w[kPollBatch];
+            for (;;) {       // the batch at once; after a wait for the first missing word, the batch again
+                const float *stale = nullptr;
 #pragma unroll
-            for (int u = 0; u < kPollBatch; ++u) {
-                const int i = i0 + u * kConsumerThreads + threadIdx.x;
-                if (i < n4) w[u] = ld_relaxed_u4(z + 4 * i);
+                for (int u = 0; u < kPollBatch; ++u) {
+                    const int i = i0 + u * kConsumerThreads + threadIdx.x;
+                    w[u] = i < n4 ? ld_relaxed_u4(z + 4 * i) : make_uint4(tag, tag, tag, tag);
+                }
+#pragma unroll
+                for (int u = kPollBatch - 1; u >= 0; --u)
+                    if (!tags_ok(w[u], tag)) stale = z + 4 * (i0 + u * kConsumerThreads + threadIdx.x);
+                if (stale == nullptr) break;
+                poll_u4(D, S.ctl, stale, tag);
+                if (S.ctl->dead) break;
             }
 #pragma unroll
             for (int u = 0; u < kPollBatch; ++u) {
                 const int i = i0 + u * kConsumerThreads + threadIdx.x;
-                if (i < n4) {
-                    if (!tags_ok(w[u], tag)) w[u] = poll_u4(D, S.ctl, z + 4 * i, tag);
+                if (i < n4)
                     *reinterpret_cast<float4 *>(row + 4 * i) = make_float4(untag(w[u].x), untag(w[u].y), untag(w[u].z), untag(w[u].w));
-                }
             }
         }
     } else {
