@@ -516,7 +516,7 @@ template <> __device__ __forceinline__ float4 load_gain4<bf16>(const bf16 *gain,
                        __uint_as_float(u.y & 0xffff0000u));
 }
 
-constexpr int kPollBatch = 8;   // tagged 16-byte loads a thread keeps in flight
+constexpr int kPollBatch = 6;   // tagged 16-byte loads a thread keeps in flight (20 KB of activations over 224 threads: one batch)
 
 // walks the (row, 16-byte word) pairs of a staging pass without dividing: thread t starts at word t of row 0
 struct RowWalk {

@@ -26,8 +26,8 @@ def speedup(scr: float, latency_base: float, latency_spec: float) -> float:
 # decoding steps at contexts 0..63, see profiles/), as a ratio to the algorithmic bytes of the same launch.  Traffic
 # grows in proportion to the units processed (weights once per step plus the cache), so a launch of the benchmark is
 # its algorithmic bytes times this ratio.  None: no capture of the current kernel for that configuration.
-_TRAFFIC_RATIO = {1: (19.541292e9 + 46.927360e6) / 19304546304.0,
-                  2: (63.645289e9 + 76.575488e6) / 63021514752.0}
+_TRAFFIC_RATIO = {1: (19.538215e9 + 46.177536e6) / 19304546304.0,
+                  2: (63.644030e9 + 77.415936e6) / 63021514752.0}
 
 
 def measured_traffic(config_index: int, algorithmic_bytes_per_launch: float):
