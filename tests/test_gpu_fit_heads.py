@@ -28,3 +28,55 @@ def test_fitted_heads_are_accepted_far_more_often_than_the_configured_ones():
         ctx.xsm_destroy()
     assert scr["configured"] < 1.1           # independent heads: about k / V of the drafts pass
     assert scr["fitted"] > 1.5, scr
+
+
+def _first_difference_is_a_near_tie(cfg0, w0, ref, got, margin=1e-3):
+    """ref: tokens of the plain one-token-per-step path; got: tokens of a speculative run of the same model.  Equal,
+    or the first differing token sits where the plain path's two best logits are closer than `margin` (after it the
+    two runs decode different sequences and cannot be compared)."""
+    from paper_2507_23777_b200 import binding
+    if np.array_equal(ref, got):
+        return True, -1, 0.0
+    i = int(np.argmax(ref != got))
+    ctx = binding.Context(cfg0, w0, max_batch=1)
+    ctx.prefill(inputs.make_cond(cfg0, 1), [cfg0["bos_id"]], binding.decode_config(cfg0))
+    for _ in range(i + 1):
+        ctx.step()
+    z0, _ = ctx.xsm_debug_get_logits()
+    ctx.xsm_destroy()
+    z = np.sort(z0[0, 0])[::-1]
+    return float(z[0] - z[1]) < margin, i, float(z[0] - z[1])
+
+
+def test_configuration_1_in_full_decodes_what_plain_greedy_decoding_decodes():
+    """Greedy verification leaves the output unchanged (Sec. 4.2: a draft is accepted only where the backbone agrees):
+    the 4096 tokens of configuration 1 from the K-head path, through xsm_generate as the benchmark launches it, against
+    the library's own K = 0 path; once with the configured heads and once with fitted heads, whose drafts are
+    accepted now and then (commit of several tokens, rollback of the rest, at contexts up to 4096)."""
+    import torch
+    assert torch.cuda.is_available(), "this test needs a B200"
+    from paper_2507_23777_b200 import binding, build, fit_heads
+    build.build()
+    cfg = inputs.config(1)
+    cfg0 = dict(cfg, n_draft=0)
+    w = inputs.make_weights(cfg)
+    w0 = np.ascontiguousarray(w[:inputs.n_weight_elements(cfg0)])
+    T = cfg["gen_tokens"]
+
+    def run(c, ww):
+        ctx = binding.Context(c, ww, max_batch=1)
+        ctx.prefill(inputs.make_cond(c, 1), [c["bos_id"]], binding.decode_config(c))
+        toks, lens, st = ctx.generate(T)
+        ctx.xsm_destroy()
+        assert int(lens[0]) == T
+        return toks[0], st
+
+    ref, _ = run(cfg0, w0)
+    got, st = run(cfg, w)
+    ok, i, m = _first_difference_is_a_near_tie(cfg0, w0, ref, got)
+    assert ok, f"configured heads: token {i} differs with a top-2 margin of {m}"
+    fitted, _ = fit_heads.fit(cfg, w, n_meshes=24, n_tokens=512, iters=100, eval_every=25)
+    got, st = run(cfg, fitted)
+    assert st.scr > 1.0 and sum(st.accept_hist[1:]) > 0
+    ok, i, m = _first_difference_is_a_near_tie(cfg0, w0, ref, got)
+    assert ok, f"fitted heads: token {i} differs with a top-2 margin of {m}"
