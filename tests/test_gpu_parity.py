@@ -185,9 +185,9 @@ def test_long_context_split_attention(P, shape):
     ls.close()
 
 
-def _shape(d, H, dh, f, K, L=2, V=1500, C=40, **kw):
+def _shape(d, H, dh, f, K, L=2, V=1500, C=40, max_seq_len=256, **kw):
     return dict(d_model=d, n_heads=H, d_head=dh, d_ff=f, d_cond=d, head_hidden=d, n_draft=K, n_layers=L, vocab=V,
-                n_cond=C, max_seq_len=256, **kw)
+                n_cond=C, max_seq_len=max_seq_len, **kw)
 
 
 SHAPES = {
@@ -201,6 +201,8 @@ SHAPES = {
     "rows of 1280 and 3840 bytes": (_shape(640, 10, 64, 1920, 3), 1),
     "no heads, five sequences": (_shape(768, 12, 64, 3072, 0), 5),
     "several tile groups per projection": (_shape(2048, 16, 128, 2048, 3, V=3000), 2),
+    "two attention items per CTA, pages owned by warps": (_shape(1024, 16, 64, 4096, 0), 16),
+    "two attention items per CTA, three token rows each": (_shape(512, 8, 64, 2048, 2, V=900), 24),
 }
 
 
@@ -214,6 +216,22 @@ def test_shape_sweep_bf16(P, shape):
     for _ in range(3):
         ls.step(**BF16_TOL)
     ls.compare_cache(**BF16_TOL)
+    ls.close()
+
+
+def test_long_prompt_many_pages_per_attention_split(P):
+    """64 heads leave two key splits per head, so at a context of 1100 tokens a split walks nine cache pages and a warp
+    owns more than one of them.  The prompt is ingested through the same step kernel; then logits, decisions and the
+    whole cache of the last layer are compared with the oracle."""
+    cfg = inputs.config(2, **_shape(2048, 64, 32, 2048, 4, max_seq_len=1400))
+    cfg["max_seq_len"] = 1400
+    ls = P.LockStep(cfg, batch=1)
+    prompt = [0] + [int(t) for t in np.random.default_rng(5).integers(1, cfg["vocab"], 1100)]
+    st = ls.begin(prompt)
+    assert st["len"][0] == len(prompt) - 1
+    for _ in range(8):
+        ls.step(**BF16_TOL)
+    ls.compare_cache(layers=[1], **BF16_TOL)
     ls.close()
 
 
