@@ -91,19 +91,24 @@ typedef struct {
     double scr;                             /* tokens / steps (Sec. 5.1) */
 } xsm_stats;
 
-/* Bytes of the flat weight buffer for this shape. */
+/* Bytes of the flat weight buffer for this shape: the backbone of Sec. 4.1 with its decoder W0 (Eq. 2) and the
+ * K decoding heads, in the layout given above. */
 XSM_API size_t xsm_weights_bytes(const xsm_model_config *cfg);
 
 /* Bytes of workspace that hold max_batch sequences of max_seq_len positions
  * (page pool, cross-attention cache, activations, decoding state). */
 XSM_API size_t xsm_workspace_bytes(const xsm_model_config *cfg);
 
-/* Binds a context to DEVICE weights and DEVICE workspace (both 256-byte
+/* Algorithm 1's inputs other than the condition: the backbone M and the decoding
+ * heads {H_i}, as one weight buffer in the layout above.
+ * Binds a context to DEVICE weights and DEVICE workspace (both 256-byte
  * aligned, borrowed until xsm_destroy) and a CUDA stream (cudaStream_t passed
  * as void*, may be NULL for the default stream).  A workspace larger than
  * xsm_workspace_bytes adds pages to the shared pool; a smaller one that still
  * holds at least one sequence's pages is accepted and XSM_ERR_CAPACITY is then
- * decided per xsm_prefill. */
+ * decided per xsm_prefill.  bf16 models keep cached keys and values as fp16:
+ * a key or value element beyond +-65504 is stored as +-65504 without any status
+ * (projections of normalised activations by N(0, 0.02) weights stay far below). */
 XSM_API xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *d_workspace,
                       size_t workspace_bytes, void *cuda_stream, xsm_ctx **out);
 
@@ -112,7 +117,9 @@ XSM_API xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights
  * dtype), runs prompt tokens 0..prompt_len-2 into the cache, sets x_s to the
  * last prompt token, s = prompt_len-1, draws the K initial drafts uniformly on
  * [0, V) and resets the step counters.  d_prompt: DEVICE int32 [batch,
- * prompt_len].  Asynchronous. */
+ * prompt_len].  Synchronises the stream once (the stage tables of the batch
+ * are uploaded from host memory of the context); the prefill kernels and the
+ * ingestion of the prompt are then enqueued without waiting. */
 XSM_API xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_t *d_prompt,
                        int prompt_len, const xsm_decode_config *dc);
 
@@ -132,12 +139,15 @@ XSM_API xsm_status xsm_spec_step(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d
  * device.  Every GPU that loads the library holds the 1 MiB until the process exits.  The first call on a
  * device looks up the array's device address; make that call before any stream capture.  A batch whose
  * partials exceed the array (batch * n_heads * splits * (K+1) * (d_head+2) floats, twice) is refused with
- * XSM_ERR_CAPACITY.  All contexts of a process share the array and it keeps the last call's contents; the
+ * XSM_ERR_CAPACITY.  The two step calls may alternate freely on one context: when xsm_spec_step, xsm_generate or
+ * another call that steps follows this one, the workspace copy of the partials is cleared first.  All contexts of a process share the array and it keeps the last call's contents; the
  * call clears the part it uses first, so calls must not overlap on the GPU (same stream, or otherwise
  * ordered): overlapping calls race.  Arguments and results as xsm_spec_step.  Asynchronous. */
 XSM_API xsm_status xsm_spec_step_static(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_n_new);
 
-/* Runs steps until every sequence has committed max_new_tokens tokens since
+/* Algorithm 1's loop (line 2: while s < L_max and no EOS is committed) and its
+ * output x_{0:i_EOS} (line 14), for every mesh of the batch.
+ * Runs steps until every sequence has committed max_new_tokens tokens since
  * xsm_prefill, met EOS, or reached max_seq_len.  d_tokens: DEVICE int32
  * [batch, max_new_tokens] (x_1, x_2, ...; unused tail -1); d_lengths: DEVICE
  * int32 [batch].  host_stats (HOST, may be NULL) is filled before returning.
@@ -153,6 +163,7 @@ XSM_API xsm_status xsm_generate_host(xsm_ctx *ctx, int batch, const void *h_cond
                              int prompt_len, const xsm_decode_config *dc, int max_new_tokens,
                              int32_t *h_tokens, int32_t *h_lengths, xsm_stats *host_stats);
 
+/* Ends the context (waits for its stream); weights and workspace go back to the caller. */
 XSM_API xsm_status xsm_destroy(xsm_ctx *ctx);
 
 /* Text of the last error of this context (or of the last failed xsm_create when ctx is NULL). */
@@ -185,6 +196,23 @@ XSM_API xsm_status xsm_debug_get_state(xsm_ctx *ctx, int32_t *h_len, int32_t *h_
  * outputs; one column per CTA of the persistent kernel; 0 = that CTA had nothing to wait for in that stage.
  * capacity = number of uint64 words h_times can hold.  Synchronises the stream. */
 XSM_API xsm_status xsm_debug_trace_step(xsm_ctx *ctx, uint64_t *h_times, size_t capacity, int *n_rows, int *n_ctas);
+
+/* Load generator for Sec. 5.1's speedup = SCR x latency(K = 0) / latency(K): from the next step on, the drafts of
+ * every sequence are taken from h_tokens (HOST int32 [batch, n], token of every absolute position 0..n-1) instead
+ * of from the decoding heads; at step t the first floor((t+1) a) - floor(t a) drafts are left intact and the others
+ * are made wrong (a = mean_accept in [0, K]).  With a script that the backbone reproduces (its own greedy
+ * continuation under strict-greedy verification) the accept length of every step is forced, and SCR = 1 + a.
+ * h_tokens == NULL or n == 0 turns it off; xsm_prefill turns it off too.  Synchronises the stream. */
+XSM_API xsm_status xsm_debug_set_script(xsm_ctx *ctx, const int32_t *h_tokens, int n, float mean_accept);
+
+/* Bounds of the device-side waits: polls of one exchanged word and tries of one shared-memory barrier before a
+ * CTA gives up, raises XSM_ERR_TIMEOUT and leaves at the end of the step.  0 restores the default (2^21, 2^22). */
+XSM_API xsm_status xsm_debug_set_wait_limits(xsm_ctx *ctx, uint32_t polls, uint32_t barrier_tries);
+
+/* Launches stage `stage` (0-based: eight per layer, then the tail) of the current step alone, without advancing the
+ * step counter.  A stage whose inputs no earlier launch has published waits for them until the limit above runs
+ * out; the status then shows at the next synchronising call, and xsm_prefill starts afresh. */
+XSM_API xsm_status xsm_debug_launch_stage(xsm_ctx *ctx, int stage);
 
 /* Runs the step one stage per launch instead of as one persistent kernel (1) or back (0). */
 XSM_API xsm_status xsm_debug_set_phase_launch(xsm_ctx *ctx, int on);

@@ -22,7 +22,8 @@ EXPORTS = [
     "xsm_weights_bytes", "xsm_workspace_bytes", "xsm_create", "xsm_prefill", "xsm_spec_step", "xsm_generate",
     "xsm_generate_host", "xsm_destroy", "xsm_last_error", "xsm_kernel_launches", "xsm_debug_get_logits",
     "xsm_debug_get_kv", "xsm_debug_set_drafts", "xsm_debug_get_state", "xsm_debug_set_phase_launch",
-    "xsm_debug_trace_step", "xsm_spec_step_static",
+    "xsm_debug_trace_step", "xsm_spec_step_static", "xsm_debug_set_wait_limits", "xsm_debug_launch_stage",
+    "xsm_debug_set_script",
 ]
 
 
@@ -83,6 +84,9 @@ def load(path: str | None = None):
     L.xsm_debug_set_drafts.argtypes = [vp, ip]
     L.xsm_debug_get_state.argtypes = [vp, ip, ip, ip, ip, ip]
     L.xsm_debug_set_phase_launch.argtypes = [vp, C.c_int]
+    L.xsm_debug_set_script.argtypes = [vp, ip, C.c_int, C.c_float]
+    L.xsm_debug_set_wait_limits.argtypes = [vp, C.c_uint32, C.c_uint32]
+    L.xsm_debug_launch_stage.argtypes = [vp, C.c_int]
     L.xsm_debug_trace_step.argtypes = [vp, vp, C.c_size_t, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     if path is None:
         _lib = L
@@ -231,6 +235,20 @@ class Context:
 
     def xsm_debug_set_phase_launch(self, on: bool):
         self._check(self.lib.xsm_debug_set_phase_launch(self._h, int(on)))
+
+    def xsm_debug_set_script(self, tokens, mean_accept: float):
+        """tokens: [batch, n] token of every absolute position (None: off)."""
+        if tokens is None:
+            self._check(self.lib.xsm_debug_set_script(self._h, None, 0, 0.0))
+            return
+        a = np.ascontiguousarray(tokens, dtype=np.int32).reshape(self.batch, -1)
+        self._check(self.lib.xsm_debug_set_script(self._h, _np_ptr(a), a.shape[1], float(mean_accept)))
+
+    def xsm_debug_set_wait_limits(self, polls: int = 0, barrier_tries: int = 0):
+        self._check(self.lib.xsm_debug_set_wait_limits(self._h, polls, barrier_tries))
+
+    def xsm_debug_launch_stage(self, stage: int):
+        self._check(self.lib.xsm_debug_launch_stage(self._h, stage))
 
     def xsm_destroy(self):
         if self._h:

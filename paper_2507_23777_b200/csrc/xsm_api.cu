@@ -8,6 +8,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <atomic>
 #include <string>
 #include <vector>
 
@@ -26,7 +27,7 @@ struct Layout {
     size_t total = 0;
     size_t phases, jobs, wkc_off, wvc_off;
     size_t len, window, cand, acc_len, finished, n_gen, n_blocks, ingest_left, step_idx, block_table, free_stack,
-        scalars, hist, steps, tok_log, step_tokens, step_n_new, prompt;
+        scalars, hist, steps, tok_log, step_tokens, step_n_new, prompt, script;
     size_t h, rope_cs;
     size_t xchg_begin, hpub, qkv, attn, qc, cattn, act, y, logits0, hlogits, part, cpart, candx, header, done, sspub, xchg_end;
     size_t stage_cond, stage_kv, stage_tok, trace, ckv_pool, kv_pool;
@@ -73,6 +74,7 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.step_tokens = take(cur, 4 * M);
     L.step_n_new = take(cur, 4 * B);
     L.prompt = take(cur, 4 * B * (c.max_seq_len + 1));
+    L.script = take(cur, 4 * B * L.tok_ld);
     L.h = take(cur, 4 * M * d);
     L.rope_cs = take(cur, 8 * (size_t)(c.max_seq_len + K1 + 1) * (dh / 2));
     // tagged exchange buffers, cleared together at every xsm_prefill
@@ -198,6 +200,7 @@ struct xsm_ctx {
     Dev dev;
     int grid, sm_count, smem_bytes, phase_launch, prefilled, batch;
     uint32_t serial;          // decoding steps launched since the last xsm_prefill
+    int static_steps;         // the latest step kept its attention partials in the library's own scratch array
     uint64_t launches;
     std::string err;
     Tables h_tab;
@@ -356,8 +359,15 @@ xsm_status check_device_status(xsm_ctx *ctx) {
 }
 
 // n_steps decoding steps on the stream
-xsm_status run_steps(xsm_ctx *ctx, int n_steps) {
+xsm_status run_steps(xsm_ctx *ctx, int n_steps, bool static_scratch = false) {
     const int np = ctx->n_stages;
+    if (!static_scratch && ctx->static_steps) {
+        // The steps since the workspace partials were last written went through the library's scratch array, so the
+        // workspace copy still carries the tags of an older step; tags repeat with period three, and a stale word
+        // could pass for a fresh partial.  It restarts from "never written".
+        XSM_CUDA(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.part, 0, ctx->lay.candx - ctx->lay.part, ctx->stream));
+    }
+    ctx->static_steps = static_scratch ? 1 : 0;
     if (!ctx->phase_launch) {
         XSM_CUDA(ctx, launch_step(ctx->dev, ctx->cfg.dtype, 0, np, n_steps, ctx->serial, ctx->grid, ctx->smem_bytes, ctx->stream));
         ctx->launches += 1;
@@ -412,6 +422,7 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     ctx->ws_bytes = workspace_bytes;
     ctx->stream = (cudaStream_t)cuda_stream;
     ctx->phase_launch = 0; ctx->prefilled = 0; ctx->batch = 0; ctx->launches = 0; ctx->last_wall_ms = 0; ctx->serial = 0;
+    ctx->static_steps = 0;
     ctx->pinned = nullptr; ctx->ev0 = ctx->ev1 = nullptr;
     auto bail = [&](cudaError_t e, const char *what) {
         g_create_error = std::string(what) + ": " + cudaGetErrorString(e);
@@ -468,6 +479,7 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     D.max_seq_len = cfg->max_seq_len; D.tok_ld = L.tok_ld;
     D.eps = cfg->rms_eps; D.scale = (float)(1.0 / sqrt((double)cfg->d_head)); D.bos = cfg->bos_id; D.eos = cfg->eos_id;
     D.max_new = INT_MAX;
+    D.spin_limit = kSpinLimit; D.mbar_limit = kMbarSpinLimit;
     D.tables = at<Tables>(ctx, L.phases);
     D.E = wptr(ctx, ctx->wo.E);
     D.len = at<int>(ctx, L.len); D.window = at<int>(ctx, L.window); D.cand = at<int>(ctx, L.cand);
@@ -544,6 +556,8 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
     // no tag of an earlier generation may survive: the exchange buffers restart from "never written"
     XSM_CUDA(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.xchg_begin, 0, ctx->lay.xchg_end - ctx->lay.xchg_begin, ctx->stream));
     ctx->serial = 0;
+    ctx->static_steps = 0;
+    D.script = nullptr; D.script_n = 0; D.script_acc = 0;
     // the table above is read from host memory that the next prefill rewrites
     XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     XSM_CUDA(ctx, launch_cross_kv(D, c.dtype, ctx->weights, at<size_t>(ctx, ctx->lay.wkc_off),
@@ -578,8 +592,7 @@ xsm_status xsm_spec_step(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_n_new) 
 // for once per device (cudaGetSymbolAddress) and kept.
 constexpr size_t kStaticScratchBytes = (size_t)1 << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-constexpr int kMaxDevices = 64;
-static void *g_static_scratch_addr[kMaxDevices];   // by device ordinal; null until the first call on that device
+static std::atomic<void *> g_static_scratch_addr[kMaxDevices];   // by device ordinal; null until the first call on that device
 
 xsm_status xsm_spec_step_static(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_n_new) {
     if (!ctx) return XSM_ERR_INVALID_ARG;
@@ -595,19 +608,19 @@ xsm_status xsm_spec_step_static(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_
     int dev = 0;
     XSM_CUDA(ctx, cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return fail(ctx, XSM_ERR_INVALID_ARG, "device ordinal out of range");
-    if (g_static_scratch_addr[dev] == nullptr) {   // set-up, once per device, with that device current
-        void *p = nullptr;
+    if (g_static_scratch_addr[dev].load() == nullptr) {   // set-up, once per device, with that device current
+        void *p = nullptr;                                // (threads that race here all store the same address)
         XSM_CUDA(ctx, cudaGetSymbolAddress(&p, g_static_scratch));
-        g_static_scratch_addr[dev] = p;
+        g_static_scratch_addr[dev].store(p);
     }
-    char *scratch = static_cast<char *>(g_static_scratch_addr[dev]);
+    char *scratch = static_cast<char *>(g_static_scratch_addr[dev].load());
     // the array keeps what the last call left; a stale tag would pass for a fresh partial, so it restarts from zero
     XSM_CUDA(ctx, cudaMemsetAsync(scratch, 0, 2 * half, ctx->stream));
     float *const ws_part = D.part, *const ws_cpart = D.cpart;
     D.part = reinterpret_cast<float *>(scratch);
     D.cpart = reinterpret_cast<float *>(scratch + half);
     D.max_new = INT_MAX;
-    const xsm_status st = run_steps(ctx, 1);     // the kernel arguments are copied at launch
+    const xsm_status st = run_steps(ctx, 1, true);     // the kernel arguments are copied at launch
     D.part = ws_part;
     D.cpart = ws_cpart;
     if (st != XSM_OK) return st;
@@ -799,6 +812,38 @@ xsm_status xsm_debug_trace_step(xsm_ctx *ctx, uint64_t *h_times, size_t capacity
     XSM_CUDA(ctx, cudaMemcpy(h_times, d_trace, 8 * words, cudaMemcpyDeviceToHost));
     *n_rows = rows;
     *n_ctas = ctx->grid;
+    return XSM_OK;
+}
+
+xsm_status xsm_debug_set_script(xsm_ctx *ctx, const int32_t *h_tokens, int n, float mean_accept) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "xsm_debug_set_script before xsm_prefill");
+    Dev &D = ctx->dev;
+    if (h_tokens == nullptr || n <= 0) { D.script = nullptr; D.script_n = 0; D.script_acc = 0; return XSM_OK; }
+    if (n > ctx->lay.tok_ld) return fail(ctx, XSM_ERR_INVALID_ARG, "script longer than max_seq_len + n_draft + 1");
+    if (!(mean_accept >= 0.f) || mean_accept > (float)D.K) return fail(ctx, XSM_ERR_INVALID_ARG, "mean_accept must be in [0, n_draft]");
+    for (long long i = 0; i < (long long)D.B * n; ++i)
+        if (h_tokens[i] < 0 || h_tokens[i] >= D.V) return fail(ctx, XSM_ERR_INVALID_ARG, "script token out of range");
+    int *d_script = at<int>(ctx, ctx->lay.script);
+    XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    XSM_CUDA(ctx, cudaMemcpy(d_script, h_tokens, sizeof(int32_t) * (size_t)D.B * n, cudaMemcpyHostToDevice));
+    D.script = d_script; D.script_n = n; D.script_acc = (int)lrintf(mean_accept * 1024.f);
+    return XSM_OK;
+}
+
+xsm_status xsm_debug_set_wait_limits(xsm_ctx *ctx, uint32_t polls, uint32_t barrier_tries) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    ctx->dev.spin_limit = polls ? polls : kSpinLimit;
+    ctx->dev.mbar_limit = barrier_tries ? barrier_tries : kMbarSpinLimit;
+    return XSM_OK;
+}
+
+xsm_status xsm_debug_launch_stage(xsm_ctx *ctx, int stage) {
+    if (!ctx) return XSM_ERR_INVALID_ARG;
+    if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "xsm_debug_launch_stage before xsm_prefill");
+    if (stage < 0 || stage >= ctx->n_stages) return fail(ctx, XSM_ERR_INVALID_ARG, "no such stage");
+    XSM_CUDA(ctx, launch_step(ctx->dev, ctx->cfg.dtype, stage, stage + 1, 1, ctx->serial, ctx->grid, ctx->smem_bytes, ctx->stream));
+    ctx->launches += 1;
     return XSM_OK;
 }
 

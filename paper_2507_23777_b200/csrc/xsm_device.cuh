@@ -27,13 +27,13 @@
 #include <cuda_fp16.h>
 #include <math.h>
 
+#include <atomic>
+
 namespace xsm {
 
 typedef __nv_bfloat16 bf16;
 
 constexpr int XSM_STATUS_TIMEOUT = 5, XSM_STATUS_CAPACITY = 3;
-constexpr unsigned kSpinLimit = 1u << 21;      // polls of a tagged word (each an L2 round trip)
-constexpr unsigned kMbarSpinLimit = 1u << 22;  // mbarrier try_wait calls
 constexpr float kNegBig = -1.0e30f;            // "no key seen yet" (finite: tags must not turn it into a NaN)
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -277,7 +277,7 @@ __device__ __forceinline__ uint4 poll_u4(const Dev &D, Ctl *ctl, const void *p, 
     unsigned it = 0;
     while (!tags_ok(v, tag)) {
         if (ctl->dead) break;
-        if (++it > kSpinLimit) { raise_timeout(D, ctl); break; }
+        if (++it > D.spin_limit) { raise_timeout(D, ctl); break; }
         if ((it & 1023u) == 0u && ld_relaxed_u32(D.status) != 0u) { ctl->dead = 1; break; }
         v = ld_relaxed_u4(p);
     }
@@ -288,7 +288,7 @@ __device__ __forceinline__ uint32_t poll_u32(const Dev &D, Ctl *ctl, const void 
     unsigned it = 0;
     while ((v & 3u) != tag) {
         if (ctl->dead) break;
-        if (++it > kSpinLimit) { raise_timeout(D, ctl); break; }
+        if (++it > D.spin_limit) { raise_timeout(D, ctl); break; }
         if ((it & 1023u) == 0u && ld_relaxed_u32(D.status) != 0u) { ctl->dead = 1; break; }
         v = ld_relaxed_u32(p);
     }
@@ -313,7 +313,7 @@ __device__ __forceinline__ uint32_t ring_add(const Smem &S, uint32_t pos, int k)
 }
 
 __device__ __forceinline__ void mbar_wait(const Dev &D, Ctl *ctl, uint32_t bar, uint32_t parity) {
-    for (unsigned it = 0; it < kMbarSpinLimit; ++it)
+    for (unsigned it = 0; it < D.mbar_limit; ++it)
         if (mbar_try_wait(bar, parity)) return;
     raise_timeout(D, ctl);
 }
@@ -1340,7 +1340,8 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
 
 // One (sequence, head, split) item.  Self-attention: the K+1 window rows (positions len+j) against the
 // cached keys of this split's pages; the last split also takes the window's own keys (row j sees window
-// keys 0..j, fp32) and appends them to the cache.  Cross-attention: the same rows against the cached
+// keys 0..j; 16-bit caches: one more tensor-core unit over a tile in the cache's format, fp32 caches: FMA) and
+// appends them to the cache.  Cross-attention: the same rows against the cached
 // condition keys, no mask, no rotation.  Splits leave (m, l, O) partials; the last split merges them.
 template <typename WT, int DH>
 static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const Stage &st, const AttnItem &it, uint32_t serial) {
@@ -1490,7 +1491,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
                 if (lane == 0) {
                     unsigned it2 = 0;
                     while (S.ctl->landed[ring_slot(S, pos)] != (unsigned char)(ring_parity(S, pos) ^ 1u) && !S.ctl->dead)
-                        if (++it2 > kMbarSpinLimit) { raise_timeout(D, S.ctl); break; }
+                        if (++it2 > D.mbar_limit) { raise_timeout(D, S.ctl); break; }
                 }
                 __syncwarp();
             }
@@ -1672,7 +1673,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
 #pragma unroll
                     for (int q = 0; q < 8; ++q) ok = ok && (wm[q] & 3u) == tag_part && (wo[q] & 3u) == tag_part;
                     if (ok || S.ctl->dead) break;
-                    if (tries > kSpinLimit) { raise_timeout(D, S.ctl); break; }
+                    if (tries > D.spin_limit) { raise_timeout(D, S.ctl); break; }
                 }
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
@@ -2070,6 +2071,19 @@ template <typename WT> __device__ __noinline__ void commit_stage(const Dev &D, u
                         s_win[j] = s_cand[j];
                         __stcg(D.cand + b * K1 + j, s_cand[j]);
                     }
+                    if (D.script != nullptr) {
+                        // scripted drafts: the next window drafts the script's tokens; the first `keep` stay as they
+                        // are, the others are made wrong (a forced accept length for a backbone that reproduces the script)
+                        const long long t = (long long)s_state[3] + 1;
+                        const int keep = (int)((((t + 1) * D.script_acc) >> 10) - ((t * D.script_acc) >> 10));
+                        const int *sc = D.script + (size_t)b * D.script_n;
+                        for (int j = 1; j < K1; ++j) {
+                            const int pos = len + j;
+                            int tok = pos < D.script_n ? sc[pos] : 0;
+                            if (j > keep) tok = tok + 1 < D.V ? tok + 1 : 0;
+                            s_win[j] = tok;
+                        }
+                    }
                     __stcg(D.step_idx + b, (uint32_t)s_state[3] + 1u);
                     atomicAdd(D.hist + (size_t)b * (kMaxDraft + 1) + a, 1ull);
                     atomicAdd(D.steps + b, 1ull);
@@ -2219,11 +2233,15 @@ template <typename WT, int NTM, int DH>
 cudaError_t launch_step_instance(const Dev &D, int st_lo, int st_hi, int n_steps, uint32_t serial0, int grid, int smem_bytes,
                                  cudaStream_t st, int *max_grid) {
     const void *fn = (const void *)step_kernel<WT, NTM, DH>;
-    static int attr_bytes = 0;     // largest dynamic shared memory this instance has been opened for
+    // largest dynamic shared memory this instance has been opened for, per device (the attribute is per device)
+    static std::atomic<int> attr_bytes[kMaxDevices];
     cudaError_t e;
-    if (smem_bytes > attr_bytes) {
+    int cur_dev = 0;
+    if ((e = cudaGetDevice(&cur_dev)) != cudaSuccess) return e;
+    if (cur_dev < 0 || cur_dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (smem_bytes > attr_bytes[cur_dev].load()) {
         if ((e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes)) != cudaSuccess) return e;
-        attr_bytes = smem_bytes;
+        attr_bytes[cur_dev].store(smem_bytes);
     }
     if (max_grid != nullptr) {     // set-up query: how many CTAs can be resident
         int dev = 0, sms = 0, per_sm = 0;

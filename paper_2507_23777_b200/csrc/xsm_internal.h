@@ -12,6 +12,9 @@ constexpr int kThreads = kConsumerThreads + 32;      // + one producer warp that
 constexpr int kMaxDraft = 16;                        // size of the histogram rows (n_draft itself is <= 15)
 constexpr int kMaxTokens = 128;                      // largest M = batch * (K + 1)
 constexpr int kMaxBatch = 128;
+constexpr int kMaxDevices = 64;                      // device ordinals the per-device host tables cover
+// Every device-side wait is bounded: polls of a tagged word (each an L2 round trip) and mbarrier try_wait calls.
+constexpr unsigned kSpinLimit = 1u << 21, kMbarSpinLimit = 1u << 22;
 
 // Ring of shared-memory slots filled by bulk copies.  A weight item is a run of consecutive weight rows at full
 // width (at most kSlotBytes, one bulk copy); a cache item is one (page, head) tile of keys followed by the tile
@@ -89,6 +92,7 @@ struct Dev {
     float delta, temperature;
     uint32_t key0, key1;
     int max_new;
+    unsigned spin_limit, mbar_limit;   // bounds of the device-side waits (kSpinLimit, kMbarSpinLimit unless a test shortens them)
     // stage tables
     const Tables *tables;
     int n_stages;                  // 8 L + stages of the tail
@@ -103,6 +107,10 @@ struct Dev {
     int *tok_log, *step_tokens, *step_n_new;
     const int *prompt;
     int prompt_len;
+    // scripted drafts (load generator of the benchmark): null, or [B][script_n] tokens by absolute position; the commit
+    // then drafts script tokens, of which the first floor((t+1) a) - floor(t a) are left intact at step t (a = script_acc / 1024)
+    const int *script;
+    int script_n, script_acc;
     // tagged exchange buffers
     float *hpub, *qkv, *attn, *qc, *cattn, *act, *y, *logits0, *hlogits, *part, *cpart;
     uint32_t *candx, *header;      // [B][K1 + 1] resampled tokens and accept length; [B][4] len, flags

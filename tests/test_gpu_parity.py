@@ -336,3 +336,153 @@ def test_capacity_and_state_errors(P):
     with pytest.raises(binding.XsmError):
         binding.Context(cfg, w, max_batch=2, workspace_bytes=4096)
     ctx.xsm_destroy()
+
+
+# ---------------------------------------------------------------- long contexts, ragged batches, sampling modes on bf16
+
+
+def _rank(z, r):
+    """Token at rank r of logits z (larger logit first, then smaller index)."""
+    return int(np.lexsort((np.arange(z.size), -z))[r])
+
+
+def planted_chain(ls, b, n_good, rank=1):
+    """Drafts for sequence b whose first n_good entries the backbone will accept: draft j is the token of rank `rank`
+    of the oracle's backbone row j-1 given the drafts before it (the rows are run through the oracle's forward,
+    which touches only cache positions the step overwrites anyway); the rest stay as they are."""
+    st = ls.ctx.xsm_debug_get_state()
+    n, win = int(st["len"][b]), st["window"][b].copy()
+    for j in range(n_good):
+        z, _ = ls.seqs[b].forward_row(int(win[j]), n + j)
+        win[j + 1] = _rank(z, rank)
+    return win[1:]
+
+
+def test_twelve_key_splits_merge_in_two_batches(P):
+    """Twelve heads of 64 leave twelve key splits per head; at a context of about 3000 tokens the last split folds in
+    eleven partials, in two batches of up to eight.  The prompt is ingested by the step kernel."""
+    cfg = inputs.config(1, n_layers=2, vocab=1500, n_cond=40, max_seq_len=3200)
+    ls = P.LockStep(cfg, batch=1)
+    prompt = [0] + [int(t) for t in np.random.default_rng(11).integers(1, cfg["vocab"], 3010)]
+    st = ls.begin(prompt)
+    assert st["len"][0] == len(prompt) - 1 and (-(-int(st["len"][0]) // 64) + 3) // 4 >= 12
+    for _ in range(6):
+        ls.step(**BF16_TOL)
+    assert ls.excused <= 2
+    ls.compare_cache(layers=[1], **BF16_TOL)
+    ls.close()
+
+
+def test_block_table_reload_after_32_pages_of_one_split(P):
+    """Sixteen heads and four sequences leave two key splits per item; with 32-token pages a context of about 2400
+    tokens gives each split 38 pages, so the producer fetches a second batch of block-table entries."""
+    cfg = inputs.config(2, **_shape(512, 16, 32, 1024, 2, V=900, C=33, page_size=32, max_seq_len=2600))
+    ls = P.LockStep(cfg, batch=4)
+    prompt = [0] + [int(t) for t in np.random.default_rng(12).integers(1, cfg["vocab"], 2420)]
+    st = ls.begin(prompt)
+    assert (st["len"] == len(prompt) - 1).all() and -(-int(st["len"][0]) // 32) // 2 > 32
+    for _ in range(6):
+        ls.step(**BF16_TOL)
+    assert ls.excused <= 4
+    ls.compare_cache(layers=[1], **BF16_TOL)
+    ls.close()
+
+
+def test_context_of_twelve_thousand_tokens_at_the_width_of_configuration_2(P):
+    """The regime the benchmark ends in: 16 heads of 64, nine key splits per head, 21 pages per split (a warp owns
+    three of them).  One layer and a narrow feed-forward block keep the oracle's ingestion affordable."""
+    cfg = inputs.config(2, n_layers=1, d_ff=1024, vocab=1500, n_cond=40, max_seq_len=12288)
+    ls = P.LockStep(cfg, batch=1)
+    prompt = [0] + [int(t) for t in np.random.default_rng(13).integers(1, cfg["vocab"], 12050)]
+    st = ls.begin(prompt)
+    assert st["len"][0] == len(prompt) - 1
+    for _ in range(4):
+        ls.step(**BF16_TOL)
+    assert ls.excused <= 2
+    n = int(ls.ctx.xsm_debug_get_state()["len"][0])
+    # the cache of the last pages (appended by the steps above and by the end of the ingestion)
+    k, v = ls.ctx.xsm_debug_get_kv(0, 0, n - 200, 200)
+    ok = np.stack([ls.seqs[0].kv(0, 0, p) for p in range(n - 200, n)])
+    ov = np.stack([ls.seqs[0].kv(0, 1, p) for p in range(n - 200, n)])
+    assert P.logits_close(k, ok, **BF16_TOL).all() and P.logits_close(v, ov, **BF16_TOL).all()
+    ls.close()
+
+
+def test_ragged_accept_lengths_across_a_batch_of_sixteen(P):
+    """Configuration 3's shape at reduced depth: sixteen meshes, top-5 acceptance, top-5 / T = 0.5 resampling.  Every
+    second sequence gets drafts of which the first 1..K are the backbone's own runner-up tokens, so accept lengths
+    differ across the batch and every sequence rolls back by its own amount in the shared pool."""
+    cfg = inputs.config(3, n_layers=2, max_seq_len=256)
+    ls = P.LockStep(cfg, batch=16)
+    ls.begin()
+    K, seen = cfg["n_draft"], set()
+    for it in range(6):
+        st = ls.ctx.xsm_debug_get_state()
+        drafts = st["window"][:, 1:].copy()
+        want = {}
+        for b in range(0, 16, 2):
+            want[b] = 1 + (b // 2 + it) % K
+            drafts[b] = planted_chain(ls, b, want[b])
+        _, acc = ls.step(drafts=drafts, **BF16_TOL)
+        seen.update(acc)
+        if ls.excused == 0:
+            assert all(acc[b] >= want[b] for b in want), (acc, want)
+    assert len(seen) >= 4 and ls.excused <= 6
+    ls.compare_cache(layers=[1], **BF16_TOL)
+    st = ls.ctx.xsm_debug_get_state()
+    assert all(st["pages"][b] == -(-(st["len"][b] + K + 1) // 64) for b in range(16))
+    ls.close()
+
+
+@pytest.mark.parametrize("mode", ["top-5 acceptance, top-5 / T = 0.5", "threshold 0.5", "threshold 0.05"])
+def test_multi_token_commits_on_a_bf16_model(P, mode):
+    """Configuration 2 at reduced depth for 24 steps with planted drafts, so that several tokens are committed per
+    step: with the configured rule (draft within the backbone's top 5, candidates drawn from the top 5 at T = 0.5)
+    and with the paper's main rule (backbone probability of the draft above delta, Sec. 4.2)."""
+    over = dict(n_layers=3, max_seq_len=512)
+    if mode.startswith("threshold"):
+        over.update(verify_mode=2, delta=float(mode.split()[1]))
+    cfg = inputs.config(2, **over)
+    ls = P.LockStep(cfg, batch=1)
+    ls.begin()
+    K, acc = cfg["n_draft"], []
+    for it in range(24):
+        # threshold: the backbone's best token (the only one that can pass 0.5); top-k: its runner-up
+        drafts = planted_chain(ls, 0, it % (K + 1), rank=0 if cfg["verify_mode"] == 2 else 1)
+        _, a = ls.step(drafts=np.asarray([drafts]), **BF16_TOL)
+        acc.extend(a)
+    assert ls.excused <= 4
+    if cfg["verify_mode"] == 1:
+        assert max(acc) == K and sum(acc) >= 24
+    else:
+        assert cfg["delta"] >= 0.5 or max(acc) >= 1, acc      # the best token of a row holds about a tenth of the mass
+    ls.compare_cache(layers=[2], **BF16_TOL)
+    ls.close()
+
+
+def test_a_wait_that_runs_out_ends_the_kernel_cleanly_and_prefill_recovers(P):
+    """A stage is launched alone whose inputs no launch has published (the out-projection of layer 0, which reads the
+    attention rows), with the poll limit cut to a few thousand: every CTA gives up, finishes its ring protocol and
+    leaves; the host reports XSM_ERR_TIMEOUT at the next synchronising call; the context works again after xsm_prefill.
+    Nothing here faults or hangs: the wait is a bounded loop of loads that ends by counting."""
+    from paper_2507_23777_b200 import binding
+    cfg = gpu_cfg(dtype=1, n_draft=2, sigma=0.05)
+    w = inputs.make_weights(cfg, random_gains=True)
+    cond = inputs.make_cond(cfg, 1)
+    dc = binding.decode_config(cfg)
+    ref = binding.Context(cfg, w)
+    ref.prefill(cond, [0], dc)
+    want, _, _ = ref.generate(24)
+    ref.xsm_destroy()
+    ctx = binding.Context(cfg, w)
+    ctx.prefill(cond, [0], dc)
+    ctx.xsm_debug_set_wait_limits(3000, 0)
+    ctx.xsm_debug_launch_stage(2)
+    with pytest.raises(binding.XsmError) as e:
+        ctx.xsm_debug_get_state()
+    assert e.value.status == binding.XSM_ERR_TIMEOUT
+    ctx.xsm_debug_set_wait_limits(0, 0)
+    ctx.prefill(cond, [0], dc)
+    got, lens, _ = ctx.generate(24)
+    assert lens[0] == 24 and np.array_equal(got, want)
+    ctx.xsm_destroy()

@@ -52,6 +52,39 @@ def test_static_scratch_step_matches_workspace_step():
     sta.xsm_destroy()
 
 
+def test_the_two_step_calls_alternate_on_one_context():
+    """One ordinary step, two through the built-in scratch, one ordinary, and so on, on ONE context, well past the
+    context length where self-attention is split over several CTAs: the tokens equal those of a context that only
+    takes ordinary steps.  (The partials carry a tag that repeats every three writes; the library clears the
+    workspace copy when a caller comes back from the built-in scratch, or a stale partial could pass for a new one.)"""
+    import torch
+    assert torch.cuda.is_available(), "this test needs a B200"
+    from paper_2507_23777_b200 import binding, build
+    build.build()
+    for n_layers in (2, 4):          # the tag of a layer's partials depends on (step * layers + layer) mod 3
+        cfg = gpu_cfg(dtype=1, n_draft=2, max_seq_len=512, sigma=0.05, seed=9, n_layers=n_layers)
+        w = inputs.make_weights(cfg, random_gains=True)
+        cond = inputs.make_cond(cfg, 2)
+        dc = binding.decode_config(cfg)
+        ref = binding.Context(cfg, w, max_batch=2)
+        mix = binding.Context(cfg, w, max_batch=2)
+        ref.prefill(cond, [0], dc)
+        mix.prefill(cond, [0], dc)
+        K1 = cfg["n_draft"] + 1
+        mk = lambda: (torch.empty((2, K1), dtype=torch.int32, device="cuda"), torch.empty(2, dtype=torch.int32, device="cuda"))
+        (rt, rn), (mt, mn) = mk(), mk()
+        for step in range(260):
+            ref.xsm_spec_step(rt, rn)
+            if step % 4 in (1, 2):
+                mix.xsm_spec_step_static(mt, mn)
+            else:
+                mix.xsm_spec_step(mt, mn)
+            assert torch.equal(rn, mn) and torch.equal(rt, mt), f"step {step} differs ({n_layers} layers)"
+        assert int(ref.xsm_debug_get_state()["len"].max()) > 5 * cfg["page_size"]
+        ref.xsm_destroy()
+        mix.xsm_destroy()
+
+
 def test_static_scratch_refuses_what_does_not_fit():
     import torch
     assert torch.cuda.is_available(), "this test needs a B200"
