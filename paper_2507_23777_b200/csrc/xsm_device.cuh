@@ -400,7 +400,15 @@ struct SegPlan {
 };
 struct SegRec { int lo, hi; SegPlan p; };    // rows [lo, hi) of the job belong to this CTA
 static_assert(sizeof(SegRec) == kSegRecBytes, "size of a plan record");
-template <typename WT> __device__ __forceinline__ SegPlan seg_plan(const Smem &S, const GemvJob &J, int lo, int hi) {
+// Projections of at most eight token rows whose activations fit the staging area at once (batch 1) take the path of
+// consume_small: every warp multiplies all tiles of a group over its share of the columns.
+constexpr int kSmallTiles = 4;        // tiles of a group on that path (their accumulators live in registers)
+constexpr int kSmallRedBytes = 512;   // partial products of one warp for one tile: [8 tokens][16 rows] floats
+template <typename WT> __device__ __forceinline__ bool small_mode(const Dev &D, int kdim) {
+    return sizeof(WT) == 2 && D.M <= 8 && D.kca >= kdim && (int)gridDim.x * D.M <= 1536 && (((int)gridDim.x * D.M) & 3) == 0 &&
+           D.acts_bytes - D.M * (kdim * 4 + 16) >= kConsumerWarps * kSmallRedBytes;
+}
+template <typename WT> __device__ __forceinline__ SegPlan seg_plan(const Dev &D, const Smem &S, const GemvJob &J, int lo, int hi) {
     SegPlan p;
     p.row_bytes = J.kdim * (int)sizeof(WT);            // the host refuses rows beyond kItemBytes
     const int fit = kItemBytes / p.row_bytes;          // whole rows per item
@@ -413,6 +421,11 @@ template <typename WT> __device__ __forceinline__ SegPlan seg_plan(const Smem &S
     p.n_tiles = (hi - lo + p.tile_units - 1) / p.tile_units;
     p.ipt = max(1, p.tile_rows >> p.rpi_shift);
     p.tpg = max(1, min(kConsumerWarps, S.n_slots / p.ipt));
+    if (small_mode<WT>(D, J.kdim)) {
+        // the warps' partial products of a group sit behind the staged activations
+        const int room = D.acts_bytes - D.M * (J.kdim * 4 + 16);
+        p.tpg = max(1, min(min(kSmallTiles, p.tpg), room / (kConsumerWarps * kSmallRedBytes)));
+    }
     return p;
 }
 // valid weight rows of item `it` of a tile that starts at unit u0 and has nu units, and where they come from
@@ -1086,11 +1099,315 @@ __device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, con
     }
 }
 
+// ------------------------------------------------------------- projection: consumer, few token rows (batch 1)
+
+// the same product as mma16816, left to the compiler's scheduler (no ordering against other statements)
+__device__ __forceinline__ void mma16816_free(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0,
+                                              unsigned b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Stages the whole tagged input of job J (at most eight rows) as {hi01, hi23, lo01, lo23} words, NB 16-byte loads per
+// thread in flight.  With want_ss the CTAs' shares of the rows' sums of squares travel in the same batch and are left,
+// tags stripped, in S.sspart as [CTA][row].  Ends with a barrier of the consumer warps.
+template <int NB>
+static __device__ __forceinline__ void stage_small(const Dev &D, const Smem &S, const GemvJob &J, uint32_t tag, bool want_ss) {
+    const int M = D.M, tid = threadIdx.x, kdim = J.kdim;
+    const int v4 = kdim >> 2, total = M * v4, pitch = kdim * 4 + 16;
+    const uint32_t inv = 0xFFFFFFFFu / (uint32_t)v4 + 1u;       // i / v4 == umulhi(i, inv) for i, v4 < 2^16
+    const float *x = J.x;
+    const bool dead_rows = S.ctl->any_dead != 0;
+    const int n_sh = want_ss ? ((int)gridDim.x * M) >> 2 : 0;   // 16-byte words of shares (a multiple of four words)
+    for (int i0 = 0; i0 < total; i0 += kConsumerThreads * NB) {
+        const float *src[NB];      // nullptr: nothing to fetch (past the end, or a finished sequence's row)
+        int dst[NB];               // byte offset in the staging area, -1: past the end
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+            const int i = i0 + u * kConsumerThreads + tid;
+            src[u] = nullptr; dst[u] = -1;
+            if (i < total) {
+                const int m = (int)__umulhi((uint32_t)i, inv), c4 = i - m * v4;
+                dst[u] = m * pitch + (c4 << 4);
+                if (!(dead_rows && S.ctl->row_dead[m])) src[u] = x + (size_t)m * kdim + (c4 << 2);
+            }
+        }
+        // the shares: 16-byte words tid and tid + 224 of [CTA][row] (at most 1536 floats)
+        const float *sh_src[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) sh_src[q] = (i0 == 0 && tid + q * kConsumerThreads < n_sh) ? D.sspub + 4 * (tid + q * kConsumerThreads) : nullptr;
+        uint4 w[NB], sw[2];
+        // the whole batch is requested at once; where a word has not arrived, the thread waits for the first such word
+        // alone and then requests the batch again
+        for (;;) {
+            const float *stale = nullptr;
+#pragma unroll
+            for (int u = 0; u < NB; ++u) w[u] = src[u] != nullptr ? ld_relaxed_u4(src[u]) : make_uint4(tag, tag, tag, tag);
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                sw[q] = make_uint4(tag, tag, tag, tag);
+                if (sh_src[q] != nullptr) {
+                    sw[q] = ld_relaxed_u4(sh_src[q]);
+                    if (dead_rows) {      // nobody publishes the shares of a finished sequence's rows
+                        const int r0 = (4 * (tid + q * kConsumerThreads)) % M;
+                        if (S.ctl->row_dead[r0]) sw[q].x = tag;
+                        if (S.ctl->row_dead[(r0 + 1) % M]) sw[q].y = tag;
+                        if (S.ctl->row_dead[(r0 + 2) % M]) sw[q].z = tag;
+                        if (S.ctl->row_dead[(r0 + 3) % M]) sw[q].w = tag;
+                    }
+                }
+                if (!tags_ok(sw[q], tag)) stale = sh_src[q];
+            }
+#pragma unroll
+            for (int u = NB - 1; u >= 0; --u)
+                if (!tags_ok(w[u], tag)) stale = src[u];
+            if (stale == nullptr) break;
+            poll_u4(D, S.ctl, stale, tag);
+            if (S.ctl->dead) break;
+        }
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+            if (dst[u] >= 0) {
+                uint4 o;
+                o.x = __byte_perm(w[u].x, w[u].y, 0x7632);
+                o.y = __byte_perm(w[u].z, w[u].w, 0x7632);
+                o.z = __byte_perm(w[u].x, w[u].y, 0x5410) & 0xFFFCFFFCu;
+                o.w = __byte_perm(w[u].z, w[u].w, 0x5410) & 0xFFFCFFFCu;
+                *reinterpret_cast<uint4 *>(S.acts + dst[u]) = o;
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 2; ++q)
+            if (sh_src[q] != nullptr)
+                *reinterpret_cast<float4 *>(S.sspart + 4 * (tid + q * kConsumerThreads)) =
+                    make_float4(untag(sw[q].x), untag(sw[q].y), untag(sw[q].z), untag(sw[q].w));
+    }
+    csync();
+}
+
+// Products of the warp's column blocks (32 columns each: kb = warp, warp + 7, ...) for TL tiles, KU blocks per round
+// with accumulators of their own: sixteen independent products per round whatever the shape.
+template <int TL, int KU>
+__device__ __forceinline__ void mma_small(float (&c)[kSmallTiles][4], const uint32_t (&row_a)[kSmallTiles], const uint32_t (&row_b)[kSmallTiles],
+                                          uint32_t x_addr, bool has_x, int n_kb) {
+    const int warp = threadIdx.x >> 5;
+    float acc[KU][TL][2][4];
+#pragma unroll
+    for (int ku = 0; ku < KU; ++ku)
+#pragma unroll
+        for (int tl = 0; tl < TL; ++tl)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[ku][tl][0][q] = acc[ku][tl][1][q] = 0.f;
+    for (int kb0 = warp; kb0 < n_kb; kb0 += kConsumerWarps * KU) {
+        uint4 xa[KU], xb[KU], wa[KU][TL], wb[KU][TL];
+#pragma unroll
+        for (int ku = 0; ku < KU; ++ku) {
+            const int kb = kb0 + ku * kConsumerWarps;
+            const bool ok = kb < n_kb;
+            xa[ku] = xb[ku] = make_uint4(0u, 0u, 0u, 0u);
+            if (ok && has_x) {
+                xa[ku] = lds_u4(x_addr + (uint32_t)kb * 128u);
+                xb[ku] = lds_u4(x_addr + (uint32_t)kb * 128u + 16u);
+            }
+#pragma unroll
+            for (int tl = 0; tl < TL; ++tl) {
+                wa[ku][tl] = wb[ku][tl] = make_uint4(0u, 0u, 0u, 0u);
+                if (ok) {
+                    wa[ku][tl] = lds_u4(row_a[tl] + (uint32_t)kb * 64u);
+                    wb[ku][tl] = lds_u4(row_b[tl] + (uint32_t)kb * 64u);
+                }
+            }
+        }
+        // products of one accumulator are issued as far apart as the round allows
+#pragma unroll
+        for (int ku = 0; ku < KU; ++ku)
+#pragma unroll
+            for (int tl = 0; tl < TL; ++tl) mma16816_free(acc[ku][tl][0], wa[ku][tl].x, wb[ku][tl].x, wa[ku][tl].y, wb[ku][tl].y, xa[ku].x, xa[ku].y);
+#pragma unroll
+        for (int ku = 0; ku < KU; ++ku)
+#pragma unroll
+            for (int tl = 0; tl < TL; ++tl) mma16816_free(acc[ku][tl][1], wa[ku][tl].x, wb[ku][tl].x, wa[ku][tl].y, wb[ku][tl].y, xa[ku].z, xa[ku].w);
+#pragma unroll
+        for (int ku = 0; ku < KU; ++ku)
+#pragma unroll
+            for (int tl = 0; tl < TL; ++tl) mma16816_free(acc[ku][tl][0], wa[ku][tl].z, wb[ku][tl].z, wa[ku][tl].w, wb[ku][tl].w, xb[ku].x, xb[ku].y);
+#pragma unroll
+        for (int ku = 0; ku < KU; ++ku)
+#pragma unroll
+            for (int tl = 0; tl < TL; ++tl) mma16816_free(acc[ku][tl][1], wa[ku][tl].z, wb[ku][tl].z, wa[ku][tl].w, wb[ku][tl].w, xb[ku].z, xb[ku].w);
+    }
+#pragma unroll
+    for (int tl = 0; tl < kSmallTiles; ++tl)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float v = 0.f;
+            if (tl < TL) {
+#pragma unroll
+                for (int ku = 0; ku < KU; ++ku) v += acc[ku][tl][0][q] + acc[ku][tl][1][q];
+            }
+            c[tl][q] = v;
+        }
+}
+
+// The consumer of produce_segment for at most eight token rows.  Two barriers per tile group: after the staging of
+// the activations (once per job), and after every warp has parked its partial products.  Between them warp w
+// multiplies every tile of the group over the column blocks w, w + 7, ..., and (w < M) adds up the sums of squares of
+// token row w; after them warp w finishes the outputs of token row w (unit = lane), so the row's share of the new
+// sum of squares is a shuffle reduction and no further barrier is needed.
+template <typename WT>
+static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
+    const SegPlan p = R.p;
+    const int lo = R.lo, hi = R.hi;
+    const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int kdim = J.kdim, pitch = kdim * 4 + 16;
+    const uint32_t tag_in = tag_of(serial, J.in), tag_out = tag_of(serial, J.outt);
+    const bool normed = J.gain != nullptr;
+    const bool want_ss = J.epi == EPI_ADD && J.gain_out != nullptr;
+    const int tu_shift = p.tu_shift, tu_mask = p.tile_units - 1;
+    // EPI_ADD: the residual stream's old values and the gains of the published copy for the first group, fetched while
+    // the inputs are on their way (token row = warp, unit = lane and lane + 32)
+    float hpre[2] = {0.f, 0.f}, gpre[2] = {1.f, 1.f};
+    if (J.epi == EPI_ADD && warp < M) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int u = lo + lane + 32 * q;
+            if (u < hi && lane + 32 * q < p.tpg * p.tile_units) {
+                hpre[q] = __ldcg(J.hm + (size_t)warp * J.out_ld + u);
+                if (J.gain_out != nullptr) gpre[q] = to_f(reinterpret_cast<const WT *>(J.gain_out)[u]);
+            }
+        }
+    }
+    if (M * (kdim >> 2) <= 6 * kConsumerThreads) stage_small<6>(D, S, J, tag_in, normed);
+    else stage_small<12>(D, S, J, tag_in, normed);
+    if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
+    // 1 / rms of token row `warp` (and of row warp + 7): the shares are added in a fixed order
+    float inv_rms[2] = {1.f, 1.f};
+    if (normed) {
+        const int G = (int)gridDim.x;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int m = warp + q * kConsumerWarps;
+            if (m < M) {
+                float sum = 0.f;
+                for (int c = lane; c < G; c += 32) sum += S.sspart[c * M + m];
+                sum = warp_sum(sum);
+                inv_rms[q] = S.ctl->row_dead[m] ? 1.f : 1.0f / sqrtf(sum / (float)kdim + D.eps);
+            }
+        }
+    }
+    float *red = reinterpret_cast<float *>(S.acts + M * pitch);      // [warp][tile of the group: p.tpg][token 8][row 16]
+    float ss_acc[2] = {0.f, 0.f};
+    const uint32_t x_addr = smem_u32(S.acts) + (uint32_t)(min(g, M - 1) * pitch) + (uint32_t)t * 32u;
+    for (int tg0 = 0; tg0 < p.n_tiles; tg0 += p.tpg) {
+        const int tg = min(p.tpg, p.n_tiles - tg0), n_items = tg * p.ipt;
+        const uint32_t pos0 = ring.pos;
+        // every warp reads every tile of the group: lane i waits for item i
+        if (lane < n_items) {
+            Ring r;
+            r.pos = ring_add(S, pos0, lane);
+            ring_wait(D, S, r);
+        }
+        __syncwarp();
+        uint32_t row_a[kSmallTiles], row_b[kSmallTiles];
+#pragma unroll
+        for (int tl = 0; tl < kSmallTiles; ++tl) {
+            const uint32_t pos_tile = ring_add(S, pos0, min(tl, tg - 1) * p.ipt);
+            row_a[tl] = tile_row_addr(S, p, pos_tile, g) + (uint32_t)t * 16u;
+            row_b[tl] = tile_row_addr(S, p, pos_tile, g + 8) + (uint32_t)t * 16u;
+        }
+        float c[kSmallTiles][4];
+        if (tg == 1) mma_small<1, 4>(c, row_a, row_b, x_addr, g < M, kdim >> 5);
+        else if (tg == 2) mma_small<2, 2>(c, row_a, row_b, x_addr, g < M, kdim >> 5);
+        else mma_small<4, 1>(c, row_a, row_b, x_addr, g < M, kdim >> 5);
+        __syncwarp();
+        if (lane < n_items) mbar_arrive(S.empty0 + 8u * ring_slot(S, ring_add(S, pos0, lane)));
+        ring.pos = ring_add(S, pos0, n_items);
+        if (tg0 != 0) csync();        // the previous group's partial products have been read
+#pragma unroll
+        for (int tl = 0; tl < kSmallTiles; ++tl) {
+            if (tl < tg) {
+                float *r = red + ((size_t)(warp * p.tpg + tl) * 8) * 16;
+                r[(2 * t) * 16 + g] = c[tl][0];
+                r[(2 * t + 1) * 16 + g] = c[tl][1];
+                r[(2 * t) * 16 + g + 8] = c[tl][2];
+                r[(2 * t + 1) * 16 + g + 8] = c[tl][3];
+            }
+        }
+        // EPI_HEADY adds the normalised input itself: taken from the staged copy before anyone may overwrite it
+        const int u_first = lo + tg0 * p.tile_units, ug = min(tg * p.tile_units, hi - u_first);
+        float xin[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+        if (J.epi == EPI_HEADY) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int m = warp + q * kConsumerWarps;
+#pragma unroll
+                for (int jq = 0; jq < 2; ++jq) {
+                    const int j = lane + 32 * jq;
+                    if (m < M && j < ug) {
+                        const int u = u_first + j;
+                        const uint4 o = *reinterpret_cast<const uint4 *>(S.acts + (size_t)m * pitch + ((u >> 2) << 4));
+                        const uint32_t hw = (u & 2) ? o.y : o.x, lw = (u & 2) ? o.w : o.z;
+                        const uint32_t hb = (u & 1) ? (hw & 0xFFFF0000u) : (hw << 16), lb = (u & 1) ? (lw & 0xFFFF0000u) : (lw << 16);
+                        xin[q][jq] = __uint_as_float(hb) + __uint_as_float(lb);
+                    }
+                }
+            }
+        }
+        csync();
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int m = warp + q * kConsumerWarps;
+            if (m >= M) break;
+            const float inv = inv_rms[q];
+#pragma unroll
+            for (int jq = 0; jq < 2; ++jq) {
+                const int j = lane + 32 * jq;
+                if (j >= ug) break;
+                const int tl = j >> tu_shift, ui = j & tu_mask, u = u_first + j;
+                const float *rr = red + ((size_t)tl * 8 + m) * 16 + ui;
+                float v = 0.f, v2 = 0.f;
+#pragma unroll
+                for (int w2 = 0; w2 < kConsumerWarps; ++w2) {
+                    v += rr[(size_t)w2 * p.tpg * 128];
+                    if (J.epi == EPI_GATEUP) v2 += rr[(size_t)w2 * p.tpg * 128 + 8];
+                }
+                v *= inv; v2 *= inv;
+                float *o = J.out + (size_t)m * J.out_ld + u;
+                float pub;
+                if (J.epi == EPI_STORE) pub = v;
+                else if (J.epi == EPI_GATEUP) pub = silu_f(v) * v2;
+                else if (J.epi == EPI_ADD) {
+                    float *hm = J.hm + (size_t)m * J.out_ld + u;
+                    const bool pre = tg0 == 0 && q == 0;
+                    const float r = (pre ? hpre[jq] : __ldcg(hm)) + v;
+                    __stcg(hm, r);
+                    pub = r;
+                    if (J.gain_out != nullptr) pub = r * (pre ? gpre[jq] : to_f(reinterpret_cast<const WT *>(J.gain_out)[u]));
+                    ss_acc[q] += r * r;
+                } else pub = xin[q][jq] * inv + silu_f(v);
+                st_relaxed_u32(o, publish_word<WT>(pub, tag_out, J.out_plain != 0));
+            }
+        }
+    }
+    if (want_ss) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int m = warp + q * kConsumerWarps;
+            if (m < M) {
+                const float sh = warp_sum(ss_acc[q]);
+                if (lane == 0) st_relaxed_u32(D.sspub + (size_t)blockIdx.x * M + m, tagged(sh, tag_out));
+            }
+        }
+    }
+}
+
 // NTM: token tiles of 8 (bf16 weights) or token rows (fp32 weights) the kernel is compiled for
 template <typename WT, int NTM> struct ConsumeSegment;
 template <int NTM> struct ConsumeSegment<bf16, NTM> {
     static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
         if (D.kca < J.kdim) { consume_segment_chunked<bf16>(D, S, ring, J, R, serial); return; }
+        if (NTM == 1 && small_mode<bf16>(D, J.kdim)) { consume_small<bf16>(D, S, ring, J, R, serial); return; }
         consume_segment_bf16<bf16, NTM>(D, S, ring, J, R, serial);
     }
 };
@@ -1108,7 +1425,7 @@ template <typename WT> static __device__ void plan_segments(const Dev &D, const 
     for (int i = threadIdx.x; i < n_jobs; i += blockDim.x) {
         SegRec r;
         r.lo = r.hi = 0;
-        r.p = seg_plan<WT>(S, T.jobs[i], 0, 0);
+        r.p = seg_plan<WT>(D, S, T.jobs[i], 0, 0);
         for (int s = 0; s < n_st; ++s) {
             const Stage &st = T.stages[s];
             if (st.kind != ST_GEMV || i < st.job0 || i >= st.job0 + st.njobs) continue;
@@ -1121,7 +1438,7 @@ template <typename WT> static __device__ void plan_segments(const Dev &D, const 
             const int u_lo = (int)(total * blockIdx.x / gridDim.x), u_hi = (int)(total * (blockIdx.x + 1) / gridDim.x);
             r.lo = max(u_lo - base, 0);
             r.hi = max(min(u_hi - base, T.jobs[i].rows), r.lo);
-            r.p = seg_plan<WT>(S, T.jobs[i], r.lo, r.hi);
+            r.p = seg_plan<WT>(D, S, T.jobs[i], r.lo, r.hi);
         }
         S.seg[i] = r;
     }
