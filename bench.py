@@ -104,6 +104,41 @@ def oracle_sample(cfg, weights, cond, seconds_budget=20.0, min_steps=4):
     return toks / dt, steps, dt, os.cpu_count()
 
 
+def spot_check(cfg, weights, cond, n_steps=12):
+    """The library against the oracle on one decoding step of the benchmark's own model: after n_steps steps the oracle
+    is brought to the same state (the committed tokens run through its forward) and both evaluate the next window."""
+    import oracle
+    from paper_2507_23777_b200 import binding
+    oracle.build()
+    ctx = binding.Context(cfg, weights, max_batch=1)
+    ctx.prefill(cond[:1], [cfg["bos_id"]], binding.decode_config(cfg))
+    toks = [cfg["bos_id"]]
+    for _ in range(n_steps):
+        nt, nn = ctx.step()
+        toks.extend(int(t) for t in nt[0][:nn[0]])
+    st = ctx.xsm_debug_get_state()
+    n, win = int(st["len"][0]), st["window"][0].copy()
+    assert n == len(toks) - 1 and win[0] == toks[-1]
+    ctx.step()
+    z0g, zhg = ctx.xsm_debug_get_logits()
+    ctx.xsm_destroy()
+    P = cfg["page_size"]
+    orc = oracle.Oracle(cfg, weights, n_pages=(n + 2 * cfg["n_draft"] + 2) // P + 2)
+    dc = oracle.decode_config(cfg)
+    s = orc.new_seq(cond[0], 0)
+    s.begin(toks, dc)
+    s.set_window(win)
+    _, _, z0, zh = s.step(dc, want_logits=True)
+    err = float(np.abs(z0g[0] - z0).max())
+    bound = 2e-2 + 1e-2 * np.abs(z0)
+    ok = bool((np.abs(z0g[0] - z0) <= bound).all())
+    if cfg["n_draft"]:
+        err = max(err, float(np.abs(zhg[:, 0] - zh).max()))
+        ok = ok and bool((np.abs(zhg[:, 0] - zh) <= 2e-2 + 1e-2 * np.abs(zh)).all())
+    orc.close()
+    return {"context": n, "max_logit_err": err, "bound": "2e-2 + 1e-2 |ref|", "ok": ok}
+
+
 def run_reference(args):
     cfg = workload(args)
     rank = int(os.environ.get("RANK", "0"))
@@ -154,7 +189,9 @@ def fitted_heads_arm(args, cfg, w, cond, T):
 
     cfg0 = dict(cfg, n_draft=0)
     k0 = timed(cfg0, np.ascontiguousarray(w[:inputs.n_weight_elements(cfg0)]))
-    fitted, report = fit_heads.fit(cfg, w, n_meshes=args.fit_meshes, n_tokens=512)
+    seqs, conds = fit_heads.corpus(cfg, w, args.fit_meshes, 512)
+    fitted, report = fit_heads.fit_from_corpus(cfg, w, seqs, conds)
+    report.update({"tokens_per_mesh": 512, "corpus_seed0": 5000})
     report.pop("curve")
     fh = timed(cfg, fitted)
     fh["speedup_vs_k0"] = fh["value"] / k0["value"]
@@ -162,7 +199,15 @@ def fitted_heads_arm(args, cfg, w, cond, T):
     fh["note"] = ("heads = copies of the LM head fine-tuned on the frozen backbone's own sequences of other meshes "
                   "(stage-1 loss, w(d) = 0.8^d, best held-out checkpoint); backbone and K = 0 path unchanged; the "
                   "synthetic backbone's token dynamics are far more repetitive than a trained mesh model's")
-    return {"k0": k0, "fitted_heads": fh}
+    out = {"k0": k0, "fitted_heads": fh}
+    from paper_2507_23777_b200 import sweeps
+    Ts = min(T, 2048)
+    # the paper's own acceptance rule, delta swept (Sec. 5.4), with the fitted heads
+    out["threshold_sweep"] = sweeps.threshold(cfg, fitted, cond, k0["value"], T=Ts)
+    if args.head_sweep:
+        out["head_sweep"] = sweeps.heads(cfg, lambda K: inputs.make_weights(dict(cfg, n_draft=K, seed=args.config)), cond, seqs, conds,
+                                         k0["value"], T=Ts)
+    return out
 
 
 def run_gpu(args):
@@ -275,10 +320,21 @@ def run_gpu(args):
     }
     if world == 1 and K >= 1 and not args.k0 and not args.no_fitted_heads:
         line.update(fitted_heads_arm(args, cfg, w, cond, T))
+    if world == 1 and K >= 1 and not args.k0 and not args.no_scripted and B == 1:
+        from paper_2507_23777_b200 import sweeps
+        line["scripted_drafts"] = sweeps.scripted_drafts(cfg, w, cond, T=min(T, 2048))
     if not args.no_cpu_baseline and world == 1:
+        import oracle
+        line["oracle_spot_check"] = spot_check(cfg, w, cond)
+        assert line["oracle_spot_check"]["ok"], line["oracle_spot_check"]
         v, steps, dt, cores = oracle_sample(cfg, w, cond, seconds_budget=15.0)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"first {steps} decoding steps of one mesh ({dt:.1f} s)"}
+        oracle.set_threads(1)
+        v1, steps1, dt1, _ = oracle_sample(cfg, w, cond, seconds_budget=8.0, min_steps=2)
+        oracle.set_threads(cores)
+        line["cpu_baseline"]["one_thread"] = {"value": v1, "unit": UNIT, "cores": 1,
+                                              "sample": f"first {steps1} decoding steps of one mesh ({dt1:.1f} s)"}
     print(json.dumps(line))
     ctx.xsm_destroy()
     if world > 1:
@@ -297,6 +353,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fitted-heads", action="store_true", help="skip the K = 0 and fitted-heads runs of the same mesh")
     ap.add_argument("--fit-meshes", type=int, default=64, help="meshes of 512 tokens the heads are fitted on")
+    ap.add_argument("--no-scripted", action="store_true", help="skip the scripted-draft sweep (tokens/s against forced SCR)")
+    ap.add_argument("--head-sweep", action="store_true", help="also sweep the number of decoding heads (heads fitted per count)")
     ap.add_argument("--reference-seconds", type=float, default=0.0,
                     help="--impl reference: CPU seconds per step (default: 120 s spread over the steps, 4 to 30 s each)")
     args = ap.parse_args()

@@ -200,8 +200,10 @@ XSM_API xsm_status xsm_debug_trace_step(xsm_ctx *ctx, uint64_t *h_times, size_t 
 /* Load generator for Sec. 5.1's speedup = SCR x latency(K = 0) / latency(K): from the next step on, the drafts of
  * every sequence are taken from h_tokens (HOST int32 [batch, n], token of every absolute position 0..n-1) instead
  * of from the decoding heads; at step t the first floor((t+1) a) - floor(t a) drafts are left intact and the others
- * are made wrong (a = mean_accept in [0, K]).  With a script that the backbone reproduces (its own greedy
- * continuation under strict-greedy verification) the accept length of every step is forced, and SCR = 1 + a.
+ * are made wrong (a = mean_accept in [0, K]); the token resampled at the first rejected position is replaced by the
+ * script's too.  With a script that the backbone reproduces (its own greedy continuation under strict-greedy
+ * verification) the accept length of every step is forced, and SCR = 1 + a; where the backbone's two best logits
+ * nearly tie and it disagrees with the script, that one step accepts less and the run stays on the script.
  * h_tokens == NULL or n == 0 turns it off; xsm_prefill turns it off too.  Synchronises the stream. */
 XSM_API xsm_status xsm_debug_set_script(xsm_ctx *ctx, const int32_t *h_tokens, int n, float mean_accept);
 

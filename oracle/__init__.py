@@ -50,7 +50,8 @@ class ModelConfig(C.Structure):
     _fields_ = [(n, C.c_int) for n in (
         "n_layers", "d_model", "n_heads", "d_head", "d_ff", "vocab", "n_cond", "d_cond",
         "n_draft", "head_hidden", "wdtype", "page_size", "n_pages")] + [
-        ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("bos_id", C.c_int), ("eos_id", C.c_int)]
+        ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("bos_id", C.c_int), ("eos_id", C.c_int),
+        ("head_kind", C.c_int)]
 
 
 class DecodeConfig(C.Structure):
@@ -92,6 +93,10 @@ def lib():
         L.orc_forward_row.argtypes = [vp, C.c_int, C.c_int, fp, fp]
         L.orc_head.argtypes = [vp, C.c_int, fp, fp]
         L.orc_head.restype = None
+        L.orc_seq_head.argtypes = [vp, C.c_int, fp, fp]
+        L.orc_seq_head.restype = None
+        L.orc_sample_tree.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_uint32, ip]
+        L.orc_sample_tree.restype = None
         L.orc_seq_begin.argtypes = [vp, ip, C.c_int, C.POINTER(DecodeConfig)]
         L.orc_step.argtypes = [vp, C.POINTER(DecodeConfig), ip, C.POINTER(C.c_int), fp, fp, fp]
         L.orc_generate.argtypes = [vp, C.POINTER(DecodeConfig), C.c_int, C.c_int, ip,
@@ -99,6 +104,12 @@ def lib():
         L.orc_generate_plain.argtypes = [vp, ip, C.c_int, C.POINTER(DecodeConfig), C.c_int, ip]
         _lib = L
     return _lib
+
+
+def set_threads(n: int) -> None:
+    """Number of OpenMP threads the oracle's row loops use from now on (results do not depend on it)."""
+    lib()
+    C.CDLL("libgomp.so.1").omp_set_num_threads(int(n))
 
 
 def _fp(a):
@@ -131,6 +142,14 @@ def accept(z: np.ndarray, x: int, dc: DecodeConfig) -> bool:
     return bool(lib().orc_accept(_fp(z), z.size, int(x), C.byref(dc)))
 
 
+def sample_tree(zh: np.ndarray, k_s: int, r24: int) -> np.ndarray:
+    """One path of the top-k_s probability tree over the heads' logits zh [D, V] (Appendix)."""
+    zh = np.ascontiguousarray(zh, dtype=np.float32)
+    out = np.empty(zh.shape[0], dtype=np.int32)
+    lib().orc_sample_tree(_fp(zh), zh.shape[0], zh.shape[1], int(k_s), int(r24), _ip(out))
+    return out
+
+
 def sample(z: np.ndarray, dc: DecodeConfig, r24: int) -> int:
     z = np.ascontiguousarray(z, dtype=np.float32)
     return int(lib().orc_sample(_fp(z), z.size, C.byref(dc), r24))
@@ -147,7 +166,7 @@ class Oracle:
         self.mc = ModelConfig(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["d_head"], cfg["d_ff"],
                               cfg["vocab"], cfg["n_cond"], cfg["d_cond"], cfg["n_draft"], cfg["head_hidden"],
                               cfg["dtype"], P, n_pages, cfg["rope_theta"], cfg["rms_eps"], cfg["bos_id"],
-                              cfg["eos_id"])
+                              cfg["eos_id"], cfg.get("head_kind", 0))
         want = np.uint16 if cfg["dtype"] == 1 else np.float32
         assert weights.dtype == want and weights.flags.c_contiguous
         assert weights.size == lib().orc_weight_elements(C.byref(self.mc))
@@ -240,6 +259,13 @@ class Seq:
         return out
 
     # --- compute
+    def head(self, i: int, g: np.ndarray) -> np.ndarray:
+        """Logits of decoding head i (1-based) on final hidden state g, whichever kind the model has."""
+        g = np.ascontiguousarray(g, dtype=np.float32)
+        out = np.empty(self.V, dtype=np.float32)
+        lib().orc_seq_head(self._h, i, _fp(g), _fp(out))
+        return out
+
     def forward_row(self, token: int, pos: int):
         z = np.empty(self.V, dtype=np.float32)
         g = np.empty(self.d, dtype=np.float32)

@@ -12,11 +12,15 @@
  *     to the condition c, feed-forward network) and the backbone decoder
  *     p0 = softmax(W0 h): Sec. 4.1, Eq. 2;
  *   - the causal multi-position forward: Sec. 3.1, Eq. 1;
- *   - decoding heads on the final hidden state, in the MLP form of the
- *     ablation (Table 3 rows B and C): y = g + SiLU(W1 g), logits = Wout y;
+ *   - decoding heads on the final hidden state: the cross-attention head of
+ *     Eq. 3, p(d) = softmax(W(d) CrossAttn(d)(h_s, c)), read as one residual
+ *     cross-attention layer with weights of its own (head_kind 1), and the MLP
+ *     form of the ablation (Table 3 rows B and C, head_kind 0):
+ *     y = g + SiLU(W1 g), logits = Wout y;
  *   - verification, resampling and the outer loop: Sec. 4.2 and Algorithm 1;
  *   - probability-threshold and Top-K_a acceptance: Sec. 5.4;
- *   - independent sampling of the D+1 candidates: Appendix;
+ *   - independent sampling of the D+1 candidates, and Top-K_s probability
+ *     tree sampling over the heads: Appendix (Ablation of Sampling Strategies);
  *   - step compression ratio: Sec. 5.1.
  *
  * Arithmetic: every stored value is fp32; every dot product, norm, softmax and
@@ -45,13 +49,14 @@ typedef struct {
     int page_size, n_pages;
     float rope_theta, rms_eps;
     int bos_id, eos_id;    /* eos_id < 0: no EOS */
+    int head_kind;         /* 0: MLP heads (Table 3 B, C); 1: cross-attention heads (Eq. 3) */
 } orc_model_config;
 
 typedef struct {
     int verify_mode;       /* 0 strict greedy, 1 top-K_a, 2 probability threshold */
     int k_accept;
     float delta;
-    int sample_mode;       /* 0 argmax, 1 top-k with temperature */
+    int sample_mode;       /* 0 argmax, 1 top-k with temperature, 2 top-k_sample probability tree over the heads */
     int k_sample;
     float temperature;
     uint64_t seed;
@@ -66,7 +71,8 @@ typedef struct orc_ctx {
     const void *w;
     size_t off_E, off_gf, off_W0;
     layer_off *lo;
-    size_t *off_W1, *off_Wout;
+    size_t *off_W1, *off_Wout;                 /* MLP heads */
+    size_t *off_hq, *off_hk, *off_hv, *off_ho; /* cross-attention heads: Wq, Wk, Wv, Wo of head i (then off_Wout) */
     /* shared page pool: page p holds [layer][k|v][slot][d_model] floats */
     float *pool;
     int *free_stack;
@@ -77,6 +83,7 @@ typedef struct orc_seq {
     orc_ctx *ctx;
     int seq_id;
     float *ck, *cv;        /* cross K, V: [layer][n_cond][d_model] */
+    float *hk, *hv;        /* cross-attention heads: K, V of the condition per head [head][n_cond][d_model] */
     int *block_table;      /* logical page -> physical page */
     int n_blocks, max_blocks;
     int len;               /* s: positions 0..s-1 are committed in the cache */
@@ -187,7 +194,8 @@ static void seq_release_beyond(orc_seq *s, int upto) {
 size_t orc_weight_elements(const orc_model_config *c) {
     size_t d = c->d_model, f = c->d_ff, V = c->vocab, dc = c->d_cond, hd = c->head_hidden;
     size_t per_layer = 3 * d + 6 * d * d + 2 * d * dc + 3 * d * f;
-    return V * d + c->n_layers * per_layer + d + V * d + (size_t)c->n_draft * (hd * d + V * hd);
+    size_t per_head = c->head_kind == 1 ? 2 * d * d + 2 * d * dc + V * d : hd * d + V * hd;
+    return V * d + c->n_layers * per_layer + d + V * d + (size_t)c->n_draft * per_head;
 }
 
 int orc_create(const orc_model_config *c, const void *weights, orc_ctx **out) {
@@ -221,9 +229,21 @@ int orc_create(const orc_model_config *c, const void *weights, orc_ctx **out) {
     ctx->off_W0 = o; o += V * d;
     ctx->off_W1 = (size_t *)calloc(c->n_draft + 1, sizeof(size_t));
     ctx->off_Wout = (size_t *)calloc(c->n_draft + 1, sizeof(size_t));
+    ctx->off_hq = (size_t *)calloc(c->n_draft + 1, sizeof(size_t));
+    ctx->off_hk = (size_t *)calloc(c->n_draft + 1, sizeof(size_t));
+    ctx->off_hv = (size_t *)calloc(c->n_draft + 1, sizeof(size_t));
+    ctx->off_ho = (size_t *)calloc(c->n_draft + 1, sizeof(size_t));
     for (int i = 0; i < c->n_draft; ++i) {
-        ctx->off_W1[i] = o; o += hd * d;
-        ctx->off_Wout[i] = o; o += V * hd;
+        if (c->head_kind == 1) {
+            ctx->off_hq[i] = o; o += d * d;
+            ctx->off_hk[i] = o; o += d * dc;
+            ctx->off_hv[i] = o; o += d * dc;
+            ctx->off_ho[i] = o; o += d * d;
+            ctx->off_Wout[i] = o; o += V * d;
+        } else {
+            ctx->off_W1[i] = o; o += hd * d;
+            ctx->off_Wout[i] = o; o += V * hd;
+        }
     }
     ctx->pool = (float *)calloc((size_t)c->n_pages * page_floats(ctx), sizeof(float));
     ctx->free_stack = (int *)malloc(sizeof(int) * (c->n_pages > 0 ? c->n_pages : 1));
@@ -237,6 +257,7 @@ int orc_create(const orc_model_config *c, const void *weights, orc_ctx **out) {
 void orc_destroy(orc_ctx *ctx) {
     if (!ctx) return;
     free(ctx->pool); free(ctx->free_stack); free(ctx->lo); free(ctx->off_W1); free(ctx->off_Wout);
+    free(ctx->off_hq); free(ctx->off_hk); free(ctx->off_hv); free(ctx->off_ho);
     free(ctx);
 }
 
@@ -290,6 +311,7 @@ int orc_accept(const float *z, int V, int x, const orc_decode_config *dc) {
 
 /* Draw one token from logits z with u = r24 * 2^-24. */
 int orc_sample(const float *z, int V, const orc_decode_config *dc, uint32_t r24) {
+    /* sample_mode 2 draws a single distribution (the backbone's) like sample_mode 1 */
     if (dc->sample_mode == 0) {
         int best = 0;
         for (int v = 1; v < V; ++v) if (before(z, v, best)) best = v;
@@ -339,6 +361,18 @@ int orc_seq_create(orc_ctx *ctx, const float *cond, int seq_id, int max_position
             matvec(ctx, ctx->lo[l].wvc, c->d_model, c->d_cond, cond + (size_t)j * c->d_cond,
                    s->cv + ((size_t)l * c->n_cond + j) * d);
         }
+    /* cross-attention heads: every head projects the condition with its own Wk, Wv */
+    if (c->head_kind == 1 && c->n_draft > 0) {
+        s->hk = (float *)malloc(sizeof(float) * c->n_draft * c->n_cond * d);
+        s->hv = (float *)malloc(sizeof(float) * c->n_draft * c->n_cond * d);
+        for (int i = 0; i < c->n_draft; ++i)
+            for (int j = 0; j < c->n_cond; ++j) {
+                matvec(ctx, ctx->off_hk[i], c->d_model, c->d_cond, cond + (size_t)j * c->d_cond,
+                       s->hk + ((size_t)i * c->n_cond + j) * d);
+                matvec(ctx, ctx->off_hv[i], c->d_model, c->d_cond, cond + (size_t)j * c->d_cond,
+                       s->hv + ((size_t)i * c->n_cond + j) * d);
+            }
+    }
     s->max_blocks = (max_positions + c->page_size - 1) / c->page_size;
     s->block_table = (int *)malloc(sizeof(int) * (s->max_blocks > 0 ? s->max_blocks : 1));
     s->window = (int32_t *)calloc(c->n_draft + 1, sizeof(int32_t));
@@ -349,7 +383,7 @@ int orc_seq_create(orc_ctx *ctx, const float *cond, int seq_id, int max_position
 void orc_seq_destroy(orc_seq *s) {
     if (!s) return;
     seq_release_beyond(s, 0);
-    free(s->ck); free(s->cv); free(s->block_table); free(s->window); free(s);
+    free(s->ck); free(s->cv); free(s->hk); free(s->hv); free(s->block_table); free(s->window); free(s);
 }
 
 int orc_seq_len(const orc_seq *s) { return s->len; }
@@ -465,6 +499,93 @@ void orc_head(const orc_ctx *ctx, int i, const float *g, float *logits) {
     free(y);
 }
 
+/* Cross-attention decoding head i (1-based) on final hidden state g (Eq. 3): one residual cross-attention layer with
+ * the head's own weights, y = g + Wo Attn(Wq g, Wk c, Wv c) with the backbone's head count and scale, logits = W(i) y. */
+void orc_head_ca(const orc_seq *s, int i, const float *g, float *logits) {
+    const orc_ctx *ctx = s->ctx;
+    const orc_model_config *c = &ctx->c;
+    int d = c->d_model, H = c->n_heads, dh = c->d_head;
+    float *q = (float *)malloc(sizeof(float) * d), *a = (float *)malloc(sizeof(float) * d);
+    float *t = (float *)malloc(sizeof(float) * d), *y = (float *)malloc(sizeof(float) * d);
+    const float **kr = (const float **)malloc(sizeof(float *) * c->n_cond);
+    const float **vr = (const float **)malloc(sizeof(float *) * c->n_cond);
+    matvec(ctx, ctx->off_hq[i - 1], d, d, g, q);
+    for (int j = 0; j < c->n_cond; ++j) {
+        kr[j] = s->hk + ((size_t)(i - 1) * c->n_cond + j) * d;
+        vr[j] = s->hv + ((size_t)(i - 1) * c->n_cond + j) * d;
+    }
+    for (int hh = 0; hh < H; ++hh) attend(q + hh * dh, dh, c->n_cond, kr, vr, hh * dh, a + hh * dh);
+    matvec(ctx, ctx->off_ho[i - 1], d, d, a, t);
+    for (int j = 0; j < d; ++j) y[j] = (float)((double)g[j] + (double)t[j]);
+    matvec(ctx, ctx->off_Wout[i - 1], c->vocab, d, y, logits);
+    free(q); free(a); free(t); free(y); free(kr); free(vr);
+}
+
+/* head i of either kind */
+void orc_seq_head(const orc_seq *s, int i, const float *g, float *logits) {
+    if (s->ctx->c.head_kind == 1) orc_head_ca(s, i, g, logits);
+    else orc_head(s->ctx, i, g, logits);
+}
+
+/*
+ * Top-K_s probability tree sampling over the D heads (Appendix, Ablation of Sampling Strategies).  Level d of the
+ * tree branches over the K_s most probable tokens of head d (full-vocabulary softmax probabilities m), the weight of
+ * a root-to-leaf path is the product of its m's, branches whose running product falls below 1e-5 are pruned, and
+ * one complete path is drawn with probability proportional to its weight: the leaves are walked depth first,
+ * children by rank (larger probability first, then smaller token), and the first leaf whose cumulative weight
+ * exceeds u * total is taken.  If no complete path survives the pruning, the path of every head's most probable
+ * token is returned.  zh: [D][V] logits of the heads (row of the first rejection); out: D tokens.
+ */
+#define ORC_TREE_PRUNE 1e-5
+typedef struct { int D, ks; const int *tok; const double *m; double target, cum; int found; int *path, *best; } tree_walk;
+static void tree_dfs(tree_walk *w, int depth, double weight, int pass) {
+    if (w->found) return;
+    if (depth == w->D) {
+        w->cum += weight;
+        if (pass == 1 && w->cum > w->target) { memcpy(w->best, w->path, sizeof(int) * w->D); w->found = 1; }
+        else if (pass == 1) memcpy(w->best, w->path, sizeof(int) * w->D);   /* rounding at the very end: last leaf */
+        return;
+    }
+    for (int k = 0; k < w->ks; ++k) {
+        double nw = weight * w->m[depth * w->ks + k];
+        if (nw < ORC_TREE_PRUNE) continue;
+        w->path[depth] = w->tok[depth * w->ks + k];
+        tree_dfs(w, depth + 1, nw, pass);
+        if (w->found) return;
+    }
+}
+void orc_sample_tree(const float *zh, int D, int V, int ks, uint32_t r24, int32_t *out) {
+    if (ks < 1) ks = 1;
+    if (ks > V) ks = V;
+    int *tok = (int *)malloc(sizeof(int) * D * ks), *path = (int *)malloc(sizeof(int) * D), *best = (int *)malloc(sizeof(int) * D);
+    double *m = (double *)malloc(sizeof(double) * D * ks);
+    for (int d = 0; d < D; ++d) {
+        const float *z = zh + (size_t)d * V;
+        double mx = z[0], sum = 0;
+        for (int v = 1; v < V; ++v) if (z[v] > mx) mx = z[v];
+        for (int v = 0; v < V; ++v) sum += exp((double)z[v] - mx);
+        for (int j = 0; j < ks; ++j) {           /* j-th candidate: best not yet taken */
+            int b = -1;
+            for (int v = 0; v < V; ++v) {
+                if (j > 0 && !before(z, tok[d * ks + j - 1], v)) continue;
+                if (b < 0 || before(z, v, b)) b = v;
+            }
+            tok[d * ks + j] = b;
+            m[d * ks + j] = exp((double)z[b] - mx) / sum;
+        }
+        best[d] = tok[d * ks];
+    }
+    tree_walk w = {D, ks, tok, m, 0.0, 0.0, 0, path, best};
+    tree_dfs(&w, 0, 1.0, 0);                     /* pass 0: total weight of the surviving leaves */
+    if (w.cum > 0.0) {
+        w.target = (double)r24 * (1.0 / 16777216.0) * w.cum;
+        w.cum = 0.0;
+        tree_dfs(&w, 0, 1.0, 1);
+    }
+    for (int d = 0; d < D; ++d) out[d] = best[d];
+    free(tok); free(path); free(best); free(m);
+}
+
 /* Algorithm 1, line 1: x_0 = SOS, x_{1:D} ~ U(0, V), s = 0 (prompt longer than
  * one token: all but the last prompt token are run into the cache first). */
 int orc_seq_begin(orc_seq *s, const int32_t *prompt, int prompt_len, const orc_decode_config *dc) {
@@ -508,16 +629,30 @@ int orc_step(orc_seq *s, const orc_decode_config *dc, int32_t *new_tokens, int *
     }
     /* lines 4-6: every head on every row of the window */
     for (int i = 1; i <= K; ++i)
-        for (int j = 0; j < M; ++j) orc_head(ctx, i, g + (size_t)j * d, zh + ((size_t)(i - 1) * M + j) * V);
+        for (int j = 0; j < M; ++j) orc_seq_head(s, i, g + (size_t)j * d, zh + ((size_t)(i - 1) * M + j) * V);
     /* lines 7-10: accept drafts while the backbone agrees */
     int a = 0;
     while (a < K && orc_accept(z0 + (size_t)a * V, V, s->window[a + 1], dc)) ++a;
     /* line 11: resample D+1 candidates from the row of the first rejection */
     int32_t *nw = (int32_t *)malloc(sizeof(int32_t) * M);
-    nw[0] = orc_sample(z0 + (size_t)a * V, V, dc, orc_rand24(dc->seed, s->seq_id, s->step_idx, 0, 0));
-    for (int i = 1; i <= K; ++i)
-        nw[i] = orc_sample(zh + ((size_t)(i - 1) * M + a) * V, V, dc,
-                           orc_rand24(dc->seed, s->seq_id, s->step_idx, (uint32_t)i, 0));
+    if (dc->sample_mode == 2) {
+        /* x_{s*} from the backbone's own distribution (top-K_s logits at the configured temperature), the D drafts
+         * as one path of the probability tree; slot 1's random number draws the path */
+        orc_decode_config one = *dc;
+        one.sample_mode = 1;
+        nw[0] = orc_sample(z0 + (size_t)a * V, V, &one, orc_rand24(dc->seed, s->seq_id, s->step_idx, 0, 0));
+        if (K > 0) {
+            float *rows = (float *)malloc(sizeof(float) * (size_t)K * V);
+            for (int i = 1; i <= K; ++i) memcpy(rows + (size_t)(i - 1) * V, zh + ((size_t)(i - 1) * M + a) * V, sizeof(float) * V);
+            orc_sample_tree(rows, K, V, dc->k_sample, orc_rand24(dc->seed, s->seq_id, s->step_idx, 1, 0), nw + 1);
+            free(rows);
+        }
+    } else {
+        nw[0] = orc_sample(z0 + (size_t)a * V, V, dc, orc_rand24(dc->seed, s->seq_id, s->step_idx, 0, 0));
+        for (int i = 1; i <= K; ++i)
+            nw[i] = orc_sample(zh + ((size_t)(i - 1) * M + a) * V, V, dc,
+                               orc_rand24(dc->seed, s->seq_id, s->step_idx, (uint32_t)i, 0));
+    }
     for (int j = 0; j < M; ++j) new_tokens[j] = -1;
     for (int j = 0; j < a; ++j) new_tokens[j] = s->window[j + 1];
     new_tokens[a] = nw[0];

@@ -227,7 +227,7 @@ class Context:
 
     def xsm_debug_trace_step(self) -> np.ndarray:
         """Timeline of one decoding step: uint64 [1 + 2 * stages, CTAs] nanoseconds (see include/xsm.h)."""
-        cap = (1 + 2 * (8 * self.cfg["n_layers"] + 4)) * 256
+        cap = (1 + 2 * (8 * self.cfg["n_layers"] + 6)) * 256
         buf = np.zeros(cap, dtype=np.uint64)
         rows, ctas = C.c_int(), C.c_int()
         self._check(self.lib.xsm_debug_trace_step(self._h, _np_ptr(buf), cap, C.byref(rows), C.byref(ctas)))

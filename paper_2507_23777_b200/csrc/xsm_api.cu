@@ -25,12 +25,13 @@ thread_local std::string g_create_error;
 
 struct Layout {
     size_t total = 0;
-    size_t phases, jobs, wkc_off, wvc_off;
+    size_t phases, jobs, wkc_off, wvc_off, hk_off, hv_off;
     size_t len, window, cand, acc_len, finished, n_gen, n_blocks, ingest_left, step_idx, block_table, free_stack,
         scalars, hist, steps, tok_log, step_tokens, step_n_new, prompt, script;
     size_t h, rope_cs;
-    size_t xchg_begin, hpub, qkv, attn, qc, cattn, act, y, logits0, hlogits, part, cpart, candx, header, done, sspub, xchg_end;
-    size_t stage_cond, stage_kv, stage_tok, trace, ckv_pool, kv_pool;
+    size_t xchg_begin, hpub, qkv, attn, qc, cattn, act, y, logits0, hlogits, part, cpart, candx, header, done, sspub, qh, hattn, gpub,
+        hpart, xchg_end;
+    size_t stage_cond, stage_kv, stage_tok, trace, ckv_pool, hckv_pool, kv_pool;
     int n_pages = 0, max_blocks = 0, cpages = 0, tok_ld = 0, n_phases = 0, n_jobs = 0;
     size_t page_bytes = 0;
 };
@@ -50,13 +51,16 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.max_blocks = (int)((c.max_seq_len + K1 + P - 1) / P);
     L.cpages = (int)((c.n_cond + P - 1) / P);
     L.tok_ld = c.max_seq_len + (int)K1;
-    L.n_phases = c.n_layers * 8 + 3 + (c.n_draft > 0 ? 1 : 0);
-    L.n_jobs = c.n_layers * 6 + 1 + 2 * c.n_draft;
+    const bool ca = c.head_kind == 1 && c.n_draft > 0;
+    L.n_phases = c.n_layers * 8 + 3 + (c.n_draft > 0 ? 1 : 0) + (ca ? 2 : 0);
+    L.n_jobs = c.n_layers * 6 + 1 + (ca ? 3 : 2) * c.n_draft;
     size_t cur = 0;
     L.phases = take(cur, sizeof(Tables));
     L.jobs = take(cur, 256);
     L.wkc_off = take(cur, sizeof(size_t) * c.n_layers);
     L.wvc_off = take(cur, sizeof(size_t) * c.n_layers);
+    L.hk_off = take(cur, sizeof(size_t) * (c.n_draft + 1));
+    L.hv_off = take(cur, sizeof(size_t) * (c.n_draft + 1));
     L.len = take(cur, 4 * B);
     L.window = take(cur, 4 * M);
     L.cand = take(cur, 4 * M);
@@ -95,12 +99,18 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.header = take(cur, 4 * B * kHeaderWords);
     L.done = take(cur, 4 * kSizingGrid);
     L.sspub = take(cur, 4 * (size_t)kSizingGrid * M);
+    const size_t nh = ca ? (size_t)c.n_draft : 0;       // cross-attention heads: their own exchange buffers
+    L.qh = take(cur, 4 * M * d * nh);
+    L.hattn = take(cur, 4 * M * d * nh);
+    L.gpub = take(cur, 4 * M * d * (ca ? 1 : 0));
+    L.hpart = take(cur, 4 * nh * part_items * K1 * (dh + 2));
     L.xchg_end = cur;
     L.stage_cond = take(cur, esize(c) * B * c.n_cond * c.d_cond);
     L.stage_kv = take(cur, 4 * 2 * (size_t)kKvStagePositions * d);
     L.stage_tok = take(cur, 4 * B * (c.max_seq_len + 1));
     L.trace = take(cur, 8 * (size_t)(1 + 2 * L.n_phases) * kSizingGrid);
     L.ckv_pool = take(cur, esize(c) * (size_t)c.n_layers * 2 * B * L.cpages * H * P * dh);
+    L.hckv_pool = take(cur, esize(c) * nh * 2 * B * L.cpages * H * P * dh);
     L.page_bytes = esize(c) * (size_t)c.n_layers * 2 * H * P * dh;
     // the rest is the shared page pool, preceded by its free stack (4 bytes per page)
     if (workspace_bytes == 0) {
@@ -138,7 +148,7 @@ const char *check_config(const xsm_model_config &c) {
     if (c.d_head != 32 && c.d_head != 64 && c.d_head != 128) return "d_head must be 32, 64 or 128";
     if (c.n_draft < 0 || c.n_draft >= XSM_MAX_DRAFT) return "n_draft must be in [0, 15]";
     if (c.head_hidden != c.d_model) return "head_hidden must equal d_model (the head block is residual)";
-    if (c.head_kind != 0) return "only MLP heads (head_kind 0) are implemented";
+    if (c.head_kind != 0 && c.head_kind != 1) return "head_kind must be 0 (MLP heads) or 1 (cross-attention heads)";
     if (c.dtype != 0 && c.dtype != 1) return "dtype must be 0 (fp32) or 1 (bf16)";
     if (c.page_size < 32 || c.page_size % 32) return "page_size must be a positive multiple of 32";
     if ((long long)c.page_size * c.d_head * (c.dtype == 1 ? 2 : 4) > 16384 * (c.dtype == 1 ? 1 : 4))
@@ -153,7 +163,7 @@ const char *check_config(const xsm_model_config &c) {
 
 struct WeightOffsets {
     size_t E, gf, W0;
-    std::vector<size_t> g1, wq, wo, g2, wqc, wkc, wvc, woc, g3, wgate, wup, wdown, W1, Wout;
+    std::vector<size_t> g1, wq, wo, g2, wqc, wkc, wvc, woc, g3, wgate, wup, wdown, W1, Wout, hq, hk, hv, ho;
     size_t total;
 };
 
@@ -179,8 +189,16 @@ WeightOffsets weight_offsets(const xsm_model_config &c) {
     w.gf = o; o += d;
     w.W0 = o; o += V * d;
     for (int i = 0; i < c.n_draft; ++i) {
-        w.W1.push_back(o); o += hd * d;
-        w.Wout.push_back(o); o += V * hd;
+        if (c.head_kind == 1) {          // cross-attention head (Eq. 3): Wq, Wk, Wv, Wo of its own, then W(i)
+            w.hq.push_back(o); o += d * d;
+            w.hk.push_back(o); o += d * dc;
+            w.hv.push_back(o); o += d * dc;
+            w.ho.push_back(o); o += d * d;
+            w.Wout.push_back(o); o += V * d;
+        } else {
+            w.W1.push_back(o); o += hd * d;
+            w.Wout.push_back(o); o += V * hd;
+        }
     }
     w.total = o;
     return w;
@@ -330,10 +348,29 @@ void build_tables(xsm_ctx *ctx) {
     const TagRef once{1, 0};
     int j0 = n_jobs;
     job(wptr(ctx, w.W0), nullptr, V, d, D.hpub, wptr(ctx, w.gf), D.logits0, V, EPI_STORE, TagRef{hw, 3 * L}, 0, once, 0, nullptr, 1);
-    for (int i = 0; i < K; ++i)
-        job(wptr(ctx, w.W1[i]), nullptr, d, d, D.hpub, wptr(ctx, w.gf), D.y + (size_t)i * M * d, d, EPI_HEADY,
-            TagRef{hw, 3 * L}, 0, once, 0);
-    gemv1(j0, 1 + K);
+    if (c.head_kind == 1 && K > 0) {
+        // cross-attention heads (Eq. 3): q = Wq g beside the LM head (every CTA also publishes its columns of g), the
+        // heads' attention over their own keys and values of the condition, y = g + Wo a
+        for (int i = 0; i < K; ++i)
+            job(wptr(ctx, w.hq[i]), nullptr, d, d, D.hpub, wptr(ctx, w.gf), D.qh + (size_t)i * M * d, d, EPI_STORE, TagRef{hw, 3 * L}, 0, once, 0);
+        gemv1(j0, 1 + K);
+        T.stages[n_stages - 1].norm_out = 1;
+        {
+            Stage &s = T.stages[n_stages++];
+            s.kind = ST_ATTN_HEAD;
+            s.in = once; s.outt = once; s.part = once; s.jinc = 0;
+        }
+        j0 = n_jobs;
+        for (int i = 0; i < K; ++i)
+            job(wptr(ctx, w.ho[i]), nullptr, d, d, D.hattn + (size_t)i * M * d, nullptr, D.y + (size_t)i * M * d, d, EPI_ADDG, once, 0, once, 0)
+                .res = D.gpub;
+        gemv1(j0, K);
+    } else {
+        for (int i = 0; i < K; ++i)
+            job(wptr(ctx, w.W1[i]), nullptr, d, d, D.hpub, wptr(ctx, w.gf), D.y + (size_t)i * M * d, d, EPI_HEADY,
+                TagRef{hw, 3 * L}, 0, once, 0);
+        gemv1(j0, 1 + K);
+    }
     if (K > 0) {
         j0 = n_jobs;
         for (int i = 0; i < K; ++i)
@@ -366,6 +403,8 @@ xsm_status run_steps(xsm_ctx *ctx, int n_steps, bool static_scratch = false) {
         // workspace copy still carries the tags of an older step; tags repeat with period three, and a stale word
         // could pass for a fresh partial.  It restarts from "never written".
         XSM_CUDA(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.part, 0, ctx->lay.candx - ctx->lay.part, ctx->stream));
+        if (ctx->lay.xchg_end > ctx->lay.hpart)
+            XSM_CUDA(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.hpart, 0, ctx->lay.xchg_end - ctx->lay.hpart, ctx->stream));
     }
     ctx->static_steps = static_scratch ? 1 : 0;
     if (!ctx->phase_launch) {
@@ -467,6 +506,12 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
                              cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) return bail(e, "upload");
     if ((e = cudaMemcpyAsync(ctx->ws + L.wvc_off, ctx->wo.wvc.data(), sizeof(size_t) * cfg->n_layers,
                              cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) return bail(e, "upload");
+    if (cfg->head_kind == 1 && cfg->n_draft > 0) {
+        if ((e = cudaMemcpyAsync(ctx->ws + L.hk_off, ctx->wo.hk.data(), sizeof(size_t) * cfg->n_draft, cudaMemcpyHostToDevice,
+                                 ctx->stream)) != cudaSuccess) return bail(e, "upload");
+        if ((e = cudaMemcpyAsync(ctx->ws + L.hv_off, ctx->wo.hv.data(), sizeof(size_t) * cfg->n_draft, cudaMemcpyHostToDevice,
+                                 ctx->stream)) != cudaSuccess) return bail(e, "upload");
+    }
     // the caches start at zero: slots that were never written are multiplied by zero weights and must be finite
     if ((e = cudaMemsetAsync(ctx->ws + L.ckv_pool, 0, L.total - L.ckv_pool, ctx->stream)) != cudaSuccess) return bail(e, "memset");
     if ((e = cudaStreamSynchronize(ctx->stream)) != cudaSuccess) return bail(e, "sync");
@@ -500,6 +545,9 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     D.candx = at<uint32_t>(ctx, L.candx); D.header = at<uint32_t>(ctx, L.header); D.done = at<uint32_t>(ctx, L.done);
     D.sspub = at<float>(ctx, L.sspub); D.gain_first = wptr(ctx, ctx->wo.g1[0]); D.grid = grid;
     D.kv_pool = ctx->ws + L.kv_pool; D.ckv_pool = ctx->ws + L.ckv_pool;
+    D.head_kind = cfg->head_kind;
+    D.qh = at<float>(ctx, L.qh); D.hattn = at<float>(ctx, L.hattn); D.gpub = at<float>(ctx, L.gpub); D.hpart = at<float>(ctx, L.hpart);
+    D.hckv_pool = ctx->ws + L.hckv_pool;
     *out = ctx;
     return XSM_OK;
 }
@@ -561,7 +609,12 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
     // the table above is read from host memory that the next prefill rewrites
     XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     XSM_CUDA(ctx, launch_cross_kv(D, c.dtype, ctx->weights, at<size_t>(ctx, ctx->lay.wkc_off),
-                                  at<size_t>(ctx, ctx->lay.wvc_off), d_cond, ctx->stream));
+                                  at<size_t>(ctx, ctx->lay.wvc_off), d_cond, D.ckv_pool, D.L, ctx->stream));
+    if (c.head_kind == 1 && D.K > 0) {
+        XSM_CUDA(ctx, launch_cross_kv(D, c.dtype, ctx->weights, at<size_t>(ctx, ctx->lay.hk_off),
+                                      at<size_t>(ctx, ctx->lay.hv_off), d_cond, D.hckv_pool, D.K, ctx->stream));
+        ctx->launches += 1;
+    }
     XSM_CUDA(ctx, launch_init(D, c.dtype, ctx->serial, ctx->stream));
     ctx->launches += 3;
     ctx->prefilled = 1;
@@ -598,12 +651,14 @@ xsm_status xsm_spec_step_static(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_
     if (!ctx) return XSM_ERR_INVALID_ARG;
     if (!ctx->prefilled) return fail(ctx, XSM_ERR_STATE, "xsm_spec_step_static before xsm_prefill");
     Dev &D = ctx->dev;
-    // the split partials of self- and cross-attention: [B * H * S_max][K + 1][d_head + 2] floats each
+    // the split partials of self- and cross-attention: [B * H * S_max][K + 1][d_head + 2] floats each; cross-attention
+    // heads have K more such sets
     const size_t one = (size_t)D.B * D.H * D.S_max * D.K1 * (D.dh + 2) * sizeof(float);
     const size_t half = (one + 255) / 256 * 256;
-    if (2 * half > kStaticScratchBytes)
+    const size_t n_sets = 2 + (D.head_kind == 1 ? (size_t)D.K : 0);
+    if (n_sets * half > kStaticScratchBytes)
         return fail(ctx, XSM_ERR_CAPACITY, "xsm_spec_step_static: the attention partials of this batch need " +
-                                               std::to_string(2 * half) + " bytes, the built-in scratch holds " +
+                                               std::to_string(n_sets * half) + " bytes, the built-in scratch holds " +
                                                std::to_string(kStaticScratchBytes));
     int dev = 0;
     XSM_CUDA(ctx, cudaGetDevice(&dev));
@@ -615,14 +670,16 @@ xsm_status xsm_spec_step_static(xsm_ctx *ctx, int32_t *d_new_tokens, int32_t *d_
     }
     char *scratch = static_cast<char *>(g_static_scratch_addr[dev].load());
     // the array keeps what the last call left; a stale tag would pass for a fresh partial, so it restarts from zero
-    XSM_CUDA(ctx, cudaMemsetAsync(scratch, 0, 2 * half, ctx->stream));
-    float *const ws_part = D.part, *const ws_cpart = D.cpart;
+    XSM_CUDA(ctx, cudaMemsetAsync(scratch, 0, n_sets * half, ctx->stream));
+    float *const ws_part = D.part, *const ws_cpart = D.cpart, *const ws_hpart = D.hpart;
     D.part = reinterpret_cast<float *>(scratch);
     D.cpart = reinterpret_cast<float *>(scratch + half);
+    if (D.head_kind == 1) D.hpart = reinterpret_cast<float *>(scratch + 2 * half);
     D.max_new = INT_MAX;
     const xsm_status st = run_steps(ctx, 1, true);     // the kernel arguments are copied at launch
     D.part = ws_part;
     D.cpart = ws_cpart;
+    D.hpart = ws_hpart;
     if (st != XSM_OK) return st;
     if (d_new_tokens)
         XSM_CUDA(ctx, cudaMemcpyAsync(d_new_tokens, D.step_tokens, sizeof(int32_t) * D.M, cudaMemcpyDeviceToDevice, ctx->stream));

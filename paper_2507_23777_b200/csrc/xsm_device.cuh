@@ -271,6 +271,9 @@ __device__ __forceinline__ void raise_timeout(const Dev &D, Ctl *ctl) {
     ctl->dead = 1;
 }
 
+// A CTA's share of the sum of squares of row m of the published residual stream: [row][CTA]
+__device__ __forceinline__ float *ss_word(const Dev &D, int cta, int m) { return D.sspub + (size_t)m * D.grid + cta; }
+
 // Spins until the four words at p carry `tag`.  Gives up when the CTA is dead or the status word is raised.
 __device__ __forceinline__ uint4 poll_u4(const Dev &D, Ctl *ctl, const void *p, uint32_t tag) {
     uint4 v = ld_relaxed_u4(p);
@@ -405,7 +408,7 @@ static_assert(sizeof(SegRec) == kSegRecBytes, "size of a plan record");
 constexpr int kSmallTiles = 4;        // tiles of a group on that path (their accumulators live in registers)
 constexpr int kSmallRedBytes = 512;   // partial products of one warp for one tile: [8 tokens][16 rows] floats
 template <typename WT> __device__ __forceinline__ bool small_mode(const Dev &D, int kdim) {
-    return sizeof(WT) == 2 && D.M <= 8 && D.kca >= kdim && (int)gridDim.x * D.M <= 1536 && (((int)gridDim.x * D.M) & 3) == 0 &&
+    return sizeof(WT) == 2 && D.M <= 8 && D.kca >= kdim && (int)gridDim.x * D.M <= 1536 && ((int)gridDim.x & 3) == 0 &&
            D.acts_bytes - D.M * (kdim * 4 + 16) >= kConsumerWarps * kSmallRedBytes;
 }
 template <typename WT> __device__ __forceinline__ SegPlan seg_plan(const Dev &D, const Smem &S, const GemvJob &J, int lo, int hi) {
@@ -667,11 +670,11 @@ static __device__ void gather_ss(const Dev &D, const Smem &S, uint32_t tag) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     const int c = lane + 32 * q;
-                    v[q] = c < G ? ld_relaxed_u32(D.sspub + (size_t)c * M + m) : tag;
+                    v[q] = c < G ? ld_relaxed_u32(ss_word(D, c, m)) : tag;
                 }
 #pragma unroll
                 for (int q = 7; q >= 0; --q)
-                    if ((v[q] & 3u) != tag) stale = D.sspub + (size_t)(lane + 32 * q) * M + m;
+                    if ((v[q] & 3u) != tag) stale = ss_word(D, lane + 32 * q, m);
                 if (stale == nullptr) break;
                 poll_u32(D, S.ctl, stale, tag);
                 if (S.ctl->dead) break;
@@ -742,6 +745,29 @@ __device__ __forceinline__ void mma_tile_bf16(uint32_t row_a, uint32_t row_b, co
             for (int q = 0; q < 4; ++q) { acc[nt][0][q] += au[u][nt][0][q]; acc[nt][1][q] += au[u][nt][1][q]; }
 }
 
+// A word of the published final hidden state (plain tagged fp32, written once per step by some CTA of an earlier
+// stage of the same step: it carries the step's tag by now, except when that CTA is late; bounded wait).
+__device__ __forceinline__ float residual_word(const float *p, uint32_t tag) {
+    uint32_t w = ld_relaxed_u32(p);
+    for (unsigned it = 0; (w & 3u) != tag && it < kSpinLimit; ++it) w = ld_relaxed_u32(p);
+    return untag(w);
+}
+
+// Every CTA's part of the side output of a projection stage with a normed input: columns [c d / G, (c + 1) d / G) of
+// g[m] = x[m] / rms(x[m]) (times the gain where the input is published without it), as plain tagged fp32 in D.gpub.
+// inv[m] = 1 / rms(x[m]) in shared memory.  Called by all consumer threads after the inputs have arrived.
+template <typename WT>
+__device__ __forceinline__ void publish_normed_slice(const Dev &D, const float *x, int kdim, const void *gain, const float *inv, uint32_t tag) {
+    const int G = (int)gridDim.x, c = (int)blockIdx.x;
+    const int u0 = (int)((long long)kdim * c / G), u1 = (int)((long long)kdim * (c + 1) / G), nu = u1 - u0;
+    for (int i = threadIdx.x; i < D.M * nu; i += kConsumerThreads) {
+        const int m = i / nu, u = u0 + i - m * nu;
+        float v = read_word<WT>(ld_relaxed_u32(x + (size_t)m * kdim + u)) * inv[m];
+        if (sizeof(WT) == 4) v *= reinterpret_cast<const float *>(gain)[u];
+        st_relaxed_u32(D.gpub + (size_t)m * kdim + u, tagged(v, tag));
+    }
+}
+
 // What one output element becomes (after the dot product v, already scaled by 1/rms when the job has a gain).
 // hprev: the residual stream's value when the caller has fetched it ahead (have_prev), EPI_ADD only.
 // Returns the value before any gain of the next stage is applied (the residual stream's new value for EPI_ADD).
@@ -758,6 +784,8 @@ __device__ __forceinline__ float epilogue_store(const GemvJob &J, int m, int u, 
         __stcg(hm, r);
         // bf16 models: the reader's RMSNorm gain is applied here, once, instead of by every reader
         if (sizeof(WT) == 2 && J.gain_out != nullptr) pub = r * (have_prev ? gprev : to_f(reinterpret_cast<const WT *>(J.gain_out)[u]));
+    } else if (J.epi == EPI_ADDG) {   // the final hidden state g (published by the stage before the heads' attention) + v
+        pub = r = residual_word(J.res + (size_t)m * J.out_ld + u, tag_out) + v;
     } else {   // EPI_HEADY: residual on the normalised input (this CTA has already waited for that word);
                // inv = 1 / rms(x[m]), times gain[u] where the input is published without its gain (fp32 models)
         pub = r = read_word<WT>(ld_relaxed_u32(J.x + (size_t)m * J.kdim + u)) * inv + silu_f(v);
@@ -874,6 +902,7 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
         if (gain != nullptr && ss_raw && tid < M) S.ss[tid] = 1.0f / sqrtf(S.ss[tid] / (float)J.kdim + D.eps);
         ss_raw = false;
         csync();
+        if (J.norm_out && gain != nullptr && tg0 == 0) publish_normed_slice<WT>(D, J.x, J.kdim, J.gain, S.ss, tag_out);
         float *ssg = red + (size_t)kConsumerWarps * NP * 16;   // [tile][token] sums of squares of the new residual values
         const bool want_ss = J.epi == EPI_ADD && J.gain_out != nullptr;
         for (int q = 0; q < n_out_iter; ++q) {
@@ -919,7 +948,7 @@ static __device__ void consume_segment_bf16(const Dev &D, const Smem &S, Ring &r
             csync();
             if (tid < M) {
                 for (int tl = 0; tl < tg; ++tl) ss_share += ssg[tl * M + tid];
-                if (tg0 + p.tpg >= p.n_tiles) st_relaxed_u32(D.sspub + (size_t)blockIdx.x * M + tid, tagged(ss_share, tag_out));
+                if (tg0 + p.tpg >= p.n_tiles) st_relaxed_u32(ss_word(D, blockIdx.x, tid), tagged(ss_share, tag_out));
             }
         }
     }
@@ -981,6 +1010,7 @@ static __device__ void consume_segment_chunked(const Dev &D, const Smem &S, Ring
         csync();
         if (gain != nullptr && r0 == 0 && tid < M) S.ss[tid] = 1.0f / sqrtf(S.ss[tid] / (float)J.kdim + D.eps);
         csync();
+        if (J.norm_out && gain != nullptr && r0 == 0) publish_normed_slice<WT>(D, J.x, J.kdim, J.gain, S.ss, tag_out);
         const int outs = nr * p.tile_units * M;
         for (int i0 = 0; i0 < outs; i0 += kConsumerThreads) {
             const int i = i0 + tid;
@@ -1007,7 +1037,7 @@ static __device__ void consume_segment_chunked(const Dev &D, const Smem &S, Ring
             csync();
             if (tid < M) {
                 for (int tl = 0; tl < nr; ++tl) ss_share += ssg[tl * M + tid];
-                if (r0 + tr >= p.n_tiles) st_relaxed_u32(D.sspub + (size_t)blockIdx.x * M + tid, tagged(ss_share, tag_out));
+                if (r0 + tr >= p.n_tiles) st_relaxed_u32(ss_word(D, blockIdx.x, tid), tagged(ss_share, tag_out));
             }
         }
     }
@@ -1031,6 +1061,7 @@ __device__ void consume_segment_f32(const Dev &D, const Smem &S, Ring &ring, con
     csync();
     if (gain != nullptr && tid < M) S.ss[tid] = 1.0f / sqrtf(S.ss[tid] / (float)J.kdim + D.eps);
     csync();
+    if (J.norm_out && gain != nullptr) publish_normed_slice<float>(D, J.x, J.kdim, J.gain, S.ss, tag_out);
     if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
     for (int tg0 = 0; tg0 < p.n_tiles; tg0 += p.tpg) {
         const int tg = min(p.tpg, p.n_tiles - tg0);
@@ -1109,63 +1140,60 @@ __device__ __forceinline__ void mma16816_free(float (&c)[4], unsigned a0, unsign
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Stages the whole tagged input of job J (at most eight rows) as {hi01, hi23, lo01, lo23} words, NB 16-byte loads per
-// thread in flight.  With want_ss the CTAs' shares of the rows' sums of squares travel in the same batch and are left,
-// tags stripped, in S.sspart as [CTA][row].  Ends with a barrier of the consumer warps.
+// Staging of the whole tagged input x[M][kdim] of a job (at most eight rows) as {hi01, hi23, lo01, lo23} words, NB
+// 16-byte loads per thread in flight.  The loads of the first batch are issued as soon as the stage begins (plan,
+// issue); the caller then does everything that does not need them, and finish() waits for the words, stores them and
+// works through the remaining batches.  With want_ss the CTAs' shares of the rows' sums of squares travel in the first
+// batch and are left, tags stripped, in S.sspart as [row][CTA].  finish() ends with a barrier of the consumer warps.
 template <int NB>
-static __device__ __forceinline__ void stage_small(const Dev &D, const Smem &S, const GemvJob &J, uint32_t tag, bool want_ss) {
-    const int M = D.M, tid = threadIdx.x, kdim = J.kdim;
-    const int v4 = kdim >> 2, total = M * v4, pitch = kdim * 4 + 16;
-    const uint32_t inv = 0xFFFFFFFFu / (uint32_t)v4 + 1u;       // i / v4 == umulhi(i, inv) for i, v4 < 2^16
-    const float *x = J.x;
-    const bool dead_rows = S.ctl->any_dead != 0;
-    const int n_sh = want_ss ? ((int)gridDim.x * M) >> 2 : 0;   // 16-byte words of shares (a multiple of four words)
-    for (int i0 = 0; i0 < total; i0 += kConsumerThreads * NB) {
-        const float *src[NB];      // nullptr: nothing to fetch (past the end, or a finished sequence's row)
-        int dst[NB];               // byte offset in the staging area, -1: past the end
+struct ActLoads {
+    int src[NB];               // element offset into x, -1: nothing to fetch (past the end, or a finished sequence's row)
+    int dst[NB];               // byte offset in the staging area, -1: past the end
+    int sh[2];                 // the shares: 16-byte words tid and tid + 224 of [row][CTA] (at most 1536 floats), -1: none
+    uint4 w[NB], sw[2];
+
+    __device__ __forceinline__ void plan(const Dev &D, const Smem &S, int kdim, int i0, bool want_ss) {
+        const int M = D.M, tid = threadIdx.x;
+        const int v4 = kdim >> 2, total = M * v4, pitch = kdim * 4 + 16;
+        const uint32_t inv = 0xFFFFFFFFu / (uint32_t)v4 + 1u;       // i / v4 == umulhi(i, inv) for i, v4 < 2^16
+        const bool dead_rows = S.ctl->any_dead != 0;
 #pragma unroll
         for (int u = 0; u < NB; ++u) {
             const int i = i0 + u * kConsumerThreads + tid;
-            src[u] = nullptr; dst[u] = -1;
+            src[u] = -1; dst[u] = -1;
             if (i < total) {
                 const int m = (int)__umulhi((uint32_t)i, inv), c4 = i - m * v4;
                 dst[u] = m * pitch + (c4 << 4);
-                if (!(dead_rows && S.ctl->row_dead[m])) src[u] = x + (size_t)m * kdim + (c4 << 2);
+                if (!(dead_rows && S.ctl->row_dead[m])) src[u] = m * kdim + (c4 << 2);
             }
         }
-        // the shares: 16-byte words tid and tid + 224 of [CTA][row] (at most 1536 floats)
-        const float *sh_src[2];
+        const int n_sh = (want_ss && i0 == 0) ? ((int)gridDim.x * M) >> 2 : 0;
 #pragma unroll
-        for (int q = 0; q < 2; ++q) sh_src[q] = (i0 == 0 && tid + q * kConsumerThreads < n_sh) ? D.sspub + 4 * (tid + q * kConsumerThreads) : nullptr;
-        uint4 w[NB], sw[2];
-        // the whole batch is requested at once; where a word has not arrived, the thread waits for the first such word
-        // alone and then requests the batch again
-        for (;;) {
-            const float *stale = nullptr;
-#pragma unroll
-            for (int u = 0; u < NB; ++u) w[u] = src[u] != nullptr ? ld_relaxed_u4(src[u]) : make_uint4(tag, tag, tag, tag);
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                sw[q] = make_uint4(tag, tag, tag, tag);
-                if (sh_src[q] != nullptr) {
-                    sw[q] = ld_relaxed_u4(sh_src[q]);
-                    if (dead_rows) {      // nobody publishes the shares of a finished sequence's rows
-                        const int r0 = (4 * (tid + q * kConsumerThreads)) % M;
-                        if (S.ctl->row_dead[r0]) sw[q].x = tag;
-                        if (S.ctl->row_dead[(r0 + 1) % M]) sw[q].y = tag;
-                        if (S.ctl->row_dead[(r0 + 2) % M]) sw[q].z = tag;
-                        if (S.ctl->row_dead[(r0 + 3) % M]) sw[q].w = tag;
-                    }
-                }
-                if (!tags_ok(sw[q], tag)) stale = sh_src[q];
-            }
-#pragma unroll
-            for (int u = NB - 1; u >= 0; --u)
-                if (!tags_ok(w[u], tag)) stale = src[u];
-            if (stale == nullptr) break;
-            poll_u4(D, S.ctl, stale, tag);
-            if (S.ctl->dead) break;
+        for (int q = 0; q < 2; ++q) {
+            const int wi = tid + q * kConsumerThreads;
+            sh[q] = wi < n_sh ? wi : -1;
+            // nobody publishes the shares of a finished sequence's rows ([row][CTA]: a word lies in one row)
+            if (dead_rows && wi < n_sh && S.ctl->row_dead[(4 * wi) / (int)gridDim.x]) sh[q] = -1;
         }
+    }
+    __device__ __forceinline__ void issue(const Dev &D, const float *x, uint32_t tag) {
+#pragma unroll
+        for (int u = 0; u < NB; ++u) w[u] = src[u] >= 0 ? ld_relaxed_u4(x + src[u]) : make_uint4(tag, tag, tag, tag);
+#pragma unroll
+        for (int q = 0; q < 2; ++q) sw[q] = sh[q] >= 0 ? ld_relaxed_u4(D.sspub + 4 * sh[q]) : make_uint4(tag, tag, tag, tag);
+    }
+    // the first word that does not carry the tag yet (nullptr: all have arrived)
+    __device__ __forceinline__ const float *stale(const Dev &D, const float *x, uint32_t tag) const {
+        const float *st = nullptr;
+#pragma unroll
+        for (int q = 1; q >= 0; --q)
+            if (!tags_ok(sw[q], tag)) st = D.sspub + 4 * sh[q];
+#pragma unroll
+        for (int u = NB - 1; u >= 0; --u)
+            if (!tags_ok(w[u], tag)) st = x + src[u];
+        return st;
+    }
+    __device__ __forceinline__ void store(const Smem &S) const {
 #pragma unroll
         for (int u = 0; u < NB; ++u) {
             if (dst[u] >= 0) {
@@ -1179,134 +1207,100 @@ static __device__ __forceinline__ void stage_small(const Dev &D, const Smem &S, 
         }
 #pragma unroll
         for (int q = 0; q < 2; ++q)
-            if (sh_src[q] != nullptr)
-                *reinterpret_cast<float4 *>(S.sspart + 4 * (tid + q * kConsumerThreads)) =
-                    make_float4(untag(sw[q].x), untag(sw[q].y), untag(sw[q].z), untag(sw[q].w));
+            if (sh[q] >= 0)
+                *reinterpret_cast<float4 *>(S.sspart + 4 * sh[q]) = make_float4(untag(sw[q].x), untag(sw[q].y), untag(sw[q].z), untag(sw[q].w));
     }
-    csync();
-}
-
-// Products of the warp's column blocks (32 columns each: kb = warp, warp + 7, ...) for TL tiles, KU blocks per round
-// with accumulators of their own: sixteen independent products per round whatever the shape.
-template <int TL, int KU>
-__device__ __forceinline__ void mma_small(float (&c)[kSmallTiles][4], const uint32_t (&row_a)[kSmallTiles], const uint32_t (&row_b)[kSmallTiles],
-                                          uint32_t x_addr, bool has_x, int n_kb) {
-    const int warp = threadIdx.x >> 5;
-    float acc[KU][TL][2][4];
-#pragma unroll
-    for (int ku = 0; ku < KU; ++ku)
-#pragma unroll
-        for (int tl = 0; tl < TL; ++tl)
-#pragma unroll
-            for (int q = 0; q < 4; ++q) acc[ku][tl][0][q] = acc[ku][tl][1][q] = 0.f;
-    for (int kb0 = warp; kb0 < n_kb; kb0 += kConsumerWarps * KU) {
-        uint4 xa[KU], xb[KU], wa[KU][TL], wb[KU][TL];
-#pragma unroll
-        for (int ku = 0; ku < KU; ++ku) {
-            const int kb = kb0 + ku * kConsumerWarps;
-            const bool ok = kb < n_kb;
-            xa[ku] = xb[ku] = make_uint4(0u, 0u, 0u, 0u);
-            if (ok && has_x) {
-                xa[ku] = lds_u4(x_addr + (uint32_t)kb * 128u);
-                xb[ku] = lds_u4(x_addr + (uint32_t)kb * 128u + 16u);
+    // Where a word has not arrived, the thread waits for the first such word alone and then requests the batch again.
+    __device__ __forceinline__ void finish(const Dev &D, const Smem &S, const float *x, int kdim, uint32_t tag) {
+        const int total = D.M * (kdim >> 2);
+        for (int i0 = 0;;) {
+            for (;;) {
+                const float *st = stale(D, x, tag);
+                if (st == nullptr) break;
+                poll_u4(D, S.ctl, st, tag);
+                if (S.ctl->dead) break;
+                issue(D, x, tag);
             }
-#pragma unroll
-            for (int tl = 0; tl < TL; ++tl) {
-                wa[ku][tl] = wb[ku][tl] = make_uint4(0u, 0u, 0u, 0u);
-                if (ok) {
-                    wa[ku][tl] = lds_u4(row_a[tl] + (uint32_t)kb * 64u);
-                    wb[ku][tl] = lds_u4(row_b[tl] + (uint32_t)kb * 64u);
-                }
-            }
+            store(S);
+            i0 += kConsumerThreads * NB;
+            if (i0 >= total) break;
+            plan(D, S, kdim, i0, false);
+            issue(D, x, tag);
         }
-        // products of one accumulator are issued as far apart as the round allows
-#pragma unroll
-        for (int ku = 0; ku < KU; ++ku)
-#pragma unroll
-            for (int tl = 0; tl < TL; ++tl) mma16816_free(acc[ku][tl][0], wa[ku][tl].x, wb[ku][tl].x, wa[ku][tl].y, wb[ku][tl].y, xa[ku].x, xa[ku].y);
-#pragma unroll
-        for (int ku = 0; ku < KU; ++ku)
-#pragma unroll
-            for (int tl = 0; tl < TL; ++tl) mma16816_free(acc[ku][tl][1], wa[ku][tl].x, wb[ku][tl].x, wa[ku][tl].y, wb[ku][tl].y, xa[ku].z, xa[ku].w);
-#pragma unroll
-        for (int ku = 0; ku < KU; ++ku)
-#pragma unroll
-            for (int tl = 0; tl < TL; ++tl) mma16816_free(acc[ku][tl][0], wa[ku][tl].z, wb[ku][tl].z, wa[ku][tl].w, wb[ku][tl].w, xb[ku].x, xb[ku].y);
-#pragma unroll
-        for (int ku = 0; ku < KU; ++ku)
-#pragma unroll
-            for (int tl = 0; tl < TL; ++tl) mma16816_free(acc[ku][tl][1], wa[ku][tl].z, wb[ku][tl].z, wa[ku][tl].w, wb[ku][tl].w, xb[ku].z, xb[ku].w);
+        csync();
     }
-#pragma unroll
-    for (int tl = 0; tl < kSmallTiles; ++tl)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            float v = 0.f;
-            if (tl < TL) {
-#pragma unroll
-                for (int ku = 0; ku < KU; ++ku) v += acc[ku][tl][0][q] + acc[ku][tl][1][q];
-            }
-            c[tl][q] = v;
-        }
-}
+};
 
-// The consumer of produce_segment for at most eight token rows.  Two barriers per tile group: after the staging of
-// the activations (once per job), and after every warp has parked its partial products.  Between them warp w
-// multiplies every tile of the group over the column blocks w, w + 7, ..., and (w < M) adds up the sums of squares of
-// token row w; after them warp w finishes the outputs of token row w (unit = lane), so the row's share of the new
+constexpr int kSmallLoads = 6;   // 16-byte loads of activations a thread keeps in flight on this path
+
+// The consumer of produce_segment for at most eight token rows.  ONE code path serves every shape (the code of a stage
+// runs about once per stage, so what counts is how much of it the layers share: variants per shape would stream
+// through the instruction cache).  Two barriers per tile group: after the staging of the activations (once per job),
+// and after every warp has parked its partial products.  Between them warp w multiplies every tile of the group (at
+// most four, accumulators in registers) over the column blocks w, w + 7, ... and (w < M) adds up the sums of squares
+// of token row w; after them warp w finishes the outputs of token row w (unit = lane), so the row's share of the new
 // sum of squares is a shuffle reduction and no further barrier is needed.
+// J0, R: the job's entry in the table (layer 0, or the tail when layer < 0) and this CTA's plan record, both in shared
+// memory: a field is read when it is needed.
 template <typename WT>
-static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
+static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J0, int layer, const SegRec &R, uint32_t serial,
+                                     bool norm_out) {
+    static_assert(kConsumerWarps == 7, "the sum of the warps' partial products is written out for seven warps");
+    const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int kdim = J0.kdim, pitch = kdim * 4 + 16, n_kb = kdim >> 5;
+    const int lay = max(layer, 0);
+    const float *x = J0.x;
+    const bool normed = J0.gain != nullptr;
+    const uint32_t tag_in = tag_of(serial, TagRef{J0.in.wps, J0.in.j + lay * J0.in_jinc});
+    // the activations are requested before anything else: their round trip through the L2 is the longest wait of the stage
+    ActLoads<kSmallLoads> A;
+    A.plan(D, S, kdim, 0, normed);
+    A.issue(D, x, tag_in);
     const SegPlan p = R.p;
     const int lo = R.lo, hi = R.hi;
-    const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const int kdim = J.kdim, pitch = kdim * 4 + 16;
-    const uint32_t tag_in = tag_of(serial, J.in), tag_out = tag_of(serial, J.outt);
-    const bool normed = J.gain != nullptr;
-    const bool want_ss = J.epi == EPI_ADD && J.gain_out != nullptr;
+    const int epi = J0.epi, out_ld = J0.out_ld;
+    const bool out_plain = J0.out_plain != 0;
+    float *const out = J0.out, *const hmaster = J0.hm;
+    const uint32_t tag_out = tag_of(serial, TagRef{J0.outt.wps, J0.outt.j + lay * J0.out_jinc});
+    // the gain that the published copy of the residual stream carries: that of the RMSNorm which reads it next
+    const WT *gain_out = reinterpret_cast<const WT *>(J0.gain_out);
+    if (gain_out != nullptr) {
+        if (layer > 0) gain_out = reinterpret_cast<const WT *>(reinterpret_cast<const char *>(gain_out) + S.tab->layer_bytes * layer);
+        if (layer >= 0 && J0.gain_out_step != 0)
+            gain_out = layer == D.L - 1 ? reinterpret_cast<const WT *>(S.tab->gain_last)
+                                        : reinterpret_cast<const WT *>(reinterpret_cast<const char *>(gain_out) + J0.gain_out_step);
+    }
+    const bool want_ss = epi == EPI_ADD && gain_out != nullptr;
     const int tu_shift = p.tu_shift, tu_mask = p.tile_units - 1;
+    // tiles of at most eight rows: rows 8..15 of the products are never used and not read
+    const bool lower = p.tile_rows <= 8 || (epi != EPI_GATEUP && p.n_tiles == 1 && hi - lo <= 8);
     // EPI_ADD: the residual stream's old values and the gains of the published copy for the first group, fetched while
     // the inputs are on their way (token row = warp, unit = lane and lane + 32)
     float hpre[2] = {0.f, 0.f}, gpre[2] = {1.f, 1.f};
-    if (J.epi == EPI_ADD && warp < M) {
+    if (epi == EPI_ADD && warp < M) {
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             const int u = lo + lane + 32 * q;
             if (u < hi && lane + 32 * q < p.tpg * p.tile_units) {
-                hpre[q] = __ldcg(J.hm + (size_t)warp * J.out_ld + u);
-                if (J.gain_out != nullptr) gpre[q] = to_f(reinterpret_cast<const WT *>(J.gain_out)[u]);
-            }
-        }
-    }
-    if (M * (kdim >> 2) <= 6 * kConsumerThreads) stage_small<6>(D, S, J, tag_in, normed);
-    else stage_small<12>(D, S, J, tag_in, normed);
-    if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
-    // 1 / rms of token row `warp` (and of row warp + 7): the shares are added in a fixed order
-    float inv_rms[2] = {1.f, 1.f};
-    if (normed) {
-        const int G = (int)gridDim.x;
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const int m = warp + q * kConsumerWarps;
-            if (m < M) {
-                float sum = 0.f;
-                for (int c = lane; c < G; c += 32) sum += S.sspart[c * M + m];
-                sum = warp_sum(sum);
-                inv_rms[q] = S.ctl->row_dead[m] ? 1.f : 1.0f / sqrtf(sum / (float)kdim + D.eps);
+                hpre[q] = __ldcg(hmaster + (size_t)warp * out_ld + u);
+                if (gain_out != nullptr) gpre[q] = to_f(gain_out[u]);
             }
         }
     }
     float *red = reinterpret_cast<float *>(S.acts + M * pitch);      // [warp][tile of the group: p.tpg][token 8][row 16]
-    float ss_acc[2] = {0.f, 0.f};
+    float ss_acc[2] = {0.f, 0.f}, inv_rms[2] = {1.f, 1.f};
     const uint32_t x_addr = smem_u32(S.acts) + (uint32_t)(min(g, M - 1) * pitch) + (uint32_t)t * 32u;
+    const bool has_x = g < M;
     for (int tg0 = 0; tg0 < p.n_tiles; tg0 += p.tpg) {
         const int tg = min(p.tpg, p.n_tiles - tg0), n_items = tg * p.ipt;
         const uint32_t pos0 = ring.pos;
-        // every warp reads every tile of the group: lane i waits for item i
+        // every warp reads every tile of the group: lane i waits for item i (and will free it)
+        uint32_t my_empty = 0u;
         if (lane < n_items) {
             Ring r;
             r.pos = ring_add(S, pos0, lane);
             ring_wait(D, S, r);
+            my_empty = S.empty0 + 8u * ring_slot(S, r.pos);
         }
         __syncwarp();
         uint32_t row_a[kSmallTiles], row_b[kSmallTiles];
@@ -1316,28 +1310,76 @@ static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, co
             row_a[tl] = tile_row_addr(S, p, pos_tile, g) + (uint32_t)t * 16u;
             row_b[tl] = tile_row_addr(S, p, pos_tile, g + 8) + (uint32_t)t * 16u;
         }
-        float c[kSmallTiles][4];
-        if (tg == 1) mma_small<1, 4>(c, row_a, row_b, x_addr, g < M, kdim >> 5);
-        else if (tg == 2) mma_small<2, 2>(c, row_a, row_b, x_addr, g < M, kdim >> 5);
-        else mma_small<4, 1>(c, row_a, row_b, x_addr, g < M, kdim >> 5);
+        if (tg0 == 0) {
+            A.finish(D, S, x, kdim, tag_in);
+            if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
+            // 1 / rms of token row `warp` (and of row warp + 7): the shares [row][CTA] are added in a fixed order
+            if (normed) {
+                const int G4 = (int)gridDim.x >> 2;
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int m = warp + q * kConsumerWarps;
+                    if (m < M) {
+                        float sum = 0.f;
+                        for (int c4 = lane; c4 < G4; c4 += 32) {
+                            const float4 v = *reinterpret_cast<const float4 *>(S.sspart + (size_t)m * (G4 << 2) + (c4 << 2));
+                            sum += (v.x + v.y) + (v.z + v.w);
+                        }
+                        sum = warp_sum(sum);
+                        inv_rms[q] = S.ctl->row_dead[m] ? 1.f : 1.0f / sqrtf(sum / (float)kdim + D.eps);
+                        if (norm_out && lane == 0) S.ss[m] = inv_rms[q];
+                    }
+                }
+                if (norm_out) {      // the side output of the stage: this CTA's columns of the normed input (rare: once per step)
+                    csync();
+                    publish_normed_slice<WT>(D, x, kdim, J0.gain, S.ss, tag_out);
+                }
+            }
+        }
+        // products: per column block the activations once, then every tile of the group (hi and lo chains of a tile
+        // are independent, tiles are independent)
+        float acc[kSmallTiles][2][4];
+#pragma unroll
+        for (int tl = 0; tl < kSmallTiles; ++tl)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[tl][0][q] = acc[tl][1][q] = 0.f;
+        for (int kb = warp; kb < n_kb; kb += kConsumerWarps) {
+            uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = xa;
+            if (has_x) {
+                xa = lds_u4(x_addr + (uint32_t)kb * 128u);
+                xb = lds_u4(x_addr + (uint32_t)kb * 128u + 16u);
+            }
+#pragma unroll
+            for (int tl = 0; tl < kSmallTiles; ++tl) {
+                if (tl < tg) {
+                    const uint4 wa = lds_u4(row_a[tl] + (uint32_t)kb * 64u);
+                    uint4 wb = make_uint4(0u, 0u, 0u, 0u);
+                    if (!lower) wb = lds_u4(row_b[tl] + (uint32_t)kb * 64u);
+                    mma16816_free(acc[tl][0], wa.x, wb.x, wa.y, wb.y, xa.x, xa.y);
+                    mma16816_free(acc[tl][1], wa.x, wb.x, wa.y, wb.y, xa.z, xa.w);
+                    mma16816_free(acc[tl][0], wa.z, wb.z, wa.w, wb.w, xb.x, xb.y);
+                    mma16816_free(acc[tl][1], wa.z, wb.z, wa.w, wb.w, xb.z, xb.w);
+                }
+            }
+        }
         __syncwarp();
-        if (lane < n_items) mbar_arrive(S.empty0 + 8u * ring_slot(S, ring_add(S, pos0, lane)));
+        if (lane < n_items) mbar_arrive(my_empty);
         ring.pos = ring_add(S, pos0, n_items);
         if (tg0 != 0) csync();        // the previous group's partial products have been read
 #pragma unroll
         for (int tl = 0; tl < kSmallTiles; ++tl) {
             if (tl < tg) {
                 float *r = red + ((size_t)(warp * p.tpg + tl) * 8) * 16;
-                r[(2 * t) * 16 + g] = c[tl][0];
-                r[(2 * t + 1) * 16 + g] = c[tl][1];
-                r[(2 * t) * 16 + g + 8] = c[tl][2];
-                r[(2 * t + 1) * 16 + g + 8] = c[tl][3];
+                r[(2 * t) * 16 + g] = acc[tl][0][0] + acc[tl][1][0];
+                r[(2 * t + 1) * 16 + g] = acc[tl][0][1] + acc[tl][1][1];
+                r[(2 * t) * 16 + g + 8] = acc[tl][0][2] + acc[tl][1][2];
+                r[(2 * t + 1) * 16 + g + 8] = acc[tl][0][3] + acc[tl][1][3];
             }
         }
         // EPI_HEADY adds the normalised input itself: taken from the staged copy before anyone may overwrite it
         const int u_first = lo + tg0 * p.tile_units, ug = min(tg * p.tile_units, hi - u_first);
         float xin[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-        if (J.epi == EPI_HEADY) {
+        if (epi == EPI_HEADY) {
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 const int m = warp + q * kConsumerWarps;
@@ -1366,27 +1408,30 @@ static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, co
                 if (j >= ug) break;
                 const int tl = j >> tu_shift, ui = j & tu_mask, u = u_first + j;
                 const float *rr = red + ((size_t)tl * 8 + m) * 16 + ui;
-                float v = 0.f, v2 = 0.f;
+                float pv[kConsumerWarps], pv2[kConsumerWarps];
 #pragma unroll
                 for (int w2 = 0; w2 < kConsumerWarps; ++w2) {
-                    v += rr[(size_t)w2 * p.tpg * 128];
-                    if (J.epi == EPI_GATEUP) v2 += rr[(size_t)w2 * p.tpg * 128 + 8];
+                    pv[w2] = rr[(size_t)w2 * p.tpg * 128];
+                    pv2[w2] = epi == EPI_GATEUP ? rr[(size_t)w2 * p.tpg * 128 + 8] : 0.f;
                 }
+                float v = ((pv[0] + pv[1]) + (pv[2] + pv[3])) + ((pv[4] + pv[5]) + pv[6]);
+                float v2 = ((pv2[0] + pv2[1]) + (pv2[2] + pv2[3])) + ((pv2[4] + pv2[5]) + pv2[6]);
                 v *= inv; v2 *= inv;
-                float *o = J.out + (size_t)m * J.out_ld + u;
+                float *o = out + (size_t)m * out_ld + u;
                 float pub;
-                if (J.epi == EPI_STORE) pub = v;
-                else if (J.epi == EPI_GATEUP) pub = silu_f(v) * v2;
-                else if (J.epi == EPI_ADD) {
-                    float *hm = J.hm + (size_t)m * J.out_ld + u;
+                if (epi == EPI_STORE) pub = v;
+                else if (epi == EPI_GATEUP) pub = silu_f(v) * v2;
+                else if (epi == EPI_ADD) {
+                    float *hm = hmaster + (size_t)m * out_ld + u;
                     const bool pre = tg0 == 0 && q == 0;
                     const float r = (pre ? hpre[jq] : __ldcg(hm)) + v;
                     __stcg(hm, r);
                     pub = r;
-                    if (J.gain_out != nullptr) pub = r * (pre ? gpre[jq] : to_f(reinterpret_cast<const WT *>(J.gain_out)[u]));
+                    if (gain_out != nullptr) pub = r * (pre ? gpre[jq] : to_f(gain_out[u]));
                     ss_acc[q] += r * r;
-                } else pub = xin[q][jq] * inv + silu_f(v);
-                st_relaxed_u32(o, publish_word<WT>(pub, tag_out, J.out_plain != 0));
+                } else if (epi == EPI_ADDG) pub = residual_word(J0.res + (size_t)m * out_ld + u, tag_out) + v;
+                else pub = xin[q][jq] * inv + silu_f(v);
+                st_relaxed_u32(o, publish_word<WT>(pub, tag_out, out_plain));
             }
         }
     }
@@ -1396,7 +1441,7 @@ static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, co
             const int m = warp + q * kConsumerWarps;
             if (m < M) {
                 const float sh = warp_sum(ss_acc[q]);
-                if (lane == 0) st_relaxed_u32(D.sspub + (size_t)blockIdx.x * M + m, tagged(sh, tag_out));
+                if (lane == 0) st_relaxed_u32(ss_word(D, blockIdx.x, m), tagged(sh, tag_out));
             }
         }
     }
@@ -1407,7 +1452,6 @@ template <typename WT, int NTM> struct ConsumeSegment;
 template <int NTM> struct ConsumeSegment<bf16, NTM> {
     static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
         if (D.kca < J.kdim) { consume_segment_chunked<bf16>(D, S, ring, J, R, serial); return; }
-        if (NTM == 1 && small_mode<bf16>(D, J.kdim)) { consume_small<bf16>(D, S, ring, J, R, serial); return; }
         consume_segment_bf16<bf16, NTM>(D, S, ring, J, R, serial);
     }
 };
@@ -1447,10 +1491,20 @@ template <typename WT> static __device__ void plan_segments(const Dev &D, const 
 // A projection stage, seen by the producer warp (PRODUCER) or by the consumer warps.
 template <typename WT, int NTM, bool PRODUCER>
 static __device__ void gemv_stage(const Dev &D, const Smem &S, Ring &ring, const Stage &st, uint32_t serial) {
+    bool norm_out = st.norm_out != 0;      // the first job this CTA has rows of carries the stage's side output
     for (int j = 0; j < st.njobs; ++j) {
+        if (!PRODUCER && sizeof(WT) == 2 && NTM == 1 && small_mode<WT>(D, S.tab->jobs[st.job0 + j].kdim)) {
+            if (S.seg[st.job0 + j].lo < S.seg[st.job0 + j].hi) {
+                consume_small<bf16>(D, S, ring, S.tab->jobs[st.job0 + j], st.layer, S.seg[st.job0 + j], serial, norm_out);
+                norm_out = false;
+            }
+            continue;
+        }
         const SegRec R = S.seg[st.job0 + j];
         if (R.lo < R.hi) {
-            const GemvJob J = job_at(D, S, st.job0 + j, st.layer);
+            GemvJob J = job_at(D, S, st.job0 + j, st.layer);
+            J.norm_out = norm_out ? 1 : 0;
+            norm_out = false;
             if (PRODUCER) {
                 if (sizeof(WT) == 2 && D.kca < J.kdim) produce_segment_chunked<WT>(D, S, ring, J, R);
                 else produce_segment<WT>(D, S, ring, J, R);
@@ -1480,7 +1534,7 @@ template <> __device__ __forceinline__ size_t tile_off<__half>(int r, int e, int
     return (size_t)r * dh + (size_t)swz(r, e >> 3, dh * 2) * 8 + (e & 7);
 }
 
-struct AttnItem { int b, h, s, S; };
+struct AttnItem { int b, h, s, S, hd; };     // hd: decoding head (stage ST_ATTN_HEAD), else 0
 
 // number of key splits of sequence b's self-attention this step
 __device__ __forceinline__ int self_splits(const Dev &D, int len) {
@@ -1488,14 +1542,16 @@ __device__ __forceinline__ int self_splits(const Dev &D, int len) {
     return min(max((np + 3) / 4, 1), D.S_max);
 }
 // the idx-th live item of the stage (sequences that are finished have none); false when idx is past the end
-__device__ __forceinline__ bool attn_item_at(const Dev &D, const Ctl *ctl, bool cross, int idx, AttnItem &it) {
-    for (int b = 0; b < D.B; ++b) {
-        if (ctl->flags[b] & 1) continue;
-        const int S = cross ? D.S_cross : self_splits(D, ctl->len[b]);
-        const int n = D.H * S;
-        if (idx < n) { it.b = b; it.h = idx / S; it.s = idx - it.h * S; it.S = S; return true; }
-        idx -= n;
-    }
+__device__ __forceinline__ bool attn_item_at(const Dev &D, const Ctl *ctl, int kind, int idx, AttnItem &it) {
+    const int sets = kind == ST_ATTN_HEAD ? D.K : 1;      // the decoding heads attend one after the other
+    for (int hd = 0; hd < sets; ++hd)
+        for (int b = 0; b < D.B; ++b) {
+            if (ctl->flags[b] & 1) continue;
+            const int S = kind != ST_ATTN_SELF ? D.S_cross : self_splits(D, ctl->len[b]);
+            const int n = D.H * S;
+            if (idx < n) { it.b = b; it.h = idx / S; it.s = idx - it.h * S; it.S = S; it.hd = hd; return true; }
+            idx -= n;
+        }
     return false;
 }
 // pages [p_lo, p_hi) of cached keys that split s of S covers
@@ -1511,12 +1567,12 @@ template <typename WT>
 static __device__ void produce_attn(const Dev &D, const Smem &S, Ring &ring, const Stage &st) {
     typedef typename CacheT<WT>::type KVT;
     if (sizeof(KVT) != 2) return;   // the fp32 cache is read straight from global memory
-    const bool cross = st.kind == ST_ATTN_CROSS;
+    const bool cross = st.kind != ST_ATTN_SELF, headx = st.kind == ST_ATTN_HEAD;
     const int lane = threadIdx.x & 31;
-    void *pool = cross ? D.ckv_pool : D.kv_pool;
+    void *pool = headx ? D.hckv_pool : cross ? D.ckv_pool : D.kv_pool;
     const int pool_pages = cross ? D.B * D.cpages : D.n_pages;
     AttnItem it;
-    for (int idx = blockIdx.x; attn_item_at(D, S.ctl, cross, idx, it); idx += gridDim.x) {
+    for (int idx = blockIdx.x; attn_item_at(D, S.ctl, st.kind, idx, it); idx += gridDim.x) {
         int p_lo, p_hi;
         split_pages(cross ? D.C : S.ctl->len[it.b], D.P, it.s, it.S, p_lo, p_hi);
         int table = 0;      // block-table entries of 32 consecutive pages, one per lane: one round trip per 32 pages
@@ -1524,8 +1580,9 @@ static __device__ void produce_attn(const Dev &D, const Smem &S, Ring &ring, con
             const int k32 = (pg - p_lo) & 31;
             if (!cross && k32 == 0 && pg + lane < p_hi) table = __ldcg(D.block_table + (size_t)it.b * D.max_blocks + pg + lane);
             const int page = cross ? it.b * D.cpages + pg : __shfl_sync(0xffffffffu, table, k32);
-            const KVT *kt = kv_tile<KVT>(D, pool, pool_pages, st.layer, 0, page, it.h);
-            const KVT *vt = kv_tile<KVT>(D, pool, pool_pages, st.layer, 1, page, it.h);
+            const int set = headx ? it.hd : st.layer;
+            const KVT *kt = kv_tile<KVT>(D, pool, pool_pages, set, 0, page, it.h);
+            const KVT *vt = kv_tile<KVT>(D, pool, pool_pages, set, 1, page, it.h);
             uint32_t dst, bar;
             if (D.kv_one_item) {
                 ring_claim(D, S, ring, 2u * (uint32_t)D.tile_bytes, dst, bar);
@@ -1664,18 +1721,20 @@ template <typename WT, int DH>
 static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const Stage &st, const AttnItem &it, uint32_t serial) {
     typedef typename CacheT<WT>::type KVT;
     constexpr bool MMA = sizeof(KVT) == 2;
-    const bool cross = st.kind == ST_ATTN_CROSS;
+    const bool cross = st.kind != ST_ATTN_SELF, headx = st.kind == ST_ATTN_HEAD;
     const int K1 = D.K1, P = D.P, d = D.d, half = DH / 2, b = it.b, h = it.h;
+    const int kv_set = headx ? it.hd : st.layer;                       // which set of cache tiles: layer, or decoding head
+    const int part_item = (headx ? it.hd * D.B * D.H : 0) + b * D.H + h;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n = cross ? D.C : S.ctl->len[b];
     const bool win = !cross && it.s == it.S - 1;
     const bool merger = it.s == it.S - 1;
-    const float *qsrc = cross ? D.qc : D.qkv;
+    const float *qsrc = headx ? D.qh + (size_t)it.hd * D.M * d : cross ? D.qc : D.qkv;
     const int q_ld = cross ? d : 3 * d;
-    void *pool = cross ? D.ckv_pool : D.kv_pool;
+    void *pool = headx ? D.hckv_pool : cross ? D.ckv_pool : D.kv_pool;
     const int pool_pages = cross ? D.B * D.cpages : D.n_pages;
-    float *part = cross ? D.cpart : D.part;
-    float *out = cross ? D.cattn : D.attn;
+    float *part = headx ? D.hpart : cross ? D.cpart : D.part;
+    float *out = headx ? D.hattn + (size_t)it.hd * D.M * d : cross ? D.cattn : D.attn;
     const uint32_t tag_in = tag_of(serial, st.in), tag_out = tag_of(serial, st.outt), tag_part = tag_of(serial, st.part);
     AttnSmem<DH> A(S.acts, K1);
     const float qscale = D.scale * kLog2e;
@@ -1765,7 +1824,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
             if (i >= 2 * K1 * (DH / 8)) break;
             const int kv = i / (K1 * (DH / 8)), rem = i - kv * K1 * (DH / 8), j = rem / (DH / 8), c = rem - j * (DH / 8);
             const int pos = n + j, page = page_pre[qq], r = pos % P;
-            KVT *tile = kv_tile<KVT>(D, pool, pool_pages, st.layer, kv, page, h);
+            KVT *tile = kv_tile<KVT>(D, pool, pool_pages, kv_set, kv, page, h);
             KVT *dst = tile + tile_off<KVT>(r, c * 8, DH);
             if constexpr (MMA) {
                 // the window tiles hold the rows in the cache's own format: chunk c of row j goes to chunk c of row r
@@ -1871,8 +1930,8 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
             }
             for (int key = key_lo + warp; key < key_hi; key += kConsumerWarps) {
                 const int page = cross ? b * D.cpages + key / P : __ldcg(D.block_table + (size_t)b * D.max_blocks + key / P);
-                const KVT *kt = kv_tile<KVT>(D, pool, pool_pages, st.layer, 0, page, h) + (size_t)(key % P) * DH + e0;
-                const KVT *vt = kv_tile<KVT>(D, pool, pool_pages, st.layer, 1, page, h) + (size_t)(key % P) * DH + e0;
+                const KVT *kt = kv_tile<KVT>(D, pool, pool_pages, kv_set, 0, page, h) + (size_t)(key % P) * DH + e0;
+                const KVT *vt = kv_tile<KVT>(D, pool, pool_pages, kv_set, 1, page, h) + (size_t)(key % P) * DH + e0;
                 float kf[EPL], vf[EPL];
 #pragma unroll
                 for (int i = 0; i < EPL; ++i) {
@@ -1960,7 +2019,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     csync();
     if (!merger) {
         // leave the partial for the last split
-        float *pr = part + ((size_t)(b * D.H + h) * D.S_max + it.s) * K1 * (DH + 2);
+        float *pr = part + ((size_t)part_item * D.S_max + it.s) * K1 * (DH + 2);
         for (int i = tid; i < K1 * (DH + 2); i += kConsumerThreads) st_relaxed_u32(pr + i, tagged(mg[i], tag_part));
         return;
     }
@@ -1971,7 +2030,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
         for (int i = tid; i < K1 * (DH + 1); i += kConsumerThreads) {
             const int j = i / (DH + 1), e = i - j * (DH + 1);
             const int col = e < DH ? e : DH + 1;
-            const float *pb = part + ((size_t)(b * D.H + h) * D.S_max) * K1 * (DH + 2) + (size_t)j * (DH + 2);
+            const float *pb = part + ((size_t)part_item * D.S_max) * K1 * (DH + 2) + (size_t)j * (DH + 2);
             const size_t sstride = (size_t)K1 * (DH + 2);
             const int nsp = it.S - 1;
             float m = mg[j * (DH + 2) + DH], o = mg[j * (DH + 2) + col];      // running maximum, sum scaled to it
@@ -2014,9 +2073,8 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
 
 template <typename WT, int DH>
 static __device__ void consume_attn(const Dev &D, const Smem &S, Ring &ring, const Stage &st, uint32_t serial) {
-    const bool cross = st.kind == ST_ATTN_CROSS;
     AttnItem it;
-    for (int idx = blockIdx.x; attn_item_at(D, S.ctl, cross, idx, it); idx += gridDim.x)
+    for (int idx = blockIdx.x; attn_item_at(D, S.ctl, st.kind, idx, it); idx += gridDim.x)
         attn_item<WT, DH>(D, S, ring, st, it, serial);
 }
 
@@ -2294,7 +2352,7 @@ template <typename WT> __device__ void prepare_window(const Dev &D, int b, uint3
             for (int c = lane; c < nch; c += 32) ssq += scratch[j * nch + c];
             ssq = warp_sum(ssq);
             const int row = b * K1 + j;
-            for (int c = lane; c < D.grid; c += 32) st_relaxed_u32(D.sspub + (size_t)c * D.M + row, tagged(c == 0 ? ssq : 0.f, tag));
+            for (int c = lane; c < D.grid; c += 32) st_relaxed_u32(ss_word(D, c, row), tagged(c == 0 ? ssq : 0.f, tag));
         }
     }
 }
@@ -2370,6 +2428,9 @@ template <typename WT> __device__ __noinline__ void commit_stage(const Dev &D, u
                 } else {
                     const int a = min(max(s_cand[K1], 0), D.K);
                     __stcg(D.acc_len + b, a);
+                    // scripted drafts: the token at the first rejected position is the script's as well, so that a near-tie
+                    // of the backbone's two best logits cannot take the run off the script for good
+                    if (D.script != nullptr && len + a + 1 < D.script_n) s_cand[0] = D.script[(size_t)b * D.script_n + len + a + 1];
                     int n_gen = s_state[2], fin = 0, n_out = 0;
                     for (int j = 0; j <= a; ++j) {
                         const int tok = j < a ? s_win[j + 1] : s_cand[0];
@@ -2439,7 +2500,7 @@ static __device__ __forceinline__ uint32_t consume_stages(const Dev &D, const Sm
         const Stage st = stage_at(D, S, p);
         if (threadIdx.x == 0) S.ctl->trace_row = tracing ? 1 + 2 * p : 0;
         if (st.kind == ST_GEMV) gemv_stage<WT, NTM, false>(D, S, ring, st, serial);
-        else if (st.kind == ST_ATTN_SELF || st.kind == ST_ATTN_CROSS) consume_attn<WT, DH>(D, S, ring, st, serial);
+        else if (st.kind == ST_ATTN_SELF || st.kind == ST_ATTN_CROSS || st.kind == ST_ATTN_HEAD) consume_attn<WT, DH>(D, S, ring, st, serial);
         if (tracing) trace_mark(D, 2 + 2 * p);
     }
     return ring.pos;
@@ -2453,7 +2514,7 @@ static __device__ __forceinline__ uint32_t produce_stages(const Dev &D, const Sm
     for (int p = p_lo; p < p_hi; ++p) {
         const Stage st = stage_at(D, S, p);
         if (st.kind == ST_GEMV) gemv_stage<WT, NTM, true>(D, S, ring, st, 0u);
-        else if (st.kind == ST_ATTN_SELF || st.kind == ST_ATTN_CROSS) produce_attn<WT>(D, S, ring, st);
+        else if (st.kind == ST_ATTN_SELF || st.kind == ST_ATTN_CROSS || st.kind == ST_ATTN_HEAD) produce_attn<WT>(D, S, ring, st);
     }
     return ring.pos;
 }

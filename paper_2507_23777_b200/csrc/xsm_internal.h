@@ -28,12 +28,14 @@ constexpr int kSmemMax = 227 * 1024;
 // One step of Algorithm 1 is a fixed list of stages.  A stage's output is published in global memory as
 // fp32 words whose two lowest mantissa bits carry a tag (1..3, cycling with the write index of the buffer);
 // the next stage spins on the words it needs until they carry the expected tag.  No grid barrier exists.
-enum StageKind : int { ST_GEMV = 0, ST_ATTN_SELF = 1, ST_ATTN_CROSS = 2, ST_SAMPLE = 3, ST_COMMIT = 4 };
+enum StageKind : int { ST_GEMV = 0, ST_ATTN_SELF = 1, ST_ATTN_CROSS = 2, ST_SAMPLE = 3, ST_COMMIT = 4,
+                       ST_ATTN_HEAD = 5 /* cross-attention of the decoding heads (Eq. 3) */ };
 enum Epilogue : int {
     EPI_STORE = 0,    // out[m][r]  = W[r] . x[m]
     EPI_ADD = 1,      // h[m][r]   += W[r] . x[m]; out[m][r] = h[m][r]      (residual stream)
     EPI_GATEUP = 2,   // out[m][r]  = SiLU(Wgate[r] . x[m]) * (Wup[r] . x[m])
-    EPI_HEADY = 3     // out[m][r]  = x[m][r] + SiLU(W[r] . x[m])           (x = normed input)
+    EPI_HEADY = 3,    // out[m][r]  = x[m][r] + SiLU(W[r] . x[m])           (x = normed input)
+    EPI_ADDG = 4      // out[m][r]  = res[m][r] + W[r] . x[m]               (res = the published final hidden state g)
 };
 
 // Write index of a tagged buffer = serial * wps + j (serial: decoding steps since xsm_prefill; wps: writes
@@ -53,18 +55,21 @@ struct GemvJob {
     int out_plain;           // 1: `out` is published as plain tagged fp32 (logits) even in a bf16 model
     int in_jinc, out_jinc;   // a layer job: how much in.j / outt.j grow from one layer to the next
     long long gain_out_step; // a layer job: bytes from one layer's gain_out to the next layer's
+    const float *res;        // EPI_ADDG: tagged fp32 residual [M][out_ld]
+    int norm_out, pad_;      // norm_out (set per stage by the kernel): this job also publishes the CTA's columns of the normed input
 };
 
 struct Stage {
     int kind, layer, job0, njobs;
     TagRef in, outt, part;   // attention: q/k/v (or q) in, attention rows out, split partials
     int jinc;                // a layer stage: growth of the three j's per layer
+    int norm_out;            // a projection stage whose input is normed: every CTA also publishes its columns of the normed input (D.gpub)
 };
 
 // Every layer has the same eight stages and the same weight layout, so the tables describe layer 0 (the
 // weights of layer l lie l * layer_bytes further) and the tail of the step (LM head and decoding heads, their
 // output projections, verify/resample, commit).  The step kernel works from a copy in shared memory.
-constexpr int kLayerStages = 8, kMaxTailStages = 4, kLayerJobs = 6, kMaxTailJobs = 2 * kMaxDraft + 1;
+constexpr int kLayerStages = 8, kMaxTailStages = 6, kLayerJobs = 6, kMaxTailJobs = 3 * kMaxDraft + 1;
 struct Tables {
     Stage stages[kLayerStages + kMaxTailStages];
     GemvJob jobs[kLayerJobs + kMaxTailJobs];
@@ -113,6 +118,9 @@ struct Dev {
     int script_n, script_acc;
     // tagged exchange buffers
     float *hpub, *qkv, *attn, *qc, *cattn, *act, *y, *logits0, *hlogits, *part, *cpart;
+    float *qh, *hattn, *gpub, *hpart;   // cross-attention heads: queries [K][M][d], attention rows [K][M][d], final hidden state [M][d], split partials
+    void *hckv_pool;               // [K][2][B*cpages][H] tiles: keys and values of the condition under every head's own projections
+    int head_kind;
     uint32_t *candx, *header;      // [B][K1 + 1] resampled tokens and accept length; [B][4] len, flags
     uint32_t *done;                // [grid] "this CTA has finished the projections of the step"
     float *sspub;                  // [grid][M] bf16 models: each CTA's share of the sum of squares of the rows of hpub
@@ -132,7 +140,7 @@ constexpr int kHeaderWords = 4;    // per sequence: len, flags (1 finished, 2 in
 cudaError_t launch_step(const Dev &D, int dtype, int st_lo, int st_hi, int n_steps, uint32_t serial0, int grid,
                         int smem_bytes, cudaStream_t st);
 cudaError_t launch_cross_kv(const Dev &D, int dtype, const void *W /*flat weights*/, const size_t *wkc_off,
-                            const size_t *wvc_off, const void *cond, cudaStream_t st);
+                            const size_t *wvc_off, const void *cond, void *pool, int n_sets, cudaStream_t st);
 cudaError_t launch_init(const Dev &D, int dtype, uint32_t serial, cudaStream_t st);
 cudaError_t launch_embed(const Dev &D, int dtype, uint32_t serial, cudaStream_t st);
 cudaError_t launch_gather_kv(const Dev &D, int dtype, int layer, int seq, int pos0, int n, float *out_k,

@@ -31,7 +31,7 @@ cudaError_t launch_step(const Dev &D, int dtype, int st_lo, int st_hi, int n_ste
 // out[c][r] = sum_k W[r][k] * cond[b][c][k], stored as cache tiles.
 template <typename WT>
 __global__ void __launch_bounds__(256) cross_kv_kernel(const Dev D, const WT *Wall, const size_t *wkc_off,
-                                                       const size_t *wvc_off, const WT *cond) {
+                                                       const size_t *wvc_off, const WT *cond, void *pool) {
     constexpr int T = 64, KT = 16;
     __shared__ float As[KT][T + 1], Bs[KT][T + 1];
     const int z = blockIdx.z, b = z % D.B, kv = (z / D.B) % 2, layer = z / (2 * D.B);
@@ -65,19 +65,21 @@ __global__ void __launch_bounds__(256) cross_kv_kernel(const Dev D, const WT *Wa
             if (c < D.C && r < D.d) {
                 const int page = b * D.cpages + c / D.P, head = r / D.dh, e = r % D.dh;
                 typedef typename CacheT<WT>::type KVT;
-                KVT *tile = kv_tile<KVT>(D, D.ckv_pool, D.B * D.cpages, layer, kv, page, head);
+                KVT *tile = kv_tile<KVT>(D, pool, D.B * D.cpages, layer, kv, page, head);
                 tile[tile_off<KVT>(c % D.P, e, D.dh)] = from_f<KVT>(acc[i][j]);
             }
         }
 }
 
+// n_sets projections of the condition (the layers' Wkc / Wvc into the cross-attention cache, or the decoding heads'
+// own Wk / Wv into theirs); set i of the offset tables fills set i of `pool`
 cudaError_t launch_cross_kv(const Dev &D, int dtype, const void *W, const size_t *wkc_off, const size_t *wvc_off,
-                            const void *cond, cudaStream_t st) {
-    dim3 grid((D.C + 63) / 64, (D.d + 63) / 64, D.L * 2 * D.B);
+                            const void *cond, void *pool, int n_sets, cudaStream_t st) {
+    dim3 grid((D.C + 63) / 64, (D.d + 63) / 64, n_sets * 2 * D.B);
     if (dtype == 1)
-        cross_kv_kernel<bf16><<<grid, 256, 0, st>>>(D, (const bf16 *)W, wkc_off, wvc_off, (const bf16 *)cond);
+        cross_kv_kernel<bf16><<<grid, 256, 0, st>>>(D, (const bf16 *)W, wkc_off, wvc_off, (const bf16 *)cond, pool);
     else
-        cross_kv_kernel<float><<<grid, 256, 0, st>>>(D, (const float *)W, wkc_off, wvc_off, (const float *)cond);
+        cross_kv_kernel<float><<<grid, 256, 0, st>>>(D, (const float *)W, wkc_off, wvc_off, (const float *)cond, pool);
     return cudaGetLastError();
 }
 

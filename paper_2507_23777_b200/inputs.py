@@ -15,7 +15,8 @@ that ``y = W x``):
         g3[d]  Wgate[f, d] Wup[f, d] Wdown[d, f]
     gf[d]  W0[V, d]
     for each draft head i = 1..K:
-        W1[hd, d]  Wout[V, hd]          (hd == d: the block is residual)
+        W1[hd, d]  Wout[V, hd]          (head_kind 0, hd == d: the block is residual)
+        Wq[d, d] Wk[d, dc] Wv[d, dc] Wo[d, d] Wout[V, d]     (head_kind 1: cross-attention head)
 
 ``dtype`` 0 stores fp32 elements, ``dtype`` 1 stores bf16 elements (uint16 bit
 patterns, rounded to nearest-even once, here).
@@ -31,7 +32,7 @@ import numpy as np
 
 # Verification / sampling mode numbers shared by the two C interfaces.
 VERIFY_STRICT_GREEDY, VERIFY_TOPK, VERIFY_THRESHOLD = 0, 1, 2
-SAMPLE_ARGMAX, SAMPLE_TOPK_TEMPERATURE = 0, 1
+SAMPLE_ARGMAX, SAMPLE_TOPK_TEMPERATURE, SAMPLE_TREE = 0, 1, 2
 
 
 def _cfg(name, L, d, H, dh, f, C, V, K, dtype, batch, gen, sigma, out_scale,
@@ -97,8 +98,15 @@ def weight_tensors(cfg: dict):
     yield "gf", (d,), "gain"
     yield "W0", (V, d), "out"
     for i in range(1, K + 1):
-        yield f"h{i}.W1", (hd, d), "w"
-        yield f"h{i}.Wout", (V, hd), "out"
+        if cfg.get("head_kind", 0) == 1:      # cross-attention head (Eq. 3): its own q/k/v/o projections
+            yield f"h{i}.Wq", (d, d), "w"
+            yield f"h{i}.Wk", (d, dc), "w"
+            yield f"h{i}.Wv", (d, dc), "w"
+            yield f"h{i}.Wo", (d, d), "w"
+            yield f"h{i}.Wout", (V, d), "out"
+        else:
+            yield f"h{i}.W1", (hd, d), "w"
+            yield f"h{i}.Wout", (V, hd), "out"
 
 
 def weight_offsets(cfg: dict) -> dict:
