@@ -486,3 +486,52 @@ def test_a_wait_that_runs_out_ends_the_kernel_cleanly_and_prefill_recovers(P):
     got, lens, _ = ctx.generate(24)
     assert lens[0] == 24 and np.array_equal(got, want)
     ctx.xsm_destroy()
+
+
+# ---------------------------------------------------------------- cross-attention decoding heads (Eq. 3)
+
+
+@pytest.mark.parametrize("dtype,batch,phase_launch", [(0, 1, False), (1, 1, False), (1, 3, False), (0, 2, True)])
+def test_cross_attention_heads_on_the_unit_model(P, dtype, batch, phase_launch):
+    """head_kind 1: every head is a residual cross-attention layer with its own projections of the condition.  Logits of
+    the heads, committed tokens and windows against the oracle, with scripted accept lengths."""
+    cfg = gpu_cfg(dtype=dtype, n_draft=3, head_kind=1, sigma=0.15 if dtype == 0 else 0.05)
+    tol = F32_TOL if dtype == 0 else BF16_TOL
+    ls = P.LockStep(cfg, batch=batch, random_gains=True, phase_launch=phase_launch)
+    ls.begin()
+    full = []
+    for b in range(batch):
+        ref = ls.orc.new_seq(ls.cond[b], b).generate_plain([0], ls.odc, 60)
+        full.append(np.concatenate([[0], ref]))
+    rng = np.random.default_rng(1)
+    for it in range(10):
+        good = [int(rng.integers(0, 4)) for _ in range(batch)]
+        _, acc = ls.step(drafts=scripted(ls, full, rng, good), margin=1e-3 if dtype == 0 else 1e-2, **tol)
+        if ls.excused == 0:
+            assert acc == good
+    ls.compare_cache(**tol)
+    ls.close()
+
+
+def test_cross_attention_heads_at_the_width_of_configuration_2(P):
+    """Configuration 2's shape at reduced depth with cross-attention heads (257 condition latents: five pages per head
+    and attention head), top-5 acceptance and top-5 / T = 0.5 resampling."""
+    cfg = inputs.config(2, n_layers=2, head_kind=1, max_seq_len=256)
+    ls = P.LockStep(cfg, batch=1)
+    ls.begin()
+    for it in range(8):
+        drafts = planted_chain(ls, 0, it % 3)
+        ls.step(drafts=np.asarray([drafts]), **BF16_TOL)
+    assert ls.excused <= 2
+    ls.close()
+
+
+def test_cross_attention_heads_with_split_condition_keys(P):
+    """Heads of 128 and 513 condition latents (configuration 4's width at reduced depth): the condition's keys of one
+    head exceed a CTA's ring, so the heads' attention is split over CTAs and merged, as the layers' is."""
+    cfg = inputs.config(4, n_layers=1, d_ff=2048, n_draft=2, head_kind=1, max_seq_len=256)
+    ls = P.LockStep(cfg, batch=1)
+    ls.begin()
+    for _ in range(3):
+        ls.step(**BF16_TOL)
+    ls.close()
