@@ -608,6 +608,7 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
     D.script = nullptr; D.script_n = 0; D.script_acc = 0;
     // the table above is read from host memory that the next prefill rewrites
     XSM_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    XSM_CUDA(ctx, launch_init(D, c.dtype, ctx->serial, ctx->stream));      // also clears the status word
     XSM_CUDA(ctx, launch_cross_kv(D, c.dtype, ctx->weights, at<size_t>(ctx, ctx->lay.wkc_off),
                                   at<size_t>(ctx, ctx->lay.wvc_off), d_cond, D.ckv_pool, D.L, ctx->stream));
     if (c.head_kind == 1 && D.K > 0) {
@@ -615,7 +616,6 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
                                       at<size_t>(ctx, ctx->lay.hv_off), d_cond, D.hckv_pool, D.K, ctx->stream));
         ctx->launches += 1;
     }
-    XSM_CUDA(ctx, launch_init(D, c.dtype, ctx->serial, ctx->stream));
     ctx->launches += 3;
     ctx->prefilled = 1;
     const int ingest_steps = (prompt_len - 1 + D.K1 - 1) / D.K1;

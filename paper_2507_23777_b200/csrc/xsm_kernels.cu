@@ -71,14 +71,130 @@ __global__ void __launch_bounds__(256) cross_kv_kernel(const Dev D, const WT *Wa
         }
 }
 
+// ---- the same projection on the 5th-generation tensor cores (bf16 models)
+// One CTA: D[128 weight rows][64 condition latents] = W[r0.., :] * cond[b][c0.., :]^T, fp32 accumulator in tensor memory.
+// Both operands are staged by the threads, 64 columns at a time, into the canonical K-major layout without swizzle that
+// the matrix descriptors name: a core matrix is 8 rows x 16 bytes, stored contiguously (128 bytes); core matrices that
+// follow each other along K lie 128 bytes apart (leading byte offset), 8-row groups 1024 bytes apart (stride byte
+// offset).  One elected thread issues the four K = 16 products of a chunk and commits them to an mbarrier; every wait
+// is bounded; the accumulator is read back with tcgen05.ld (thread = weight row) and written to the cache tiles.
+__device__ __forceinline__ uint64_t umma_desc_kmajor(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) | ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) |
+           (1ull << 46);      // descriptor version of sm_100, no swizzle, base offset 0
+}
+// instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, both K-major, N and M of the tile
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+                 :: "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0) : "memory");
+}
+constexpr int kUmmaTileM = 128, kUmmaTileN = 64, kUmmaChunk = 64, kUmmaCols = 64;
+
+__global__ void __launch_bounds__(128) cross_kv_umma_kernel(const Dev D, const bf16 *Wall, const size_t *wk_off, const size_t *wv_off,
+                                                            const bf16 *cond, void *pool, int *status) {
+    __shared__ __align__(1024) char sa[kUmmaTileM * kUmmaChunk * 2];     // [16 row groups][8 k-chunks][8 rows][16 B]
+    __shared__ __align__(1024) char sb[kUmmaTileN * kUmmaChunk * 2];     // [ 8 row groups][8 k-chunks][8 rows][16 B]
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t tmem_slot;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int z = blockIdx.z, b = z % D.B, kv = (z / D.B) % 2, set = z / (2 * D.B);
+    const bf16 *W = Wall + (kv == 0 ? wk_off[set] : wv_off[set]);
+    const bf16 *A = cond + (size_t)b * D.C * D.dc;
+    const int c0 = blockIdx.x * kUmmaTileN, r0 = blockIdx.y * kUmmaTileM, dc = D.dc;
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_slot)), "r"(kUmmaCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        mbar_init(smem_u32(&bar), 1u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_slot, idesc = umma_idesc_bf16(kUmmaTileM, kUmmaTileN);
+    uint32_t parity = 0;
+    bool dead = false;
+    for (int k0 = 0; k0 < dc; k0 += kUmmaChunk) {
+        // stage 16 bytes (8 columns of one row) at a time; rows and columns past the end are zeros
+        for (int i = tid; i < (kUmmaTileM + kUmmaTileN) * (kUmmaChunk / 8); i += 128) {
+            const bool is_w = i < kUmmaTileM * (kUmmaChunk / 8);
+            const int j = is_w ? i : i - kUmmaTileM * (kUmmaChunk / 8);
+            const int r = j / (kUmmaChunk / 8), c = j % (kUmmaChunk / 8), k = k0 + c * 8;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (k < dc) {
+                if (is_w) { if (r0 + r < D.d) v = __ldg(reinterpret_cast<const uint4 *>(W + (size_t)(r0 + r) * dc + k)); }
+                else if (c0 + r < D.C) v = __ldg(reinterpret_cast<const uint4 *>(A + (size_t)(c0 + r) * dc + k));
+            }
+            *reinterpret_cast<uint4 *>((is_w ? sa : sb) + (r >> 3) * 1024 + c * 128 + (r & 7) * 16) = v;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic-proxy writes, read by the tensor core's proxy
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (tid == 0) {
+#pragma unroll
+            for (int ks = 0; ks < kUmmaChunk / 16; ++ks)
+                umma_bf16(tmem, umma_desc_kmajor(smem_u32(sa) + ks * 256, 128, 1024), umma_desc_kmajor(smem_u32(sb) + ks * 256, 128, 1024), idesc,
+                          (k0 > 0 || ks > 0) ? 1u : 0u);
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(smem_u32(&bar)) : "memory");
+        }
+        // the chunk's products must be done before the buffers are overwritten (bounded wait)
+        unsigned it = 0;
+        while (!mbar_try_wait(smem_u32(&bar), parity)) {
+            if (++it > kMbarSpinLimit) { dead = true; break; }
+        }
+        parity ^= 1u;
+        if (dead) { atomicExch(status, XSM_STATUS_TIMEOUT); break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    }
+    if (!dead) {
+        typedef CacheT<bf16>::type KVT;
+        const int r = r0 + tid, head = r / D.dh, e = r % D.dh;       // thread = weight row = lane of the accumulator
+        for (int n0 = 0; n0 < kUmmaTileN; n0 += 32) {
+            uint32_t v[32];
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)n0;
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,"
+                         "%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+                           "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]),
+                           "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+                           "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                         : "r"(taddr) : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (r < D.d) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const int c = c0 + n0 + j;
+                    if (c < D.C) {
+                        KVT *tile = kv_tile<KVT>(D, pool, D.B * D.cpages, set, kv, b * D.cpages + c / D.P, head);
+                        tile[tile_off<KVT>(c % D.P, e, D.dh)] = from_f<KVT>(__uint_as_float(v[j]));
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kUmmaCols) : "memory");
+}
+
 // n_sets projections of the condition (the layers' Wkc / Wvc into the cross-attention cache, or the decoding heads'
 // own Wk / Wv into theirs); set i of the offset tables fills set i of `pool`
 cudaError_t launch_cross_kv(const Dev &D, int dtype, const void *W, const size_t *wkc_off, const size_t *wvc_off,
                             const void *cond, void *pool, int n_sets, cudaStream_t st) {
     dim3 grid((D.C + 63) / 64, (D.d + 63) / 64, n_sets * 2 * D.B);
-    if (dtype == 1)
-        cross_kv_kernel<bf16><<<grid, 256, 0, st>>>(D, (const bf16 *)W, wkc_off, wvc_off, (const bf16 *)cond, pool);
-    else
+    if (dtype == 1) {
+        // a dense contraction (n_cond x d_cond x d_model per projection): tcgen05 tiles, operands 16-byte aligned rows
+        if (D.dc % 8 == 0) {
+            dim3 g2((D.C + kUmmaTileN - 1) / kUmmaTileN, (D.d + kUmmaTileM - 1) / kUmmaTileM, n_sets * 2 * D.B);
+            cross_kv_umma_kernel<<<g2, 128, 0, st>>>(D, (const bf16 *)W, wkc_off, wvc_off, (const bf16 *)cond, pool, D.status);
+        } else
+            cross_kv_kernel<bf16><<<grid, 256, 0, st>>>(D, (const bf16 *)W, wkc_off, wvc_off, (const bf16 *)cond, pool);
+    } else
         cross_kv_kernel<float><<<grid, 256, 0, st>>>(D, (const float *)W, wkc_off, wvc_off, (const float *)cond, pool);
     return cudaGetLastError();
 }
