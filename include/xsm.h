@@ -51,7 +51,8 @@ typedef enum {
  *              g2[d] Wqc[d,d] Wkc[d,d_cond] Wvc[d,d_cond] Woc[d,d]
  *              g3[d] Wgate[f,d] Wup[f,d] Wdown[d,f]
  *   gf[d] W0[V,d]
- *   per head i=1..K: W1[head_hidden,d] Wout[V,head_hidden]
+ *   per head i=1..K: W1[head_hidden,d] Wout[V,head_hidden]                        (head_kind 0)
+ *                    Wq[d,d] Wk[d,d_cond] Wv[d,d_cond] Wo[d,d] Wout[V,d]          (head_kind 1)
  * Block (Sec. 4.1): pre-norm residual, self-attention (RoPE, causal, cached),
  * cross-attention to c, gated feed-forward network; RMSNorm gains g*.
  * Requirements: n_heads*d_head == d_model, head_hidden == d_model, d_model and d_ff multiples of 128 with rows
@@ -62,7 +63,8 @@ typedef struct {
     int n_layers, d_model, n_heads, d_head, d_ff, vocab, n_cond, d_cond;
     int n_draft;        /* K; 0 = plain one-token-per-step decoding (Table 3 row A) */
     int head_hidden;
-    int head_kind;      /* 0: MLP head, logits = Wout (g + SiLU(W1 g)) (Table 3 rows B, C) */
+    int head_kind;      /* 0: MLP head, logits = Wout (g + SiLU(W1 g)) (Table 3 rows B, C);
+                           1: cross-attention head (Eq. 3), logits = Wout (g + Wo Attn(Wq g, Wk c, Wv c)) */
     int dtype;          /* 0: fp32 weights and cache; 1: bf16 weights, fp16 cache, fp32 arithmetic */
     int page_size;      /* tokens per cache page */
     int max_batch;
@@ -77,8 +79,11 @@ typedef struct {
                            2: backbone probability of the draft > delta */
     int k_accept;
     float delta;
-    int sample_mode;    /* 0: argmax; 1: softmax(top k_sample logits / temperature) */
-    int k_sample;       /* <= 64 */
+    int sample_mode;    /* 0: argmax; 1: every candidate on its own from softmax(top k_sample logits / temperature)
+                           (the Appendix's independent sampling); 2: x_{s*} as in mode 1, the K drafts as one path
+                           of the Appendix's top-k_sample probability tree over the heads (path weight = product of
+                           the tokens' softmax probabilities, paths below 1e-5 pruned) */
+    int k_sample;       /* <= 64; mode 2: <= 8 and k_sample ^ n_draft <= 4096 */
     float temperature;
     uint64_t seed;      /* Philox4x32-10 key; sequence b uses (seed_lo ^ b, seed_hi) */
 } xsm_decode_config;

@@ -30,7 +30,7 @@ struct Layout {
         scalars, hist, steps, tok_log, step_tokens, step_n_new, prompt, script;
     size_t h, rope_cs;
     size_t xchg_begin, hpub, qkv, attn, qc, cattn, act, y, logits0, hlogits, part, cpart, candx, header, done, sspub, qh, hattn, gpub,
-        hpart, xchg_end;
+        hpart, treex, xchg_end;
     size_t stage_cond, stage_kv, stage_tok, trace, ckv_pool, hckv_pool, kv_pool;
     int n_pages = 0, max_blocks = 0, cpages = 0, tok_ld = 0, n_phases = 0, n_jobs = 0;
     size_t page_bytes = 0;
@@ -104,6 +104,7 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.hattn = take(cur, 4 * M * d * nh);
     L.gpub = take(cur, 4 * M * d * (ca ? 1 : 0));
     L.hpart = take(cur, 4 * nh * part_items * K1 * (dh + 2));
+    L.treex = take(cur, 4 * B * (c.n_draft > 0 ? c.n_draft : 1) * 8 * 2);
     L.xchg_end = cur;
     L.stage_cond = take(cur, esize(c) * B * c.n_cond * c.d_cond);
     L.stage_kv = take(cur, 4 * 2 * (size_t)kKvStagePositions * d);
@@ -259,7 +260,7 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     int need = kConsumerWarps * np * 16 * 4 + 2 * 16 * M * 4;         // reduction of the projections, new residual values
     const int attn = 2 * 16 * (dh + 8) * 2 + 4 * K1 * dh * 4 + 128 * dh + (kConsumerWarps + 1) * K1 * (dh + 2) * 4;
     if (attn > need) need = attn;
-    const int samp = (((c.vocab + 3) & ~3) + 256) * 4;
+    const int samp = (((c.vocab + 3) & ~3) + 1024) * 4;      // a logits row, reduction scratch, candidates, the probability tree's tables
     if (samp > need) need = samp;
     const int emb = 512 + K1 * (c.d_model / (c.dtype == 1 ? 8 : 4)) * 4;   // commit: scalars, partial sums of the new window's rows
     if (emb > need) need = emb;
@@ -548,6 +549,7 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     D.head_kind = cfg->head_kind;
     D.qh = at<float>(ctx, L.qh); D.hattn = at<float>(ctx, L.hattn); D.gpub = at<float>(ctx, L.gpub); D.hpart = at<float>(ctx, L.hpart);
     D.hckv_pool = ctx->ws + L.hckv_pool;
+    D.treex = at<uint32_t>(ctx, L.treex);
     *out = ctx;
     return XSM_OK;
 }
@@ -559,11 +561,18 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
     const xsm_model_config &c = ctx->cfg;
     if (batch < 1 || batch > c.max_batch) return fail(ctx, XSM_ERR_INVALID_ARG, "batch must be in [1, max_batch]");
     if (prompt_len < 1 || prompt_len - 1 > c.max_seq_len) return fail(ctx, XSM_ERR_INVALID_ARG, "prompt_len out of range");
-    if (dc->verify_mode < 0 || dc->verify_mode > 2 || dc->sample_mode < 0 || dc->sample_mode > 1)
+    if (dc->verify_mode < 0 || dc->verify_mode > 2 || dc->sample_mode < 0 || dc->sample_mode > 2)
         return fail(ctx, XSM_ERR_INVALID_ARG, "unknown verify_mode or sample_mode");
     if (dc->verify_mode == 1 && dc->k_accept < 1) return fail(ctx, XSM_ERR_INVALID_ARG, "k_accept must be >= 1");
     if (dc->sample_mode == 1 && (dc->k_sample < 1 || dc->k_sample > 64 || !(dc->temperature > 0.f)))
         return fail(ctx, XSM_ERR_INVALID_ARG, "k_sample must be in [1, 64] and temperature > 0");
+    if (dc->sample_mode == 2) {
+        if (dc->k_sample < 1 || dc->k_sample > 8 || !(dc->temperature > 0.f))
+            return fail(ctx, XSM_ERR_INVALID_ARG, "probability-tree sampling: k_sample must be in [1, 8] and temperature > 0");
+        double leaves = 1.0;
+        for (int i = 0; i < c.n_draft; ++i) leaves *= dc->k_sample;
+        if (leaves > 4096.0) return fail(ctx, XSM_ERR_INVALID_ARG, "probability-tree sampling: k_sample ^ n_draft must not exceed 4096 paths");
+    }
     if ((long long)batch * ctx->lay.max_blocks > ctx->lay.n_pages)
         return fail(ctx, XSM_ERR_CAPACITY, "the page pool cannot hold `batch` sequences of max_seq_len positions");
     Dev &D = ctx->dev;

@@ -2184,13 +2184,12 @@ static __device__ bool accept_token(const Dev &D, const float *z, int x, float *
     return (int)cnt < ka;
 }
 
-static __device__ int sample_token(const Dev &D, const float *z, uint32_t r24, float *sh) {
+// the k best (logit, token) pairs of z, ranked, left in shared memory: cv[j], ci[j] (behind the reduction scratch in sh)
+static __device__ void top_candidates(const Dev &D, const float *z, int k, float *sh) {
     const int V = D.V;
     unsigned long long *shk = reinterpret_cast<unsigned long long *>(sh);   // [kConsumerWarps], 8-byte aligned
     float *cv = sh + 2 * kConsumerWarps + 2;           // candidates (value, index), up to 64
     int *ci = reinterpret_cast<int *>(cv + 64);
-    int *pick_s = ci + 64;
-    const int k = D.sample_mode == 0 ? 1 : min(max(D.k_sample, 1), min(V, 64));
     // every thread keeps the best of its own elements; after each pick only the thread that owned the winner
     // looks for its next best (among its elements ranked after the winner)
     unsigned long long mine = 0ull;
@@ -2209,6 +2208,16 @@ static __device__ int sample_token(const Dev &D, const float *z, uint32_t r24, f
             }
         }
     }
+}
+
+static __device__ int sample_token(const Dev &D, const float *z, uint32_t r24, float *sh) {
+    const int V = D.V;
+    float *cv = sh + 2 * kConsumerWarps + 2;
+    int *ci = reinterpret_cast<int *>(cv + 64);
+    int *pick_s = ci + 64;
+    const int k = D.sample_mode == 0 ? 1 : min(max(D.k_sample, 1), min(V, 64));
+    top_candidates(D, z, k, sh);
+    csync();
     if (threadIdx.x == 0) {
         int pick = ci[0];
         if (D.sample_mode != 0) {
@@ -2226,6 +2235,53 @@ static __device__ int sample_token(const Dev &D, const float *z, uint32_t r24, f
     }
     csync();
     return *pick_s;
+}
+
+// Top-K_s probability tree over the decoding heads (Appendix, Ablation of Sampling Strategies): the leaves are the
+// K_s^K paths in lexicographic order of the heads' ranked candidates, a path weighs the product of its tokens'
+// full-vocabulary probabilities, paths whose product falls below 1e-5 are pruned, and the first leaf whose cumulative
+// weight exceeds u * total is drawn (the last surviving leaf if rounding keeps the sum below; the most probable token of
+// every head if no path survives).  One warp; m, tok: [K][8] in shared memory.  Returns the leaf's index.
+static __device__ int tree_pick(int K, int ks, const double *m, double u) {
+    const int lane = threadIdx.x & 31;
+    int n_leaves = 1;
+    for (int d = 0; d < K; ++d) n_leaves *= ks;
+    auto weight = [&](int idx) -> double {
+        if (idx >= n_leaves) return 0.0;
+        double w = 1.0;
+        int div = n_leaves;
+        for (int d = 0; d < K; ++d) {
+            div /= ks;
+            const int k = idx / div;
+            idx -= k * div;
+            w *= m[d * 8 + k];
+            if (w < 1e-5) return 0.0;
+        }
+        return w;
+    };
+    double total = 0.0;
+    for (int base = 0; base < n_leaves; base += 32) total += weight(base + lane);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    if (!(total > 0.0)) return 0;
+    const double target = u * total;
+    double cum = 0.0;
+    int last = 0;
+    for (int base = 0; base < n_leaves; base += 32) {
+        const double w = weight(base + lane);
+        double c = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, c, o);
+            if (lane >= o) c += up;
+        }
+        c += cum;
+        const unsigned alive = __ballot_sync(0xffffffffu, w > 0.0), hit = __ballot_sync(0xffffffffu, w > 0.0 && c > target);
+        if (hit) return base + __ffs(hit) - 1;
+        if (alive) last = base + 31 - __clz(alive);
+        cum = __shfl_sync(0xffffffffu, c, 31);
+    }
+    return last;
 }
 
 // item (sequence b, slot): slot 0 resamples x_{s*} from the backbone row of the first rejection, slot i
@@ -2253,6 +2309,49 @@ static __device__ __noinline__ void sample_stage(const Dev &D, uint32_t serial) 
         const float *z = slot == 0 ? D.logits0 + (size_t)(b * K1 + a) * V
                                    : D.hlogits + ((size_t)(slot - 1) * D.M + b * K1 + a) * V;
         if (!(slot == 0 && a < K)) fetch_row(D, S, z, row, tag);      // slot 0: the row that rejected its draft is still staged
+        if (D.sample_mode == 2 && slot > 0) {
+            // probability tree: this head's K_s best tokens and their probabilities for the item of slot 1, which
+            // draws one path for all heads
+            const int ks = min(max(D.k_sample, 1), min(V, 8));
+            float *cv = sh + 2 * kConsumerWarps + 2;
+            int *ci = reinterpret_cast<int *>(cv + 64);
+            top_candidates(D, row, ks, sh);
+            csync();
+            const float mx = cv[0];
+            float sum = 0.f;
+            for (int v = threadIdx.x; v < V; v += kConsumerThreads) sum += expf(row[v] - mx);
+            sum = block_sum(sum, sh + 2 * kConsumerWarps + 2 + 192);
+            uint32_t *tw = D.treex + ((size_t)(b * K + slot - 1) * 8) * 2;
+            if (threadIdx.x < ks) {
+                st_relaxed_u32(tw + 2 * threadIdx.x, tagged_int(ci[threadIdx.x], tag));
+                st_relaxed_u32(tw + 2 * threadIdx.x + 1, tagged(expf(cv[threadIdx.x] - mx) / sum, tag));
+            }
+            if (slot == 1) {
+                double *m = reinterpret_cast<double *>(sh + 512);          // [K][8], 8-byte aligned (sh is 16-byte aligned)
+                int *tk = reinterpret_cast<int *>(m + kMaxDraft * 8);      // [K][8]
+                csync();
+                for (int i = threadIdx.x; i < K * ks; i += kConsumerThreads) {
+                    const int d = i / ks, j = i - d * ks;
+                    const uint32_t *src = D.treex + ((size_t)(b * K + d) * 8 + j) * 2;
+                    tk[d * 8 + j] = untag_int(poll_u32(D, S.ctl, src, tag));
+                    m[d * 8 + j] = (double)untag(poll_u32(D, S.ctl, src + 1, tag));
+                }
+                csync();
+                if (threadIdx.x < 32) {
+                    const double u = (double)rand24(D, b, __ldcg(D.step_idx + b), 1u, 0u) * (1.0 / 16777216.0);
+                    int leaf = tree_pick(K, ks, m, u);
+                    int div = 1;
+                    for (int d = 0; d < K; ++d) div *= ks;
+                    for (int d = 0; d < K; ++d) {
+                        div /= ks;
+                        const int k = leaf / div;
+                        leaf -= k * div;
+                        if (threadIdx.x == 0) st_relaxed_u32(D.candx + (size_t)b * (K1 + 1) + 1 + d, tagged_int(tk[d * 8 + k], tag));
+                    }
+                }
+            }
+            continue;
+        }
         const uint32_t r = rand24(D, b, __ldcg(D.step_idx + b), (uint32_t)slot, 0u);
         const int tok = sample_token(D, row, r, sh);
         if (threadIdx.x == 0) {

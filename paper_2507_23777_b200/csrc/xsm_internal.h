@@ -121,6 +121,7 @@ struct Dev {
     float *qh, *hattn, *gpub, *hpart;   // cross-attention heads: queries [K][M][d], attention rows [K][M][d], final hidden state [M][d], split partials
     void *hckv_pool;               // [K][2][B*cpages][H] tiles: keys and values of the condition under every head's own projections
     int head_kind;
+    uint32_t *treex;               // probability-tree sampling: [B][K][8][2] the heads' best tokens and their probabilities
     uint32_t *candx, *header;      // [B][K1 + 1] resampled tokens and accept length; [B][4] len, flags
     uint32_t *done;                // [grid] "this CTA has finished the projections of the step"
     float *sspub;                  // [grid][M] bf16 models: each CTA's share of the sum of squares of the rows of hpub

@@ -54,6 +54,36 @@ def sample_excused(z, dc, r24, margin):
     return np.min(np.abs(cdf - r24 / 2.0 ** 24)) < margin
 
 
+def tree_excused(zh, ks, r24, margin):
+    """Probability-tree sampling (sample_mode 2): could a perturbation of the heads' logits zh [K, V] by `margin` change
+    the drawn path?  Yes if the candidates of a head nearly tie, if a path's weight lies at the pruning bound, or if
+    the uniform draw lies within `margin` of an edge of the cumulative path weights."""
+    import itertools
+    K, V = zh.shape
+    ks = min(ks, V)
+    m = []
+    for d in range(K):
+        order = np.lexsort((np.arange(V), -zh[d]))
+        top = zh[d][order[:ks + 1]].astype(np.float64)
+        if np.min(-np.diff(top)) < margin:
+            return True
+        p = np.exp(zh[d].astype(np.float64) - zh[d].max())
+        m.append((p / p.sum())[order[:ks]])
+    w = []
+    for idx in itertools.product(range(ks), repeat=K):
+        wg = 1.0
+        for d, k in enumerate(idx):
+            wg *= m[d][k]
+        if abs(wg - 1e-5) < 1e-5 * 10 * margin:
+            return True
+        w.append(wg if wg >= 1e-5 else 0.0)
+    w = np.asarray(w)
+    if w.sum() <= 0:
+        return False
+    edges = np.cumsum(w) / w.sum()
+    return bool(np.min(np.abs(edges - r24 / 2.0 ** 24)) < margin)
+
+
 def assert_logits(gpu, ref, atol, rtol, what):
     """Every logit within atol + rtol |ref| (no exceptions)."""
     ok = logits_close(gpu, ref, atol, rtol)
@@ -124,11 +154,19 @@ class LockStep:
                 excused = True
             else:
                 onw = s.window()
+                tree = self.odc.sample_mode == 2
                 for slot in range(self.K + 1):
                     if gw[slot] != onw[slot]:
+                        if tree and slot >= 1:      # the drafts are one path of the tree, drawn with slot 1's number
+                            r = oracle.rand24(self.cfg["seed"], b, step_idx, 1, 0)
+                            assert tree_excused(zh[:, oa], self.odc.k_sample, r, margin), \
+                                f"tree path: gpu {gw[1:]} vs oracle {onw[1:]} (seq {b}, step {self.steps})"
+                            excused = True
+                            break
                         z = z0[oa] if slot == 0 else zh[slot - 1][oa]
                         r = oracle.rand24(self.cfg["seed"], b, step_idx, slot, 0)
-                        assert sample_excused(z, self.odc, r, margin), \
+                        one = oracle.decode_config(dict(self.cfg, sample_mode=1)) if tree else self.odc
+                        assert sample_excused(z, one, r, margin), \
                             f"slot {slot}: gpu {gw[slot]} vs oracle {onw[slot]} (seq {b}, step {self.steps})"
                         excused = True
                 assert np.array_equal(nt[b][:ga], win[1:1 + ga])

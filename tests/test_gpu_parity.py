@@ -535,3 +535,34 @@ def test_cross_attention_heads_with_split_condition_keys(P):
     for _ in range(3):
         ls.step(**BF16_TOL)
     ls.close()
+
+
+# ---------------------------------------------------------------- probability-tree sampling (Appendix)
+
+
+@pytest.mark.parametrize("dtype,K,ks", [(0, 2, 3), (1, 3, 2), (0, 4, 4)])
+def test_probability_tree_sampling_lockstep(P, dtype, K, ks):
+    """sample_mode 2: x_{s*} from the backbone's top-k at the configured temperature, the K drafts as one path of the
+    top-k_s probability tree over the heads.  Tokens against the oracle step by step (a differing path only where the
+    draw sits at an edge of the cumulative path weights or candidates nearly tie)."""
+    cfg = gpu_cfg(dtype=dtype, n_draft=K, verify_mode=1, k_accept=3, sample_mode=2, k_sample=ks, temperature=0.8, seed=4,
+                  sigma=0.3 if dtype == 0 else 0.1)
+    ls = P.LockStep(cfg, batch=2, random_gains=True)
+    ls.begin()
+    paths = set()
+    for it in range(24):
+        ls.step(margin=1e-3 if dtype == 0 else 1e-2, **(F32_TOL if dtype == 0 else BF16_TOL))
+        st = ls.ctx.xsm_debug_get_state()
+        paths.add(tuple(st["window"][0, 1:].tolist()))
+    assert ls.excused <= 4 and len(paths) >= 4
+    ls.close()
+
+
+def test_probability_tree_sampling_at_the_width_of_configuration_2(P):
+    cfg = inputs.config(2, n_layers=2, sample_mode=2, k_sample=3, max_seq_len=256)
+    ls = P.LockStep(cfg, batch=1)
+    ls.begin()
+    for _ in range(8):
+        ls.step(**BF16_TOL)
+    assert ls.excused <= 2
+    ls.close()
