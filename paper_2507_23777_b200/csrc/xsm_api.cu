@@ -3,6 +3,8 @@
 #include "../../include/xsm.h"
 #include "xsm_internal.h"
 
+#include <cuda.h>
+
 #include <limits.h>
 #include <math.h>
 #include <stdio.h>
@@ -25,7 +27,7 @@ thread_local std::string g_create_error;
 
 struct Layout {
     size_t total = 0;
-    size_t phases, jobs, wkc_off, wvc_off, hk_off, hv_off;
+    size_t phases, jobs, wkc_off, wvc_off, hk_off, hv_off, tmaps;
     size_t len, window, cand, acc_len, finished, n_gen, n_blocks, ingest_left, step_idx, block_table, free_stack,
         scalars, hist, steps, tok_log, step_tokens, step_n_new, prompt, script;
     size_t h, rope_cs;
@@ -59,6 +61,7 @@ bool make_layout(const xsm_model_config &c, size_t workspace_bytes, Layout &L) {
     L.jobs = take(cur, 256);
     L.wkc_off = take(cur, sizeof(size_t) * c.n_layers);
     L.wvc_off = take(cur, sizeof(size_t) * c.n_layers);
+    L.tmaps = take(cur, 128 * 2 * (size_t)(kLayerJobs + kMaxTailJobs));      // two tensor maps per job
     L.hk_off = take(cur, sizeof(size_t) * (c.n_draft + 1));
     L.hv_off = take(cur, sizeof(size_t) * (c.n_draft + 1));
     L.len = take(cur, 4 * B);
@@ -223,7 +226,9 @@ struct xsm_ctx {
     uint64_t launches;
     std::string err;
     Tables h_tab;
+    std::vector<CUtensorMap> h_tmaps;   // tcgen05 path: host copies of the jobs' tensor maps (uploaded by xsm_prefill)
     int n_stages;             // stages of one decoding step
+    void *encode_tiled;       // cuTensorMapEncodeTiled of the driver (null: the tcgen05 path is not used)
     int *pinned;              // [4] n_active, status
     cudaEvent_t ev0, ev1;
     double last_wall_ms;
@@ -250,8 +255,36 @@ const void *wptr(const xsm_ctx *ctx, size_t elem_off) { return ctx->weights + el
 // Shared memory of the step kernel for a batch of `batch` sequences: header, ring slots, activation area
 // (also the scratch of attention, verification and the cross-warp reduction), sums of squares.
 // Returns nullptr or the reason why the shape cannot run.
+// may the projections of this batch run on the tcgen05 path?
+bool umma_shape(const xsm_model_config &c, int batch) {
+    const int M = batch * (c.n_draft + 1);
+    return c.dtype == 1 && M > 8 && M <= 128 && c.d_model % kUmmaK == 0 && c.d_ff % kUmmaK == 0;
+}
+
 const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_bytes) {
     const int K1 = c.n_draft + 1, M = batch * K1, dh = c.d_head;
+    if (D.umma) {
+        // tcgen05 path: the activation area holds two buffers of two planes (hi, lo) of 128 token rows x 64 columns; the
+        // other users of the area (attention, verification, commit) fit inside
+        const int tail = (kMaxTokens + 1536) * 4;
+        const int avail = kSmemMax - kSmemHeader - kSmemTables - kSmemPlans - tail;
+        int need = 2 * 16 * (dh + 8) * 2 + 4 * K1 * dh * 4 + 128 * dh + (kConsumerWarps + 1) * K1 * (dh + 2) * 4;
+        const int samp = (((c.vocab + 3) & ~3) + 1024) * 4;
+        if (samp > need) need = samp;
+        const int emb = 512 + K1 * (c.d_model / 8) * 4;
+        if (emb > need) need = emb;
+        int acts = kUmmaActsBytes > need ? kUmmaActsBytes : (need + 1023) / 1024 * 1024;
+        int slots = (avail - acts) / kSlotBytes;
+        if (slots > kMaxSlots) slots = kMaxSlots;
+        if (slots < kMinSlots) return "the shape needs more shared memory than one CTA has";
+        D.n_slots = slots;
+        D.acts_bytes = acts;
+        D.kca = c.d_model > c.d_ff ? c.d_model : c.d_ff;
+        D.tile_bytes = c.page_size * dh * 2;
+        D.kv_one_item = 2 * D.tile_bytes <= kSlotBytes ? 1 : 0;
+        smem_bytes = kSmemHeader + kSmemTables + kSmemPlans + slots * kSlotBytes + acts + tail;
+        return nullptr;
+    }
     const int kmax = c.d_model > c.d_ff ? c.d_model : c.d_ff;
     const int tail = (kMaxTokens + 1536) * 4;                        // sums of squares and their partials
     const int avail = kSmemMax - kSmemHeader - kSmemTables - kSmemPlans - tail;
@@ -290,6 +323,22 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
     D.kv_one_item = 2 * D.tile_bytes <= kSlotBytes ? 1 : 0;
     smem_bytes = kSmemHeader + kSmemTables + kSmemPlans + slots * kSlotBytes + acts + tail;
     return nullptr;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor map of a bf16 weight matrix [layers][rows][kdim] (rows of kdim elements, layers layer_bytes apart): boxes of 64
+// columns x 8 rows of one layer, 128-byte swizzle (the layout the tcgen05 matrix descriptors of the step kernel name).
+bool encode_weight_map(xsm_ctx *ctx, CUtensorMap *out, const void *W, int rows, int kdim, int layers, long long layer_bytes) {
+    if (!ctx->encode_tiled || !W) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)kdim, (cuuint64_t)rows, (cuuint64_t)(layers > 0 ? layers : 1)};
+    cuuint64_t strides[2] = {(cuuint64_t)kdim * 2, (cuuint64_t)(layers > 1 ? layer_bytes : (long long)rows * kdim * 2)};
+    cuuint32_t box[3] = {(cuuint32_t)kUmmaK, 8, 1}, estr[3] = {1, 1, 1};
+    return ((EncodeTiledFn)ctx->encode_tiled)(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(W), dims, strides, box, estr,
+                                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // stage and job tables for the current batch: the eight stages of layer 0, then the tail of the step
@@ -384,6 +433,26 @@ void build_tables(xsm_ctx *ctx) {
     T.n_tail_stages = n_stages - kLayerStages;
     T.n_tail_jobs = n_jobs - kLayerJobs;
     ctx->n_stages = kLayerStages * L + T.n_tail_stages;
+    if (ctx->dev.umma) {
+        // tcgen05 path: the weights come by TMA; one tensor map per matrix (all layers of a layer job in one map)
+        ctx->h_tmaps.assign(2 * (size_t)n_jobs, CUtensorMap{});
+        char *d_maps = ctx->ws + ctx->lay.tmaps;
+        bool ok = true;
+        for (int i = 0; i < n_jobs && ok; ++i) {
+            GemvJob &j = T.jobs[i];
+            const int layers = i < kLayerJobs ? L : 1;
+            ok = encode_weight_map(ctx, &ctx->h_tmaps[2 * i], j.W, j.rows, j.kdim, layers, T.layer_bytes);
+            j.tmap = d_maps + 128 * (2 * (size_t)i);
+            if (ok && j.W2 != nullptr) {
+                ok = encode_weight_map(ctx, &ctx->h_tmaps[2 * i + 1], j.W2, j.rows, j.kdim, layers, T.layer_bytes);
+                j.tmap2 = d_maps + 128 * (2 * (size_t)i + 1);
+            }
+        }
+        if (!ok) {        // no tensor maps: the projections take the mma.sync path
+            ctx->dev.umma = 0;
+            for (int i = 0; i < n_jobs; ++i) T.jobs[i].tmap = T.jobs[i].tmap2 = nullptr;
+        }
+    }
 }
 
 xsm_status check_device_status(xsm_ctx *ctx) {
@@ -487,6 +556,16 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     if (grid > kSizingGrid) grid = kSizingGrid;
     ctx->grid = grid;
     if ((e = cudaHostAlloc((void **)&ctx->pinned, 64, cudaHostAllocDefault)) != cudaSuccess) return bail(e, "cudaHostAlloc");
+    {   // the driver's tensor-map encoder, for the weights of the tcgen05 projections (absent: those take the mma.sync path)
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        ctx->encode_tiled = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            ctx->encode_tiled = fn;
+        else
+            (void)cudaGetLastError();
+    }
     if ((e = cudaEventCreate(&ctx->ev0)) != cudaSuccess) return bail(e, "cudaEventCreate");
     if ((e = cudaEventCreate(&ctx->ev1)) != cudaSuccess) return bail(e, "cudaEventCreate");
 
@@ -577,6 +656,7 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
         return fail(ctx, XSM_ERR_CAPACITY, "the page pool cannot hold `batch` sequences of max_seq_len positions");
     Dev &D = ctx->dev;
     int smem_bytes = 0;
+    D.umma = (umma_shape(c, batch) && ctx->encode_tiled != nullptr) ? 1 : 0;
     if (const char *m = plan_smem(c, batch, D, smem_bytes)) return fail(ctx, XSM_ERR_CAPACITY, m);
     ctx->smem_bytes = smem_bytes;
     {   // the step kernel instance for this batch must fit one CTA per multiprocessor
@@ -604,7 +684,15 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
         if (s_cross < 1) s_cross = 1;
     }
     D.S_cross = s_cross;
+    D.B = batch; D.M = batch * D.K1;
     build_tables(ctx);
+    if (!D.umma && umma_shape(c, batch)) {      // the tensor maps could not be made: plan the shared memory of the mma.sync path
+        if (const char *m = plan_smem(c, batch, D, smem_bytes)) return fail(ctx, XSM_ERR_CAPACITY, m);
+        ctx->smem_bytes = smem_bytes;
+    }
+    if (D.umma)
+        XSM_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->lay.tmaps, ctx->h_tmaps.data(), sizeof(CUtensorMap) * ctx->h_tmaps.size(),
+                                      cudaMemcpyHostToDevice, ctx->stream));
     D.n_stages = ctx->n_stages;
     XSM_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->lay.phases, &ctx->h_tab, sizeof(Tables), cudaMemcpyHostToDevice, ctx->stream));
     if ((const void *)d_prompt != (const void *)D.prompt)

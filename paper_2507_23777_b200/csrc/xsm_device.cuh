@@ -227,10 +227,13 @@ template <typename WT> __device__ __forceinline__ float read_word(uint32_t w) {
 // Per-CTA control block in shared memory (after the barriers).
 struct Ctl {
     volatile int dead;          // a wait ran out somewhere: stop waiting on global memory
+    volatile int dead_allowance;   // tries that the barrier waits of a dead CTA may still spend, all together
     int go;                     // written by the consumers before they release the producer for a step
     int trace_row;              // row of the timeline that the running stage fills when its inputs are in (0: off)
     int any_dead;               // some sequence of the batch has finished: row_dead has entries set
     volatile unsigned char landed[16];   // attention: parity of the latest fill of each ring slot that is known to have landed
+    uint32_t tmem;              // tcgen05 path: base address of the CTA's accumulator columns in tensor memory
+    volatile uint32_t umma_chunks, umma_tiles;   // tcgen05 path: column blocks and tiles multiplied since the launch (phases of abar, dbar)
     int len[kMaxBatch];
     int flags[kMaxBatch];       // 1 finished, 2 ingesting
     unsigned char row_dead[kMaxTokens];   // token rows of finished sequences (not fetched, read as zeros)
@@ -238,6 +241,8 @@ struct Ctl {
 
 struct Smem {
     uint32_t full0, empty0, go_bar;   // shared-space addresses of full[0], empty[0], go
+    uint32_t abar0, dbar, sbar0;      // tcgen05 path: "products that read activation buffer i are done" (two barriers), "the tile's accumulator is
+                                      // complete", "activation buffer i is staged" (two barriers, one arrival per staging warp)
     Ctl *ctl;
     const Tables *tab;                // shared-memory copy of the stage and job tables
     struct SegRec *seg;               // per job: this CTA's rows and their tiling
@@ -254,7 +259,10 @@ __device__ __forceinline__ Smem carve(char *smem, const Dev &D) {
     s.full0 = smem_u32(smem);
     s.empty0 = s.full0 + 8u * kMaxSlots;
     s.go_bar = s.empty0 + 8u * kMaxSlots;
-    s.ctl = reinterpret_cast<Ctl *>(smem + 256);   // 2 * 12 * 8 + 8 = 200 bytes of barriers before it
+    s.abar0 = s.go_bar + 8u;
+    s.dbar = s.abar0 + 16u;
+    s.sbar0 = s.dbar + 8u;
+    s.ctl = reinterpret_cast<Ctl *>(smem + 256);   // 2 * 12 * 8 + 8 + 40 = 240 bytes of barriers before it
     s.tab = reinterpret_cast<const Tables *>(smem + kSmemHeader);
     s.seg = reinterpret_cast<struct SegRec *>(smem + kSmemHeader + kSmemTables);
     s.ring = smem + kSmemHeader + kSmemTables + kSmemPlans;
@@ -298,6 +306,11 @@ __device__ __forceinline__ uint32_t poll_u32(const Dev &D, Ctl *ctl, const void 
     return v;
 }
 
+// the same waits as calls, for places where the wait is rare and the code around it is unrolled many times (the code of a
+// loop body should stay inside the instruction cache)
+static __device__ __noinline__ uint4 poll_u4_cold(const Dev &D, Ctl *ctl, const void *p, uint32_t tag) { return poll_u4(D, ctl, p, tag); }
+static __device__ __noinline__ uint32_t poll_u32_cold(const Dev &D, Ctl *ctl, const void *p, uint32_t tag) { return poll_u32(D, ctl, p, tag); }
+
 // ------------------------------------------------------------------------------------------- ring
 
 // A ring position is the slot (low byte) and the parity of the number of trips round the ring (bit 8): items passed so
@@ -315,10 +328,19 @@ __device__ __forceinline__ uint32_t ring_add(const Smem &S, uint32_t pos, int k)
     return slot | (par << 8);
 }
 
+// A wait on a shared-memory barrier, bounded.  Once a wait has run out somewhere (ctl->dead) the CTA still tries to
+// complete its ring protocol, but all its later waits together get one more allowance of tries, not one each.
 __device__ __forceinline__ void mbar_wait(const Dev &D, Ctl *ctl, uint32_t bar, uint32_t parity) {
-    for (unsigned it = 0; it < D.mbar_limit; ++it)
+    if (!ctl->dead) {
+        for (unsigned it = 0; it < D.mbar_limit; ++it)
+            if (mbar_try_wait(bar, parity)) return;
+        raise_timeout(D, ctl);
+        return;
+    }
+    for (unsigned it = 0; it < 4096u; ++it) {
         if (mbar_try_wait(bar, parity)) return;
-    raise_timeout(D, ctl);
+        if ((it & 255u) == 255u && atomicSub(const_cast<int *>(&ctl->dead_allowance), 256) <= 0) return;
+    }
 }
 
 // consumer: wait until the item at ring position r.pos has landed; returns its slot
@@ -1447,10 +1469,282 @@ static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, co
     }
 }
 
+// ------------------------------------------------- projection on the tcgen05 path (more than eight token rows, bf16)
+
+// K-major operand tile with the 128-byte swizzle: rows of 64 bf16 (128 bytes), 8-row groups 1024 bytes apart (stride byte
+// offset), leading byte offset unused (1), descriptor version of sm_100, layout type 2.  The tile starts on a 1024-byte
+// boundary; a K = 16 step inside the 64 columns is 32 bytes further.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t addr) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, both K-major, N and M of the tile
+__device__ __forceinline__ uint32_t umma_idesc(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_mma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+                 :: "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0) : "memory");
+}
+// one arrival at the barrier when every product issued by this thread so far has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
+}
+// box {64 columns, 8 rows, 1 layer} of a weight matrix -> shared memory (swizzled), completion on an mbarrier; no multicast
+__device__ __forceinline__ void tma_box(uint32_t dst, const void *tmap, int x, int y, int z, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 :: "r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// A tile of the CTA's segment: up to 128 weight rows (64 units of gate + up rows), 8-row groups in the order the
+// accumulator's columns take: plain jobs [rows 0-7][8-15]..., gate/up jobs [gate units 0-7][up units 0-7][gate 8-15]...
+struct UmmaTile { int u0, nu, groups; };
+__device__ __forceinline__ UmmaTile umma_tile(int epi, int u0, int hi) {
+    UmmaTile t;
+    t.u0 = u0;
+    t.nu = min(epi == EPI_GATEUP ? kUmmaTileRows / 2 : kUmmaTileRows, hi - u0);
+    t.groups = ((t.nu + 7) >> 3) * (epi == EPI_GATEUP ? 2 : 1);
+    return t;
+}
+
+// Producer: for every tile, for every block of 64 columns, one ring item with a box per row group.
+template <typename WT>
+static __device__ void produce_segment_umma(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, int layer) {
+    const int lane = threadIdx.x & 31, lay = max(layer, 0);
+    for (int u0 = R.lo; u0 < R.hi;) {
+        const UmmaTile t = umma_tile(J.epi, u0, R.hi);
+        for (int kc = 0; kc < J.kdim; kc += kUmmaK) {
+            uint32_t dst, bar;
+            ring_claim(D, S, ring, (uint32_t)t.groups * 1024u, dst, bar);
+            if (lane < t.groups) {
+                const bool up = J.epi == EPI_GATEUP && (lane & 1);
+                const int row = J.epi == EPI_GATEUP ? t.u0 + 8 * (lane >> 1) : t.u0 + 8 * lane;
+                tma_box(dst + (uint32_t)lane * 1024u, up ? J.tmap2 : J.tmap, kc, row, lay, bar);
+            }
+            ring.pos = ring_add(S, ring.pos, 1);
+        }
+        u0 += t.nu;
+    }
+}
+
+// One consumer warp issues the products; with at most 32 token rows (little to stage, the issuing thread is the limit) two
+// do, one per activation buffer, each into an accumulator of its own.  The other consumer warps stage activations.
+__host__ __device__ constexpr int umma_issuers(int m) { return m <= 32 ? 2 : 1; }
+// 16-byte loads of one column block per staging thread: NTM * 8 token rows x 16 quads over the staging threads
+__host__ __device__ constexpr int umma_loads(int ntm) {
+    return (ntm * 8 * 16 + (kConsumerWarps - umma_issuers(ntm * 8)) * 32 - 1) / ((kConsumerWarps - umma_issuers(ntm * 8)) * 32);
+}
+
+// Consumer.  Per tile and block of 64 columns: the staging warps (0..5) store the activations of the block (all token
+// rows) as two planes of bf16 (hi, lo) in the swizzled K-major layout, double buffered, the loads of the next block in
+// flight while this one is stored, and arrive at the buffer's "staged" barrier; the issuing warp (6) waits for that
+// barrier and for the block's weights, issues the eight products (four K = 16 steps, hi and lo planes into one
+// accumulator) and commits them to the buffer's "done" barrier.  Nobody waits for the issuing thread: staging runs
+// ahead until it needs a buffer back.  A ring slot is freed (one arrival per consumer warp) when the products that read
+// it are known to be done: two blocks later, or after the tile's last commit.  After the last block the accumulator
+// D[token][weight row] is read back by the thread of the token (warps 0..3), which finishes all outputs of its token
+// row: the row's share of the new sum of squares needs no reduction.  The shares of the input rows are added up on the
+// way, a few rows per staging warp and column block.
+template <typename WT, int NTM>
+static __device__ void consume_segment_umma(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
+    constexpr int kUmmaLoads = umma_loads(NTM);
+    const int M = D.M, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int kdim = J.kdim, n_kc = kdim / kUmmaK;
+    const uint32_t tag_in = tag_of(serial, J.in), tag_out = tag_of(serial, J.outt);
+    const bool normed = J.gain != nullptr;
+    const bool want_ss = J.epi == EPI_ADD && J.gain_out != nullptr;
+    const bool dead_rows = S.ctl->any_dead != 0;
+    const int n_iss = umma_issuers(M), stage_warps = kConsumerWarps - n_iss, stage_threads = stage_warps * 32;
+    const bool issuer = warp >= stage_warps;
+    const float *x = J.x;
+    char *const planes = S.acts;                     // [buffer][hi | lo][128 rows x 128 bytes]
+    const int G = (int)gridDim.x;
+    // rows whose shares a staging warp adds up per column block, so that all M rows are done by the last block
+    const int rows_per = (M + stage_warps * n_kc - 1) / (stage_warps * n_kc);
+    csync();                                         // the previous user of the activation area and of S.ss is done
+    uint32_t chunk = S.ctl->umma_chunks, tiles = S.ctl->umma_tiles;
+    float ss_acc = 0.f;
+    // a staging thread's quads of a column block: i = tid + u * 192 -> token row i / 16, quad i % 16 (four columns)
+    auto issue = [&](uint4 (&w)[kUmmaLoads], int kc) {
+#pragma unroll
+        for (int u = 0; u < kUmmaLoads; ++u) {
+            const int i = tid + u * stage_threads, r = i >> 4, q = i & 15;
+            w[u] = make_uint4(tag_in, tag_in, tag_in, tag_in);
+            if (r < M && !(dead_rows && S.ctl->row_dead[r])) w[u] = ld_relaxed_u4(x + (size_t)r * kdim + kc * kUmmaK + q * 4);
+        }
+    };
+    // one arrival of this warp at the "empty" barrier of the ring slot that held block kc of the tile
+    auto free_slot = [&](uint32_t pos0, int kc) {
+        if (lane == 0) mbar_arrive(S.empty0 + 8u * ring_slot(S, ring_add(S, pos0, kc)));
+    };
+    for (int u0 = R.lo; u0 < R.hi;) {
+        const UmmaTile t = umma_tile(J.epi, u0, R.hi);
+        const int n_cols = t.groups * 8, mma_n = (n_cols + 15) & ~15;
+        const uint32_t idesc = umma_idesc(128, mma_n);      // M = 128: row i of the accumulator is lane i of tensor memory
+        const uint32_t pos0 = ring.pos, chunk0 = chunk;
+        const bool first_tile = u0 == R.lo;
+        if (issuer) {
+            // ---- an issuing warp.  It passes every block of the tile: once a block's weights have landed the warp gives its
+            // arrival for the slot (the slot is refilled only after the staging warps' arrivals, which follow the completion
+            // of the products that read it); the blocks of its own buffer it multiplies.
+            const int me = warp - stage_warps;
+            for (int kc = 0; kc < n_kc; ++kc) {
+                const uint32_t c = chunk0 + (uint32_t)kc;
+                const int buf = (int)(c & 1u);
+                Ring r;
+                r.pos = ring_add(S, pos0, kc);
+                const uint32_t wts = smem_u32(ring_wait(D, S, r));
+                free_slot(pos0, kc);
+                if (n_iss == 2 && buf != me) continue;
+                mbar_wait(D, S.ctl, S.sbar0 + 8u * (uint32_t)buf, (c >> 1) & 1u);       // the block's activations are staged
+                tcgen05_after_sync();
+                if (lane == 0) {
+                    const uint32_t a_hi = smem_u32(planes + buf * 2 * kUmmaPlaneBytes), a_lo = a_hi + (uint32_t)kUmmaPlaneBytes;
+                    const uint32_t acc = S.ctl->tmem + (n_iss == 2 ? (uint32_t)(buf * kUmmaTileRows) : 0u);
+                    const bool fresh = kc < n_iss;                       // the accumulator's first block of the tile
+#pragma unroll
+                    for (int ks = 0; ks < kUmmaK / 16; ++ks) {
+                        const uint64_t db = umma_desc_sw128(wts + (uint32_t)ks * 32u);
+                        umma_mma(acc, umma_desc_sw128(a_hi + (uint32_t)ks * 32u), db, idesc, (!fresh || ks > 0) ? 1u : 0u);
+                        umma_mma(acc, umma_desc_sw128(a_lo + (uint32_t)ks * 32u), db, idesc, 1u);
+                    }
+                    umma_commit(S.abar0 + 8u * (uint32_t)buf);
+                }
+                __syncwarp();
+            }
+            if (lane == 0) umma_commit(S.dbar);          // one arrival per issuing warp when all its products are done
+            __syncwarp();
+        } else {
+            // ---- the staging warps
+            uint4 wa[kUmmaLoads], wb[kUmmaLoads];
+            issue(wa, 0);
+            // one column block: w holds its words, wn receives those of the next block
+            auto block = [&](uint4 (&w)[kUmmaLoads], uint4 (&wn)[kUmmaLoads], int kc) {
+                const uint32_t c = chunk0 + (uint32_t)kc;
+                const int buf = (int)(c & 1u);
+                char *p_hi = planes + buf * 2 * kUmmaPlaneBytes, *p_lo = p_hi + kUmmaPlaneBytes;
+                if (kc + 1 < n_kc) issue(wn, kc + 1);          // the loads of the next block go out before this one is looked at
+                // the shares of a few input rows per warp (normed jobs, first tile only): all loads first, then the tags
+                if (normed && first_tile) {
+                    for (int q = 0; q < rows_per; ++q) {
+                        const int m = (kc * rows_per + q) * stage_warps + warp;
+                        if (m < M) {
+                            float sum = 0.f;
+                            if (!S.ctl->row_dead[m]) {
+                                uint32_t sw[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) sw[e] = lane + 32 * e < G ? ld_relaxed_u32(ss_word(D, lane + 32 * e, m)) : tag_in;
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    if ((sw[e] & 3u) != tag_in) sw[e] = poll_u32_cold(D, S.ctl, ss_word(D, lane + 32 * e, m), tag_in);
+                                    if (lane + 32 * e < G) sum += untag(sw[e]);
+                                }
+                                sum = warp_sum(sum);
+                            }
+                            if (lane == 0) S.ss[m] = sum;
+                        }
+                    }
+                }
+                // the products that read this buffer two blocks ago must be done; their ring slot is free then
+                if (kc >= 2) {
+                    mbar_wait(D, S.ctl, S.abar0 + 8u * (uint32_t)buf, ((c >> 1) - 1u) & 1u);
+                    free_slot(pos0, kc - 2);
+                }
+#pragma unroll
+                for (int u = 0; u < kUmmaLoads; ++u) {
+                    const int i = tid + u * stage_threads, r = i >> 4, q = i & 15;
+                    if (r < M) {
+                        if (!tags_ok(w[u], tag_in) && !(dead_rows && S.ctl->row_dead[r]))
+                            w[u] = poll_u4_cold(D, S.ctl, x + (size_t)r * kdim + kc * kUmmaK + q * 4, tag_in);
+                        uint2 hi, lo;
+                        hi.x = __byte_perm(w[u].x, w[u].y, 0x7632);
+                        hi.y = __byte_perm(w[u].z, w[u].w, 0x7632);
+                        lo.x = __byte_perm(w[u].x, w[u].y, 0x5410) & 0xFFFCFFFCu;
+                        lo.y = __byte_perm(w[u].z, w[u].w, 0x5410) & 0xFFFCFFFCu;
+                        const int off = (r >> 3) * 1024 + (r & 7) * 128 + (((q >> 1) ^ (r & 7)) << 4) + ((q & 1) << 3);
+                        *reinterpret_cast<uint2 *>(p_hi + off) = hi;
+                        *reinterpret_cast<uint2 *>(p_lo + off) = lo;
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic-proxy stores to shared memory, read by the tensor core's proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(S.sbar0 + 8u * (uint32_t)buf);
+                if (kc == 0 && first_tile && S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
+            };
+            for (int kc = 0; kc < n_kc; kc += 2) {
+                block(wa, wb, kc);
+                if (kc + 1 < n_kc) block(wb, wa, kc + 1);
+            }
+        }
+        ring.pos = ring_add(S, pos0, n_kc);
+        chunk = chunk0 + (uint32_t)n_kc;
+        // ---- every product of the tile is done: the last slots are freed, the accumulator is read
+        mbar_wait(D, S.ctl, S.dbar, tiles & 1u);
+        ++tiles;
+        tcgen05_after_sync();
+        if (!issuer)       // (an issuing warp gave its arrival for every slot when the slot's weights landed)
+            for (int kc = max(n_kc - 2, 0); kc < n_kc; ++kc) free_slot(pos0, kc);
+        if (normed && first_tile) {
+            csync();
+            if (tid < M) S.ss[tid] = S.ctl->row_dead[tid] ? 1.f : 1.0f / sqrtf(S.ss[tid] / (float)kdim + D.eps);
+            csync();
+            if (J.norm_out) publish_normed_slice<WT>(D, J.x, J.kdim, J.gain, S.ss, tag_out);
+        }
+        if (warp < 4) {      // thread = token row (warps 0..3 own the accumulator's lanes 0..127)
+            const int m = tid;
+            const float inv = (normed && m < M) ? S.ss[m] : 1.f;
+            for (int c0 = 0; c0 < n_cols; c0 += 16) {
+                uint32_t v[16];
+                // (a tile of one block has used the accumulator of that block's buffer only)
+                const uint32_t taddr = S.ctl->tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0 +
+                                       ((n_iss == 2 && (chunk0 & 1u)) ? (uint32_t)kUmmaTileRows : 0u);
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                               "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                             : "r"(taddr) : "memory");
+                if (n_iss == 2 && n_kc >= 2) {       // two accumulators (one per activation buffer): their sum
+                    uint32_t v2[16];
+                    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                                 : "=r"(v2[0]), "=r"(v2[1]), "=r"(v2[2]), "=r"(v2[3]), "=r"(v2[4]), "=r"(v2[5]), "=r"(v2[6]), "=r"(v2[7]), "=r"(v2[8]),
+                                   "=r"(v2[9]), "=r"(v2[10]), "=r"(v2[11]), "=r"(v2[12]), "=r"(v2[13]), "=r"(v2[14]), "=r"(v2[15])
+                                 : "r"(taddr ^ (uint32_t)kUmmaTileRows) : "memory");
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
+                }
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (m < M) {
+                    // sixteen columns = two row groups: plain jobs sixteen units, gate/up jobs eight units (gate, up)
+                    const int units = J.epi == EPI_GATEUP ? 8 : 16;
+                    const int ub = t.u0 + (J.epi == EPI_GATEUP ? (c0 >> 1) : c0);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        if (j < units && ub + j < t.u0 + t.nu) {
+                            const float a = __uint_as_float(v[j]) * inv;
+                            const float b2 = J.epi == EPI_GATEUP ? __uint_as_float(v[(j + 8) & 15]) * inv : 0.f;
+                            const float r = epilogue_store<WT>(J, m, ub + j, a, b2, inv, tag_out);
+                            ss_acc += r * r;
+                        }
+                    }
+                }
+            }
+        }
+        tcgen05_before_sync();
+        csync();                 // the accumulator has been read: the next tile (or job) may overwrite it
+        tcgen05_after_sync();
+        u0 += t.nu;
+    }
+    if (want_ss && tid < M) st_relaxed_u32(ss_word(D, blockIdx.x, tid), tagged(ss_acc, tag_out));
+    if (tid == 0) { S.ctl->umma_chunks = chunk; S.ctl->umma_tiles = tiles; }
+}
+
 // NTM: token tiles of 8 (bf16 weights) or token rows (fp32 weights) the kernel is compiled for
 template <typename WT, int NTM> struct ConsumeSegment;
 template <int NTM> struct ConsumeSegment<bf16, NTM> {
     static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
+        if (NTM > 1 && D.umma) { consume_segment_umma<bf16, NTM>(D, S, ring, J, R, serial); return; }
         if (D.kca < J.kdim) { consume_segment_chunked<bf16>(D, S, ring, J, R, serial); return; }
         consume_segment_bf16<bf16, NTM>(D, S, ring, J, R, serial);
     }
@@ -1506,7 +1800,8 @@ static __device__ void gemv_stage(const Dev &D, const Smem &S, Ring &ring, const
             J.norm_out = norm_out ? 1 : 0;
             norm_out = false;
             if (PRODUCER) {
-                if (sizeof(WT) == 2 && D.kca < J.kdim) produce_segment_chunked<WT>(D, S, ring, J, R);
+                if (sizeof(WT) == 2 && NTM > 1 && D.umma) produce_segment_umma<WT>(D, S, ring, J, R, st.layer);
+                else if (sizeof(WT) == 2 && D.kca < J.kdim) produce_segment_chunked<WT>(D, S, ring, J, R);
                 else produce_segment<WT>(D, S, ring, J, R);
             }
             else ConsumeSegment<WT, NTM>::run(D, S, ring, J, R, serial);
@@ -2632,8 +2927,16 @@ step_kernel(const __grid_constant__ Dev D, int st_lo, int st_hi, int n_steps, ui
             mbar_init(S.empty0 + 8u * i, (uint32_t)kConsumerWarps);
         }
         mbar_init(S.go_bar, 1u);
+        mbar_init(S.abar0, 1u);
+        mbar_init(S.abar0 + 8u, 1u);
+        mbar_init(S.dbar, (uint32_t)umma_issuers(D.M));
+        mbar_init(S.sbar0, (uint32_t)(kConsumerWarps - umma_issuers(D.M)));
+        mbar_init(S.sbar0 + 8u, (uint32_t)(kConsumerWarps - umma_issuers(D.M)));
         S.ctl->dead = 0;
+        S.ctl->dead_allowance = 1 << 22;
         S.ctl->go = 0;
+        S.ctl->umma_chunks = 0u;
+        S.ctl->umma_tiles = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
@@ -2644,7 +2947,14 @@ step_kernel(const __grid_constant__ Dev D, int st_lo, int st_hi, int n_steps, ui
     }
     __syncthreads();
     plan_segments<WT>(D, S);
+    const bool use_tmem = sizeof(WT) == 2 && NTM > 1 && D.umma != 0;
+    if (use_tmem && warp == 0) {     // the accumulator columns of the tcgen05 projections, held until the launch ends
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&S.ctl->tmem)), "r"(kUmmaTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tcgen05_before_sync();
+    }
     __syncthreads();
+    if (use_tmem) tcgen05_after_sync();
     uint32_t ring_pos = 0;
     const TagRef once = {1, 0};
     const int p_sample = D.n_stages - 2, p_commit = D.n_stages - 1;
@@ -2701,6 +3011,11 @@ step_kernel(const __grid_constant__ Dev D, int st_lo, int st_hi, int n_steps, ui
             commit_stage<WT>(D, serial);
             if (tracing) trace_mark(D, 2 + 2 * p_commit);
         }
+    }
+    if (use_tmem) {     // every product has been waited for; the columns go back before the CTA ends
+        tcgen05_before_sync();
+        csync();
+        if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(S.ctl->tmem), "r"(kUmmaTmemCols) : "memory");
     }
 }
 

@@ -55,6 +55,7 @@ struct GemvJob {
     int out_plain;           // 1: `out` is published as plain tagged fp32 (logits) even in a bf16 model
     int in_jinc, out_jinc;   // a layer job: how much in.j / outt.j grow from one layer to the next
     long long gain_out_step; // a layer job: bytes from one layer's gain_out to the next layer's
+    const void *tmap, *tmap2; // tcgen05 path: tensor maps (in the workspace) of W and W2: {columns, rows, layers}, boxes of 64 x 8
     const float *res;        // EPI_ADDG: tagged fp32 residual [M][out_ld]
     int norm_out, pad_;      // norm_out (set per stage by the kernel): this job also publishes the CTA's columns of the normed input
 };
@@ -80,7 +81,16 @@ struct Tables {
 constexpr int kSmemTables = (sizeof(Tables) + 127) / 128 * 128;
 // behind the tables: one record per job with this CTA's share of its rows and how they are tiled (fixed for a launch)
 constexpr int kSegRecBytes = 40;
-constexpr int kSmemPlans = ((kLayerJobs + kMaxTailJobs) * kSegRecBytes + 127) / 128 * 128;
+// (padded so that the ring behind them starts on a 1024-byte boundary: swizzled tensor-core tiles need it)
+constexpr int kSmemPlans = ((kSmemHeader + kSmemTables + (kLayerJobs + kMaxTailJobs) * kSegRecBytes + 1023) / 1024 * 1024) - kSmemHeader - kSmemTables;
+
+// Projections over more than eight token rows on bf16 models run on the tensor cores of the 5th generation (tcgen05): the
+// token rows (as bf16 hi and lo planes) are the M side of the product, a CTA's weight rows the N side, the fp32
+// accumulator lives in tensor memory.  Weights arrive by TMA in boxes of 8 rows x 64 columns with the 128-byte swizzle;
+// a ring item is one block of 64 columns for all row groups of a tile of at most kUmmaTileRows weight rows.
+constexpr int kUmmaTileRows = 128, kUmmaK = 64, kUmmaTmemCols = 256;
+constexpr int kUmmaPlaneBytes = 128 * kUmmaK * 2;          // one plane (hi or lo) of 128 token rows x 64 columns
+constexpr int kUmmaActsBytes = 4 * kUmmaPlaneBytes;        // two buffers of two planes
 
 // Everything a kernel needs; passed by value.
 struct Dev {
@@ -121,6 +131,7 @@ struct Dev {
     float *qh, *hattn, *gpub, *hpart;   // cross-attention heads: queries [K][M][d], attention rows [K][M][d], final hidden state [M][d], split partials
     void *hckv_pool;               // [K][2][B*cpages][H] tiles: keys and values of the condition under every head's own projections
     int head_kind;
+    int umma;                      // projections on the tcgen05 path (bf16, more than eight token rows)
     uint32_t *treex;               // probability-tree sampling: [B][K][8][2] the heads' best tokens and their probabilities
     uint32_t *candx, *header;      // [B][K1 + 1] resampled tokens and accept length; [B][4] len, flags
     uint32_t *done;                // [grid] "this CTA has finished the projections of the step"
