@@ -83,6 +83,8 @@ def workload(args):
         cfg["n_draft"] = 0
     if args.tokens:
         cfg["gen_tokens"] = args.tokens
+    if args.head_kind:
+        cfg["head_kind"] = 1
     return cfg
 
 
@@ -300,7 +302,7 @@ def run_gpu(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 weights, fp16 cache, f32 arithmetic" if cfg["dtype"] == 1 else "f32", "data": "synthetic",
-        "config": {"workload": f"config {args.config} ({cfg['name']}): batch {B}, K={K} heads, {T} tokens per mesh, "
+        "config": {"workload": f"config {args.config} ({cfg['name']}): batch {B}, K={K} {'cross-attention ' if cfg.get('head_kind') else ''}heads, {T} tokens per mesh, "
                                f"verify_mode {cfg['verify_mode']}, k={cfg['k_accept']}, T={cfg['temperature']}",
                    "weights": "iid N(0, sigma) as configured (heads untrained)", "l2": "inputs larger than L2 "
                    f"({alg['fixed'] / 1e6:.0f} MB of weights streamed per decoding step)", "parallelism": "replicas"},
@@ -354,6 +356,8 @@ def main():
     ap.add_argument("--no-fitted-heads", action="store_true", help="skip the K = 0 and fitted-heads runs of the same mesh")
     ap.add_argument("--fit-meshes", type=int, default=64, help="meshes of 512 tokens the heads are fitted on")
     ap.add_argument("--no-scripted", action="store_true", help="skip the scripted-draft sweep (tokens/s against forced SCR)")
+    ap.add_argument("--head-kind", type=int, default=0, choices=[0, 1],
+                    help="1: cross-attention decoding heads (Eq. 3) in place of the configured MLP heads")
     ap.add_argument("--head-sweep", action="store_true", help="also sweep the number of decoding heads (heads fitted per count)")
     ap.add_argument("--reference-seconds", type=float, default=0.0,
                     help="--impl reference: CPU seconds per step (default: 120 s spread over the steps, 4 to 30 s each)")

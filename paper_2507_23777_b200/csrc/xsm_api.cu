@@ -659,6 +659,12 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
     D.umma = (umma_shape(c, batch) && ctx->encode_tiled != nullptr) ? 1 : 0;
     if (const char *m = plan_smem(c, batch, D, smem_bytes)) return fail(ctx, XSM_ERR_CAPACITY, m);
     ctx->smem_bytes = smem_bytes;
+    {   // at most eight token rows, all activations of the widest projection staged at once with room for the warps'
+        // partial products behind them, the CTAs' shares of a row readable by one warp pass: the compact instance
+        const int M = batch * D.K1, kmax = c.d_model > c.d_ff ? c.d_model : c.d_ff;
+        D.small = (c.dtype == 1 && M <= 8 && D.kca >= kmax && ctx->grid * M <= 1536 && (ctx->grid & 3) == 0 &&
+                   D.acts_bytes - M * (kmax * 4 + 16) >= kConsumerWarps * kSmallRedBytes) ? 1 : 0;
+    }
     {   // the step kernel instance for this batch must fit one CTA per multiprocessor
         Dev probe = D;
         probe.M = batch * D.K1;

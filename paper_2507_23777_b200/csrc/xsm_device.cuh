@@ -331,16 +331,11 @@ __device__ __forceinline__ uint32_t ring_add(const Smem &S, uint32_t pos, int k)
 // A wait on a shared-memory barrier, bounded.  Once a wait has run out somewhere (ctl->dead) the CTA still tries to
 // complete its ring protocol, but all its later waits together get one more allowance of tries, not one each.
 __device__ __forceinline__ void mbar_wait(const Dev &D, Ctl *ctl, uint32_t bar, uint32_t parity) {
-    if (!ctl->dead) {
-        for (unsigned it = 0; it < D.mbar_limit; ++it)
-            if (mbar_try_wait(bar, parity)) return;
-        raise_timeout(D, ctl);
-        return;
-    }
-    for (unsigned it = 0; it < 4096u; ++it) {
+    for (unsigned it = 0; it < D.mbar_limit; ++it) {
         if (mbar_try_wait(bar, parity)) return;
-        if ((it & 255u) == 255u && atomicSub(const_cast<int *>(&ctl->dead_allowance), 256) <= 0) return;
+        if ((it & 255u) == 255u && ctl->dead && atomicSub(const_cast<int *>(&ctl->dead_allowance), 256) <= 0) return;
     }
+    raise_timeout(D, ctl);
 }
 
 // consumer: wait until the item at ring position r.pos has landed; returns its slot
@@ -428,10 +423,8 @@ static_assert(sizeof(SegRec) == kSegRecBytes, "size of a plan record");
 // Projections of at most eight token rows whose activations fit the staging area at once (batch 1) take the path of
 // consume_small: every warp multiplies all tiles of a group over its share of the columns.
 constexpr int kSmallTiles = 4;        // tiles of a group on that path (their accumulators live in registers)
-constexpr int kSmallRedBytes = 512;   // partial products of one warp for one tile: [8 tokens][16 rows] floats
 template <typename WT> __device__ __forceinline__ bool small_mode(const Dev &D, int kdim) {
-    return sizeof(WT) == 2 && D.M <= 8 && D.kca >= kdim && (int)gridDim.x * D.M <= 1536 && ((int)gridDim.x & 3) == 0 &&
-           D.acts_bytes - D.M * (kdim * 4 + 16) >= kConsumerWarps * kSmallRedBytes;
+    return sizeof(WT) == 2 && D.small;      // (decided by the host for all projections of the model at once)
 }
 template <typename WT> __device__ __forceinline__ SegPlan seg_plan(const Dev &D, const Smem &S, const GemvJob &J, int lo, int hi) {
     SegPlan p;
@@ -1744,9 +1737,11 @@ static __device__ void consume_segment_umma(const Dev &D, const Smem &S, Ring &r
 template <typename WT, int NTM> struct ConsumeSegment;
 template <int NTM> struct ConsumeSegment<bf16, NTM> {
     static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
-        if (NTM > 1 && D.umma) { consume_segment_umma<bf16, NTM>(D, S, ring, J, R, serial); return; }
-        if (D.kca < J.kdim) { consume_segment_chunked<bf16>(D, S, ring, J, R, serial); return; }
-        consume_segment_bf16<bf16, NTM>(D, S, ring, J, R, serial);
+        if constexpr (NTM > 1) {     // (the instance for at most eight token rows holds consume_small only)
+            if (D.umma) { consume_segment_umma<bf16, NTM>(D, S, ring, J, R, serial); return; }
+            if (D.kca < J.kdim) { consume_segment_chunked<bf16>(D, S, ring, J, R, serial); return; }
+            consume_segment_bf16<bf16, NTM>(D, S, ring, J, R, serial);
+        }
     }
 };
 template <int NTM> struct ConsumeSegment<float, NTM> {
@@ -3055,7 +3050,7 @@ cudaError_t launch_step_dh(const Dev &D, int dtype, int st_lo, int st_hi, int n_
     const int M = D.M;
 #define XSM_GO(WT, NTM) return launch_step_instance<WT, NTM, DH>(D, st_lo, st_hi, n_steps, serial0, grid, smem_bytes, st, max_grid)
     if (dtype == 1) {
-        if (M <= 8) XSM_GO(bf16, 1);
+        if (M <= 8 && D.small) XSM_GO(bf16, 1);
         if (M <= 16) XSM_GO(bf16, 2);
         if (M <= 32) XSM_GO(bf16, 4);
         if (M <= 80) XSM_GO(bf16, 10);

@@ -92,6 +92,8 @@ constexpr int kUmmaTileRows = 128, kUmmaK = 64, kUmmaTmemCols = 256;
 constexpr int kUmmaPlaneBytes = 128 * kUmmaK * 2;          // one plane (hi or lo) of 128 token rows x 64 columns
 constexpr int kUmmaActsBytes = 4 * kUmmaPlaneBytes;        // two buffers of two planes
 
+constexpr int kSmallRedBytes = 512;   // at most eight token rows: partial products of one warp for one tile, [8 tokens][16 rows] floats
+
 // Everything a kernel needs; passed by value.
 struct Dev {
     // shape
@@ -132,6 +134,8 @@ struct Dev {
     void *hckv_pool;               // [K][2][B*cpages][H] tiles: keys and values of the condition under every head's own projections
     int head_kind;
     int umma;                      // projections on the tcgen05 path (bf16, more than eight token rows)
+    int small;                     // bf16, at most eight token rows, every projection's activations fit the staging area: the
+                                   // kernel instance that holds nothing but that path runs the step
     uint32_t *treex;               // probability-tree sampling: [B][K][8][2] the heads' best tokens and their probabilities
     uint32_t *candx, *header;      // [B][K1 + 1] resampled tokens and accept length; [B][4] len, flags
     uint32_t *done;                // [grid] "this CTA has finished the projections of the step"

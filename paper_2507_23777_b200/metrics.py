@@ -13,6 +13,9 @@ def algorithmic_bytes(cfg: dict, batch: int) -> dict:
     lm = d * V * e
     heads = K * (d * d + d * V) * e
     cross = batch * L * 2 * C * d * e
+    if cfg.get("head_kind", 0) == 1:      # cross-attention heads: Wq, Wo, Wout and each head's keys and values of the condition
+        heads = K * (2 * d * d + d * V) * e
+        cross += batch * K * 2 * C * d * e
     return {"fixed": backbone + lm + heads + cross, "per_position": batch * L * 2 * d * e,
             "backbone": backbone, "lm": lm, "heads": heads, "cross_kv": cross}
 
