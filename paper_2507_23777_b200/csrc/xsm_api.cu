@@ -261,8 +261,18 @@ bool umma_shape(const xsm_model_config &c, int batch) {
     return c.dtype == 1 && M > 8 && M <= 128 && c.d_model % kUmmaK == 0 && c.d_ff % kUmmaK == 0;
 }
 
-const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_bytes) {
+// jobs in the tail of a step: the LM head, then per decoding head W1 and Wout, or Wq, Wo and Wout
+int tail_jobs(const xsm_model_config &c) { return 1 + (c.head_kind == 1 ? 3 : 2) * c.n_draft; }
+
+// grid: CTAs of the step kernel if known (it sizes the staging of the sums-of-squares shares on the path for at most
+// eight token rows), 0: not known yet, plan for the largest
+const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_bytes, int grid = 0) {
     const int K1 = c.n_draft + 1, M = batch * K1, dh = c.d_head;
+    D.tab_bytes = smem_tab_bytes(tail_jobs(c));
+    D.plan_bytes = smem_plan_bytes(tail_jobs(c));
+    if (D.umma)      // swizzled tensor-core tiles: the ring starts on a 1024-byte boundary
+        D.plan_bytes = (kSmemHeader + D.tab_bytes + D.plan_bytes + 1023) / 1024 * 1024 - kSmemHeader - D.tab_bytes;
+    const int kSmemTables = D.tab_bytes, kSmemPlans = D.plan_bytes;
     if (D.umma) {
         // tcgen05 path: the activation area holds two buffers of two planes (hi, lo) of 128 token rows x 64 columns; the
         // other users of the area (attention, verification, commit) fit inside
@@ -286,7 +296,9 @@ const char *plan_smem(const xsm_model_config &c, int batch, Dev &D, int &smem_by
         return nullptr;
     }
     const int kmax = c.d_model > c.d_ff ? c.d_model : c.d_ff;
-    const int tail = (kMaxTokens + 1536) * 4;                        // sums of squares and their partials
+    // sums of squares and their partials; at most eight token rows of a bf16 model: the CTAs' shares [row][CTA]
+    int tail = (kMaxTokens + 1536) * 4;
+    if (grid > 0 && c.dtype == 1 && M <= 8 && grid * M <= 1536) tail = (kMaxTokens + ((grid * M + 31) & ~31)) * 4;
     const int avail = kSmemMax - kSmemHeader - kSmemTables - kSmemPlans - tail;
     // what the other users of the activation area need
     const int np = c.dtype == 1 ? (M <= 8 ? 8 : M <= 16 ? 16 : M <= 32 ? 32 : M <= 80 ? 80 : 128) : 8;
@@ -657,14 +669,17 @@ xsm_status xsm_prefill(xsm_ctx *ctx, int batch, const void *d_cond, const int32_
     Dev &D = ctx->dev;
     int smem_bytes = 0;
     D.umma = (umma_shape(c, batch) && ctx->encode_tiled != nullptr) ? 1 : 0;
-    if (const char *m = plan_smem(c, batch, D, smem_bytes)) return fail(ctx, XSM_ERR_CAPACITY, m);
-    ctx->smem_bytes = smem_bytes;
+    if (const char *m = plan_smem(c, batch, D, smem_bytes, ctx->grid)) return fail(ctx, XSM_ERR_CAPACITY, m);
     {   // at most eight token rows, all activations of the widest projection staged at once with room for the warps'
         // partial products behind them, the CTAs' shares of a row readable by one warp pass: the compact instance
         const int M = batch * D.K1, kmax = c.d_model > c.d_ff ? c.d_model : c.d_ff;
         D.small = (c.dtype == 1 && M <= 8 && D.kca >= kmax && ctx->grid * M <= 1536 && (ctx->grid & 3) == 0 &&
                    D.acts_bytes - M * (kmax * 4 + 16) >= kConsumerWarps * kSmallRedBytes) ? 1 : 0;
+        // (the other paths stage their partial sums of squares in the full-size area)
+        if (!D.small)
+            if (const char *m = plan_smem(c, batch, D, smem_bytes)) return fail(ctx, XSM_ERR_CAPACITY, m);
     }
+    ctx->smem_bytes = smem_bytes;
     {   // the step kernel instance for this batch must fit one CTA per multiprocessor
         Dev probe = D;
         probe.M = batch * D.K1;

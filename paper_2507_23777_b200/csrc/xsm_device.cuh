@@ -231,7 +231,7 @@ struct Ctl {
     int go;                     // written by the consumers before they release the producer for a step
     int trace_row;              // row of the timeline that the running stage fills when its inputs are in (0: off)
     int any_dead;               // some sequence of the batch has finished: row_dead has entries set
-    volatile unsigned char landed[16];   // attention: parity of the latest fill of each ring slot that is known to have landed
+    volatile unsigned char landed[16];   // attention: number (modulo 4) of the latest fill of each ring slot that is known to have landed
     uint32_t tmem;              // tcgen05 path: base address of the CTA's accumulator columns in tensor memory
     volatile uint32_t umma_chunks, umma_tiles;   // tcgen05 path: column blocks and tiles multiplied since the launch (phases of abar, dbar)
     int len[kMaxBatch];
@@ -264,8 +264,8 @@ __device__ __forceinline__ Smem carve(char *smem, const Dev &D) {
     s.sbar0 = s.dbar + 8u;
     s.ctl = reinterpret_cast<Ctl *>(smem + 256);   // 2 * 12 * 8 + 8 + 40 = 240 bytes of barriers before it
     s.tab = reinterpret_cast<const Tables *>(smem + kSmemHeader);
-    s.seg = reinterpret_cast<struct SegRec *>(smem + kSmemHeader + kSmemTables);
-    s.ring = smem + kSmemHeader + kSmemTables + kSmemPlans;
+    s.seg = reinterpret_cast<struct SegRec *>(smem + kSmemHeader + D.tab_bytes);
+    s.ring = smem + kSmemHeader + D.tab_bytes + D.plan_bytes;
     s.n_slots = D.n_slots;
     s.acts = s.ring + (size_t)D.n_slots * kSlotBytes;
     s.ss = reinterpret_cast<float *>(s.acts + D.acts_bytes);
@@ -1271,6 +1271,7 @@ static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, co
     ActLoads<kSmallLoads> A;
     A.plan(D, S, kdim, 0, normed);
     A.issue(D, x, tag_in);
+    const float inv_kdim = 1.0f / (float)kdim;
     const SegPlan p = R.p;
     const int lo = R.lo, hi = R.hi;
     const int epi = J0.epi, out_ld = J0.out_ld;
@@ -1341,7 +1342,7 @@ static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, co
                             sum += (v.x + v.y) + (v.z + v.w);
                         }
                         sum = warp_sum(sum);
-                        inv_rms[q] = S.ctl->row_dead[m] ? 1.f : 1.0f / sqrtf(sum / (float)kdim + D.eps);
+                        inv_rms[q] = S.ctl->row_dead[m] ? 1.f : rsqrtf(fmaf(sum, inv_kdim, D.eps));
                         if (norm_out && lane == 0) S.ss[m] = inv_rms[q];
                     }
                 }
@@ -1983,7 +1984,6 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
     }
     ws.l[0] = ws.l[0] * c0 + l0;
     ws.l[1] = ws.l[1] * c1 + l1;
-#pragma unroll
     if (__any_sync(0xffffffffu, c0 != 1.f || c1 != 1.f)) {     // a new maximum somewhere in the warp's rows
 #pragma unroll
         for (int dn = 0; dn < DH / 8; ++dn) { ws.o[dn][0] *= c0; ws.o[dn][1] *= c0; ws.o[dn][2] *= c1; ws.o[dn][3] *= c1; }
@@ -2030,11 +2030,28 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     const float qscale = D.scale * kLog2e;
     int p_lo, p_hi;
     split_pages(n, P, it.s, it.S, p_lo, p_hi);
+    // q (and the window's k, v) of this head: 16-byte words, row r = i / (DH / 4) of [q | k | v][K1]; two per thread
+    // are requested at once, and the first two before anything else (their round trip is the longest wait of the item)
+    const int nsrc = win ? 3 : 1, n_q = nsrc * K1 * (DH / 4);
+    auto q_word = [&](int i, int &row) -> const float * {
+        const int r = i / (DH / 4), c4 = i - r * (DH / 4), which = (r >= K1 ? 1 : 0) + (r >= 2 * K1 ? 1 : 0), j = r - which * K1;
+        row = r;
+        return qsrc + (size_t)(b * K1 + j) * q_ld + which * d + h * DH + c4 * 4;
+    };
+    uint4 qw[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int i = tid + u * kConsumerThreads;
+        int row;
+        qw[u] = make_uint4(tag_in, tag_in, tag_in, tag_in);
+        if (i < n_q) qw[u] = ld_relaxed_u4(q_word(i, row));
+    }
 
     if (MMA && tid < S.n_slots) {
-        // the fill of slot `tid` that precedes this item's first position has landed (a barrier of the CTA lies between)
-        const uint32_t slot0 = ring_slot(S, ring.pos), par0 = ring_parity(S, ring.pos);
-        S.ctl->landed[tid] = (unsigned char)((uint32_t)tid < slot0 ? par0 : par0 ^ 1u);
+        // the fill of slot `tid` that precedes this item's first position has landed (a barrier of the CTA lies between).
+        // Fills are numbered per item, modulo 4: the trip round the ring that the item starts in is number 1.
+        const uint32_t slot0 = ring_slot(S, ring.pos);
+        S.ctl->landed[tid] = (unsigned char)((uint32_t)tid < slot0 ? 1u : 0u);
     }
     csync();
     // the rotation table and the pages of the appended rows are fetched while q is awaited
@@ -2057,13 +2074,27 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
             }
         }
     }
-    // 1. fetch q (and the window's k, v) of this head
-    const int nsrc = win ? 3 : 1;
-    for (int i = tid; i < nsrc * K1 * (DH / 4); i += kConsumerThreads) {
-        const int which = i / (K1 * (DH / 4)), rem = i - which * K1 * (DH / 4), j = rem / (DH / 4), c4 = rem - j * (DH / 4);
-        const uint4 w = poll_u4(D, S.ctl, qsrc + (size_t)(b * K1 + j) * q_ld + which * d + h * DH + c4 * 4, tag_in);
-        *reinterpret_cast<float4 *>(A.raw + ((size_t)which * K1 + j) * DH + c4 * 4) =
-            make_float4(read_word<WT>(w.x), read_word<WT>(w.y), read_word<WT>(w.z), read_word<WT>(w.w));
+    // 1. q (and the window's k, v) arrive: raw[row][DH]
+    for (int i0 = 0; i0 < n_q; i0 += 2 * kConsumerThreads) {
+        if (i0 > 0) {
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int i = i0 + tid + u * kConsumerThreads;
+                int row;
+                if (i < n_q) qw[u] = ld_relaxed_u4(q_word(i, row));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i = i0 + tid + u * kConsumerThreads;
+            if (i < n_q) {
+                int row;
+                const float *src = q_word(i, row);
+                if (!tags_ok(qw[u], tag_in)) qw[u] = poll_u4(D, S.ctl, src, tag_in);
+                *reinterpret_cast<float4 *>(A.raw + (size_t)row * DH + (i % (DH / 4)) * 4) =
+                    make_float4(read_word<WT>(qw[u].x), read_word<WT>(qw[u].y), read_word<WT>(qw[u].z), read_word<WT>(qw[u].w));
+            }
+        }
     }
     csync();
     if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
@@ -2136,52 +2167,75 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     if constexpr (MMA) {
         const uint32_t q_hi = smem_u32(A.qh), q_lo = smem_u32(A.ql);
         const int upp = P / 32;   // 32-key units per page
-        // Who touches a page.  Where a page is one ring item and the ring has a slot per consumer warp, page i of the
-        // item belongs to warp i mod 7 alone: it waits for the page, multiplies both units and frees the slot with
-        // seven arrivals of its own, and the other warps never look at that page (their per-page bookkeeping would
-        // cost more than the units).  A warp that skips pages skips phases of a slot's barrier, and a parity wait
-        // cannot tell "the fill before mine is still on its way" from "mine has landed".  So every owner records the
-        // parity of the fill it has seen land (ctl->landed), and an owner waits for its slot's previous fill to be
-        // recorded before it tests the barrier; with at least seven slots the fill before that one had completed when
-        // the owner's previous page landed, so one bit is enough.  Otherwise every warp passes every page and the
-        // 32-key units go round the warps.
-        const bool own = D.kv_one_item && S.n_slots >= kConsumerWarps;
+        // Who touches a page.  Where a page is one ring item and the ring has a slot per consumer warp, the 32-key units
+        // of the item go round the warps, unit u of page i to warp (i * upp + u) mod 7, and only the warps that own a
+        // unit of a page look at it: they wait for the page and free the slot between them (seven arrivals: the owner
+        // of unit 0 gives what the others leave); the other warps never touch that page (their per-page bookkeeping
+        // would cost more than the units).  A warp that skips pages skips phases of a slot's barrier, and a parity
+        // wait cannot tell "the fill before mine is still on its way" from "mine has landed".  So every owner records
+        // the number (modulo 4) of the fill it has seen land (ctl->landed), and an owner tests the barrier only once
+        // its slot's previous fill, or the awaited one (by a fellow owner), is recorded; with at least seven slots the
+        // fill two before had completed when the owner's previous page landed, so two bits are enough.  Otherwise
+        // every warp passes every page.
+        const bool own = D.kv_one_item && S.n_slots >= kConsumerWarps && upp <= kConsumerWarps;
         const int n_it = D.kv_one_item ? 1 : 2, n_pages = p_hi - p_lo;
         uint32_t pos = ring.pos;
-        for (int pg = p_lo; pg < p_hi; ++pg, pos = ring_add(S, pos, n_it)) {
+        uint32_t fill = 1u;                         // number of the trip round the ring that `pos` is in
+        int turn = 0;                               // (pages so far * upp) mod 7: the warp of the page's unit 0
+        for (int pg = p_lo; pg < p_hi; ++pg) {
             const int rel = pg - p_lo;
-            if (own && (rel % kConsumerWarps) != warp) continue;
+            int du = warp - turn;                   // this warp's unit of the page, if below upp
+            if (du < 0) du += kConsumerWarps;
+            const uint32_t here = pos, fill_here = fill;
+            {   // the next page's position, trip and turn
+                const uint32_t nx = ring_add(S, pos, n_it);
+                if (ring_slot(S, nx) < ring_slot(S, pos)) ++fill;
+                pos = nx;
+                turn += upp;
+                if (turn >= kConsumerWarps) turn -= kConsumerWarps;
+            }
+            if (own && du >= upp) continue;
             Ring r;
-            r.pos = pos;
+            r.pos = here;
+            const uint32_t slot = ring_slot(S, here);
             if (own) {
                 if (lane == 0) {
+                    const unsigned char prev = (unsigned char)((fill_here - 1u) & 3u), cur = (unsigned char)(fill_here & 3u);
                     unsigned it2 = 0;
-                    while (S.ctl->landed[ring_slot(S, pos)] != (unsigned char)(ring_parity(S, pos) ^ 1u) && !S.ctl->dead)
+                    for (;;) {
+                        const unsigned char seen = S.ctl->landed[slot];
+                        if (seen == prev || seen == cur || S.ctl->dead) break;
                         if (++it2 > D.mbar_limit) { raise_timeout(D, S.ctl); break; }
+                    }
                 }
                 __syncwarp();
             }
             const char *ks = ring_wait(D, S, r);
-            if (own && lane == 0) S.ctl->landed[ring_slot(S, pos)] = (unsigned char)ring_parity(S, pos);
+            if (own && lane == 0) S.ctl->landed[slot] = (unsigned char)(fill_here & 3u);
             const char *vs = ks + D.tile_bytes;
-            if (n_it == 2) { r.pos = ring_add(S, pos, 1); vs = ring_wait(D, S, r); }
+            if (n_it == 2) { r.pos = ring_add(S, here, 1); vs = ring_wait(D, S, r); }
             const int nv_page = min(P, n - pg * P);
-            for (int u = 0; u < upp; ++u) {
-                const int nv = min(32, nv_page - u * 32);
-                if (nv > 0 && (own || ((rel * upp + u) % kConsumerWarps) == warp))
-                    attn_unit<DH, false>(q_hi, q_lo, smem_u32(ks), smem_u32(vs), u * 32, nv, ws);
+            if (own) {
+                const int nv = min(32, nv_page - du * 32);
+                if (nv > 0) attn_unit<DH, false>(q_hi, q_lo, smem_u32(ks), smem_u32(vs), du * 32, nv, ws);
+            } else {
+                for (int u = 0; u < upp; ++u) {
+                    const int nv = min(32, nv_page - u * 32);
+                    if (nv > 0 && ((rel * upp + u) % kConsumerWarps) == warp)
+                        attn_unit<DH, false>(q_hi, q_lo, smem_u32(ks), smem_u32(vs), u * 32, nv, ws);
+                }
             }
             __syncwarp();
             if (own) {
-                if (lane < kConsumerWarps) mbar_arrive(S.empty0 + 8u * ring_slot(S, pos));
+                if (lane < (du == 0 ? kConsumerWarps - (upp - 1) : 1)) mbar_arrive(S.empty0 + 8u * slot);
             } else if (lane == 0) {
-                mbar_arrive(S.empty0 + 8u * ring_slot(S, pos));
+                mbar_arrive(S.empty0 + 8u * slot);
                 if (n_it == 2) mbar_arrive(S.empty0 + 8u * ring_slot(S, r.pos));
             }
         }
         ring.pos = pos;
         // the window's own keys, under the causal mask, as one more unit for the warp whose turn is next
-        if (win && ((own ? n_pages : n_pages * upp) % kConsumerWarps) == warp)
+        if (win && ((n_pages * upp) % kConsumerWarps) == warp)
             attn_unit<DH, true>(q_hi, q_lo, smem_u32(A.kt), smem_u32(A.vt), 0, K1, ws);
         // quad-reduce the denominators, park the state in shared memory
         const int g = lane >> 2, t = lane & 3;
@@ -2256,15 +2310,15 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
             }
         }
     }
-    // 5. the window's own keys under the causal mask: query row j (one warp each) against window keys 0..j
-    {
+    // 5. fp32 cache: the window's own keys under the causal mask: query row j (one warp each) against window keys 0..j
+    if constexpr (!MMA) {
         float *wst = A.st + (size_t)kConsumerWarps * K1 * (DH + 2);
         constexpr int EPL = (DH + 31) / 32;
         for (int j = warp; j < K1; j += kConsumerWarps) {
             float m = kNegBig, l = 0.f, acc[EPL];
 #pragma unroll
             for (int i = 0; i < EPL; ++i) acc[i] = 0.f;
-            if (win && !MMA) {
+            if (win) {
                 for (int wk = 0; wk <= j; ++wk) {
                     float dsum = 0.f;
 #pragma unroll
@@ -2292,14 +2346,35 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
         }
     }
     csync();
-    // 6. merge the warps (and the window state); one thread per (query row, element); element DH = denominator
+    // 6. merge the warps (and, fp32 cache, the window state); element DH = denominator
+    constexpr int n_states = MMA ? kConsumerWarps : kConsumerWarps + 1;
+    if (it.S == 1) {
+        // no other split: one thread per (query row, element) forms numerator and denominator from the same weights
+        // and publishes the quotient (the same sums in the same order as the two passes below)
+        for (int i = tid; i < K1 * DH; i += kConsumerThreads) {
+            const int j = i / DH, e = i - j * DH;
+            float m = kNegBig;
+#pragma unroll
+            for (int w = 0; w < n_states; ++w) m = fmaxf(m, A.st[((size_t)w * K1 + j) * (DH + 2) + DH]);
+            float o = 0.f, l = 0.f;
+#pragma unroll
+            for (int w = 0; w < n_states; ++w) {
+                const float *sw = A.st + ((size_t)w * K1 + j) * (DH + 2);
+                const float wg = exp2f(sw[DH] - m);
+                o += wg * sw[e];
+                l += wg * sw[DH + 1];
+            }
+            st_relaxed_u32(out + (size_t)(b * K1 + j) * d + h * DH + e, publish_word<WT>(o / l, tag_out, false));
+        }
+        return;
+    }
     float *mg = A.raw;    // [K1][DH + 2] merged (O, m, l); raw q/k/v are no longer needed
     for (int i = tid; i < K1 * (DH + 1); i += kConsumerThreads) {
         const int j = i / (DH + 1), e = i - j * (DH + 1);
         float m = kNegBig;
-        for (int w = 0; w <= kConsumerWarps; ++w) m = fmaxf(m, A.st[((size_t)w * K1 + j) * (DH + 2) + DH]);
+        for (int w = 0; w < n_states; ++w) m = fmaxf(m, A.st[((size_t)w * K1 + j) * (DH + 2) + DH]);
         float o = 0.f;
-        for (int w = 0; w <= kConsumerWarps; ++w) {
+        for (int w = 0; w < n_states; ++w) {
             const float *sw = A.st + ((size_t)w * K1 + j) * (DH + 2);
             o += exp2f(sw[DH] - m) * (e < DH ? sw[e] : sw[DH + 1]);
         }
@@ -2938,7 +3013,7 @@ step_kernel(const __grid_constant__ Dev D, int st_lo, int st_hi, int n_steps, ui
     {   // the tables move to shared memory once per launch
         const uint32_t *src = reinterpret_cast<const uint32_t *>(D.tables);
         uint32_t *dst = reinterpret_cast<uint32_t *>(smem + kSmemHeader);
-        for (int i = tid; i < (int)(sizeof(Tables) / 4); i += kThreads) dst[i] = __ldg(src + i);
+        for (int i = tid; i < min(D.tab_bytes, (int)sizeof(Tables)) / 4; i += kThreads) dst[i] = __ldg(src + i);
     }
     __syncthreads();
     plan_segments<WT>(D, S);

@@ -73,16 +73,19 @@ struct Stage {
 constexpr int kLayerStages = 8, kMaxTailStages = 6, kLayerJobs = 6, kMaxTailJobs = 3 * kMaxDraft + 1;
 struct Tables {
     Stage stages[kLayerStages + kMaxTailStages];
-    GemvJob jobs[kLayerJobs + kMaxTailJobs];
     long long layer_bytes;
     const void *gain_last;   // gain_out of the last layer's down projection (the final RMSNorm)
     int n_tail_stages, n_tail_jobs;
+    GemvJob jobs[kLayerJobs + kMaxTailJobs];      // last: the copy in shared memory ends behind the jobs in use
 };
-constexpr int kSmemTables = (sizeof(Tables) + 127) / 128 * 128;
 // behind the tables: one record per job with this CTA's share of its rows and how they are tiled (fixed for a launch)
 constexpr int kSegRecBytes = 40;
-// (padded so that the ring behind them starts on a 1024-byte boundary: swizzled tensor-core tiles need it)
-constexpr int kSmemPlans = ((kSmemHeader + kSmemTables + (kLayerJobs + kMaxTailJobs) * kSegRecBytes + 1023) / 1024 * 1024) - kSmemHeader - kSmemTables;
+// shared memory of the tables' copy and of the plan records for a model with `tail_jobs` jobs in the tail of the step
+// (Dev.tab_bytes, Dev.plan_bytes: the host sizes them, so that a model with few heads leaves more room for the ring)
+constexpr int smem_tab_bytes(int tail_jobs) {
+    return ((int)(sizeof(Tables) - sizeof(GemvJob) * (kMaxTailJobs - tail_jobs)) + 127) / 128 * 128;
+}
+constexpr int smem_plan_bytes(int tail_jobs) { return ((kLayerJobs + tail_jobs) * kSegRecBytes + 127) / 128 * 128; }
 
 // Projections over more than eight token rows on bf16 models run on the tensor cores of the 5th generation (tcgen05): the
 // token rows (as bf16 hi and lo planes) are the M side of the product, a CTA's weight rows the N side, the fp32
@@ -134,6 +137,7 @@ struct Dev {
     void *hckv_pool;               // [K][2][B*cpages][H] tiles: keys and values of the condition under every head's own projections
     int head_kind;
     int umma;                      // projections on the tcgen05 path (bf16, more than eight token rows)
+    int tab_bytes, plan_bytes;     // shared memory of the tables' copy and of the plan records (the ring follows them)
     int small;                     // bf16, at most eight token rows, every projection's activations fit the staging area: the
                                    // kernel instance that holds nothing but that path runs the step
     uint32_t *treex;               // probability-tree sampling: [B][K][8][2] the heads' best tokens and their probabilities
