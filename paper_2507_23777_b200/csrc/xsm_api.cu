@@ -613,6 +613,9 @@ xsm_status xsm_create(const xsm_model_config *cfg, const void *d_weights, void *
     D.L = cfg->n_layers; D.d = cfg->d_model; D.H = cfg->n_heads; D.dh = cfg->d_head; D.f = cfg->d_ff;
     D.V = cfg->vocab; D.C = cfg->n_cond; D.dc = cfg->d_cond; D.K = cfg->n_draft; D.K1 = cfg->n_draft + 1;
     D.P = cfg->page_size; D.max_blocks = L.max_blocks; D.n_pages = L.n_pages; D.cpages = L.cpages;
+    D.p_shift = -1;
+    for (int sh = 0; sh < 30; ++sh)
+        if ((1 << sh) == cfg->page_size) D.p_shift = sh;
     D.max_seq_len = cfg->max_seq_len; D.tok_ld = L.tok_ld;
     D.eps = cfg->rms_eps; D.scale = (float)(1.0 / sqrt((double)cfg->d_head)); D.bos = cfg->bos_id; D.eos = cfg->eos_id;
     D.max_new = INT_MAX;

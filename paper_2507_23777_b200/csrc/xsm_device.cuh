@@ -1159,7 +1159,7 @@ __device__ __forceinline__ void mma16816_free(float (&c)[4], unsigned a0, unsign
 // 16-byte loads per thread in flight.  The loads of the first batch are issued as soon as the stage begins (plan,
 // issue); the caller then does everything that does not need them, and finish() waits for the words, stores them and
 // works through the remaining batches.  With want_ss the CTAs' shares of the rows' sums of squares travel in the first
-// batch and are left, tags stripped, in S.sspart as [row][CTA].  finish() ends with a barrier of the consumer warps.
+// batch and are left, tags stripped and added four by four, in S.sspart as [row][CTA / 4].  finish() ends with a barrier of the consumer warps.
 template <int NB>
 struct ActLoads {
     int src[NB];               // element offset into x, -1: nothing to fetch (past the end, or a finished sequence's row)
@@ -1222,8 +1222,8 @@ struct ActLoads {
         }
 #pragma unroll
         for (int q = 0; q < 2; ++q)
-            if (sh[q] >= 0)
-                *reinterpret_cast<float4 *>(S.sspart + 4 * sh[q]) = make_float4(untag(sw[q].x), untag(sw[q].y), untag(sw[q].z), untag(sw[q].w));
+            if (sh[q] >= 0)      // four shares of one row, added here already: [row][CTA / 4]
+                S.sspart[sh[q]] = (untag(sw[q].x) + untag(sw[q].y)) + (untag(sw[q].z) + untag(sw[q].w));
     }
     // Where a word has not arrived, the thread waits for the first such word alone and then requests the batch again.
     __device__ __forceinline__ void finish(const Dev &D, const Smem &S, const float *x, int kdim, uint32_t tag) {
@@ -1337,10 +1337,7 @@ static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, co
                     const int m = warp + q * kConsumerWarps;
                     if (m < M) {
                         float sum = 0.f;
-                        for (int c4 = lane; c4 < G4; c4 += 32) {
-                            const float4 v = *reinterpret_cast<const float4 *>(S.sspart + (size_t)m * (G4 << 2) + (c4 << 2));
-                            sum += (v.x + v.y) + (v.z + v.w);
-                        }
+                        for (int c4 = lane; c4 < G4; c4 += 32) sum += S.sspart[m * G4 + c4];
                         sum = warp_sum(sum);
                         inv_rms[q] = S.ctl->row_dead[m] ? 1.f : rsqrtf(fmaf(sum, inv_kdim, D.eps));
                         if (norm_out && lane == 0) S.ss[m] = inv_rms[q];
@@ -1827,9 +1824,13 @@ template <> __device__ __forceinline__ size_t tile_off<__half>(int r, int e, int
 
 struct AttnItem { int b, h, s, S, hd; };     // hd: decoding head (stage ST_ATTN_HEAD), else 0
 
+// page and row inside the page of a position (pages of a power of two of positions need no division: an integer
+// division by a run-time value costs a hundred cycles, and these sit at the head of every attention item)
+__device__ __forceinline__ int page_of(const Dev &D, int pos) { return D.p_shift >= 0 ? pos >> D.p_shift : pos / D.P; }
+__device__ __forceinline__ int row_in_page(const Dev &D, int pos) { return D.p_shift >= 0 ? pos & (D.P - 1) : pos % D.P; }
 // number of key splits of sequence b's self-attention this step
 __device__ __forceinline__ int self_splits(const Dev &D, int len) {
-    const int np = (len + D.P - 1) / D.P;
+    const int np = page_of(D, len + D.P - 1);
     return min(max((np + 3) / 4, 1), D.S_max);
 }
 // the idx-th live item of the stage (sequences that are finished have none); false when idx is past the end
@@ -1840,14 +1841,19 @@ __device__ __forceinline__ bool attn_item_at(const Dev &D, const Ctl *ctl, int k
             if (ctl->flags[b] & 1) continue;
             const int S = kind != ST_ATTN_SELF ? D.S_cross : self_splits(D, ctl->len[b]);
             const int n = D.H * S;
-            if (idx < n) { it.b = b; it.h = idx / S; it.s = idx - it.h * S; it.S = S; it.hd = hd; return true; }
+            if (idx < n) {
+                it.b = b; it.S = S; it.hd = hd;
+                it.h = S == 1 ? idx : idx / S;
+                it.s = idx - it.h * S;
+                return true;
+            }
             idx -= n;
         }
     return false;
 }
 // pages [p_lo, p_hi) of cached keys that split s of S covers
-__device__ __forceinline__ void split_pages(int n_keys, int P, int s, int S, int &p_lo, int &p_hi) {
-    const int np = (n_keys + P - 1) / P, pp = (np + S - 1) / S;
+__device__ __forceinline__ void split_pages(const Dev &D, int n_keys, int s, int S, int &p_lo, int &p_hi) {
+    const int np = page_of(D, n_keys + D.P - 1), pp = S == 1 ? np : (np + S - 1) / S;
     p_lo = min(np, s * pp);
     p_hi = min(np, (s + 1) * pp);
 }
@@ -1865,7 +1871,7 @@ static __device__ void produce_attn(const Dev &D, const Smem &S, Ring &ring, con
     AttnItem it;
     for (int idx = blockIdx.x; attn_item_at(D, S.ctl, st.kind, idx, it); idx += gridDim.x) {
         int p_lo, p_hi;
-        split_pages(cross ? D.C : S.ctl->len[it.b], D.P, it.s, it.S, p_lo, p_hi);
+        split_pages(D, cross ? D.C : S.ctl->len[it.b], it.s, it.S, p_lo, p_hi);
         int table = 0;      // block-table entries of 32 consecutive pages, one per lane: one round trip per 32 pages
         for (int pg = p_lo; pg < p_hi; ++pg) {
             const int k32 = (pg - p_lo) & 31;
@@ -2029,7 +2035,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     AttnSmem<DH> A(S.acts, K1);
     const float qscale = D.scale * kLog2e;
     int p_lo, p_hi;
-    split_pages(n, P, it.s, it.S, p_lo, p_hi);
+    split_pages(D, n, it.s, it.S, p_lo, p_hi);
     // q (and the window's k, v) of this head: 16-byte words, row r = i / (DH / 4) of [q | k | v][K1]; two per thread
     // are requested at once, and the first two before anything else (their round trip is the longest wait of the item)
     const int nsrc = win ? 3 : 1, n_q = nsrc * K1 * (DH / 4);
@@ -2054,14 +2060,26 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
         S.ctl->landed[tid] = (unsigned char)((uint32_t)tid < slot0 ? 1u : 0u);
     }
     csync();
-    // the rotation table and the pages of the appended rows are fetched while q is awaited
-    constexpr int kRot = (16 * DH + kConsumerThreads - 1) / kConsumerThreads;
+    // the rotation table and the pages of the appended rows are fetched while q is awaited.  16-bit caches work on
+    // pairs (e, e + half) of a row, one pass for up to seven rows; fp32 caches on single elements.
+    constexpr int kRot = MMA ? (16 * half + kConsumerThreads - 1) / kConsumerThreads : (16 * DH + kConsumerThreads - 1) / kConsumerThreads;
     float2 cs_pre[kRot];
 #pragma unroll
     for (int q = 0; q < kRot; ++q) {
-        const int i = tid + q * kConsumerThreads, j = i / DH, e = i - j * DH;
+        const int i = tid + q * kConsumerThreads, j = MMA ? i / half : i / DH, e = MMA ? i - j * half : (i - j * DH) % half;
         cs_pre[q] = make_float2(1.f, 0.f);
-        if (!cross && j < K1) cs_pre[q] = __ldcg(D.rope_cs + (n + j) * half + (e % half));
+        if (!cross && j < K1) cs_pre[q] = __ldcg(D.rope_cs + (n + j) * half + e);
+    }
+    if constexpr (MMA) {
+        // the unused query rows are zero; value rows past the window are multiplied by zero weights and must be finite
+        const uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
+        const int nq16 = (16 - K1) * A.QP * 2 / 16, nv16 = win ? (16 - K1) * DH * 2 / 16 : 0;
+        for (int i = tid; i < 2 * nq16 + nv16; i += kConsumerThreads) {
+            uint4 *dst = i < nq16       ? reinterpret_cast<uint4 *>(A.qh + K1 * A.QP) + i
+                         : i < 2 * nq16 ? reinterpret_cast<uint4 *>(A.ql + K1 * A.QP) + (i - nq16)
+                                        : reinterpret_cast<uint4 *>(A.vt + K1 * DH) + (i - 2 * nq16);
+            *dst = z4;
+        }
     }
     int page_pre[2] = {0, 0};
     if (win) {
@@ -2069,8 +2087,8 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
         for (int q = 0; q < 2; ++q) {
             const int i = tid + q * kConsumerThreads;
             if (i < 2 * K1 * (DH / 8)) {
-                const int j = (i % (K1 * (DH / 8))) / (DH / 8);
-                page_pre[q] = __ldcg(D.block_table + (size_t)b * D.max_blocks + (n + j) / P);
+                const int j = (i - (i >= K1 * (DH / 8) ? K1 * (DH / 8) : 0)) / (DH / 8);
+                page_pre[q] = __ldcg(D.block_table + (size_t)b * D.max_blocks + page_of(D, n + j));
             }
         }
     }
@@ -2098,42 +2116,57 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     }
     csync();
     if (S.ctl->trace_row) trace_mark(D, S.ctl->trace_row);
-    // 2. rotate, scale, split; zero the unused query rows
+    // 2. rotate, scale, split (fp32 caches: zero the unused query rows here)
+    if constexpr (MMA) {
 #pragma unroll
-    for (int qq = 0; qq < kRot; ++qq) {
-        const int i = tid + qq * kConsumerThreads;
-        if (i >= 16 * DH) break;
-        const int j = i / DH, e = i - j * DH;
-        float q = 0.f;
-        if (j < K1) {
-            q = A.raw[j * DH + e];
+        for (int qq = 0; qq < kRot; ++qq) {
+            const int i = tid + qq * kConsumerThreads;
+            if (i >= K1 * half) break;
+            const int j = i / half, e = i - j * half;
+            float q0 = A.raw[j * DH + e], q1 = A.raw[j * DH + e + half];
             if (!cross) {
                 const float2 cs = cs_pre[qq];
-                const float o = A.raw[j * DH + (e < half ? e + half : e - half)];
-                q = e < half ? q * cs.x - o * cs.y : o * cs.y + q * cs.x;
+                const float r0 = q0 * cs.x - q1 * cs.y, r1 = q0 * cs.y + q1 * cs.x;
+                q0 = r0; q1 = r1;
                 if (win) {
-                    const float kr = A.raw[(K1 + j) * DH + e], ko = A.raw[(K1 + j) * DH + (e < half ? e + half : e - half)];
-                    const float kn = e < half ? kr * cs.x - ko * cs.y : ko * cs.y + kr * cs.x, vn = A.raw[(2 * K1 + j) * DH + e];
-                    if (MMA) {
-                        A.kt[tile_off<__half>(j, e, DH)] = from_f<__half>(kn);
-                        A.vt[tile_off<__half>(j, e, DH)] = from_f<__half>(vn);
-                    } else {
+                    const float k0 = A.raw[(K1 + j) * DH + e], k1 = A.raw[(K1 + j) * DH + e + half];
+                    A.kt[tile_off<__half>(j, e, DH)] = from_f<__half>(k0 * cs.x - k1 * cs.y);
+                    A.kt[tile_off<__half>(j, e + half, DH)] = from_f<__half>(k0 * cs.y + k1 * cs.x);
+                    A.vt[tile_off<__half>(j, e, DH)] = from_f<__half>(A.raw[(2 * K1 + j) * DH + e]);
+                    A.vt[tile_off<__half>(j, e + half, DH)] = from_f<__half>(A.raw[(2 * K1 + j) * DH + e + half]);
+                }
+            }
+            unsigned hi, lo;
+            split_f16(q0 * qscale, hi, lo);
+            A.qh[j * A.QP + e] = __ushort_as_bfloat16((unsigned short)hi);
+            A.ql[j * A.QP + e] = __ushort_as_bfloat16((unsigned short)lo);
+            split_f16(q1 * qscale, hi, lo);
+            A.qh[j * A.QP + e + half] = __ushort_as_bfloat16((unsigned short)hi);
+            A.ql[j * A.QP + e + half] = __ushort_as_bfloat16((unsigned short)lo);
+        }
+    } else {
+#pragma unroll
+        for (int qq = 0; qq < kRot; ++qq) {
+            const int i = tid + qq * kConsumerThreads;
+            if (i >= 16 * DH) break;
+            const int j = i / DH, e = i - j * DH;
+            float q = 0.f;
+            if (j < K1) {
+                q = A.raw[j * DH + e];
+                if (!cross) {
+                    const float2 cs = cs_pre[qq];
+                    const float o = A.raw[j * DH + (e < half ? e + half : e - half)];
+                    q = e < half ? q * cs.x - o * cs.y : o * cs.y + q * cs.x;
+                    if (win) {
+                        const float kr = A.raw[(K1 + j) * DH + e], ko = A.raw[(K1 + j) * DH + (e < half ? e + half : e - half)];
+                        const float kn = e < half ? kr * cs.x - ko * cs.y : ko * cs.y + kr * cs.x, vn = A.raw[(2 * K1 + j) * DH + e];
                         A.kw[j * DH + e] = kn;
                         A.vw[j * DH + e] = vn;
                     }
                 }
+                q *= qscale;
+                A.qf[j * DH + e] = q;
             }
-            q *= qscale;
-            A.qf[j * DH + e] = q;
-        } else if (MMA && win) {
-            // value rows past the window are multiplied by zero weights: they must be finite
-            A.vt[tile_off<__half>(j, e, DH)] = from_f<__half>(0.f);
-        }
-        if (MMA) {
-            unsigned hi, lo;
-            split_f16(q, hi, lo);
-            A.qh[j * A.QP + e] = __ushort_as_bfloat16((unsigned short)hi);
-            A.ql[j * A.QP + e] = __ushort_as_bfloat16((unsigned short)lo);
         }
     }
     csync();
@@ -2143,8 +2176,8 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
         for (int qq = 0; qq < 2; ++qq) {
             const int i = tid + qq * kConsumerThreads;
             if (i >= 2 * K1 * (DH / 8)) break;
-            const int kv = i / (K1 * (DH / 8)), rem = i - kv * K1 * (DH / 8), j = rem / (DH / 8), c = rem - j * (DH / 8);
-            const int pos = n + j, page = page_pre[qq], r = pos % P;
+            const int kv = i >= K1 * (DH / 8) ? 1 : 0, rem = i - kv * K1 * (DH / 8), j = rem / (DH / 8), c = rem - j * (DH / 8);
+            const int pos = n + j, page = page_pre[qq], r = row_in_page(D, pos);
             KVT *tile = kv_tile<KVT>(D, pool, pool_pages, kv_set, kv, page, h);
             KVT *dst = tile + tile_off<KVT>(r, c * 8, DH);
             if constexpr (MMA) {

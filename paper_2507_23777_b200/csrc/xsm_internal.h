@@ -137,6 +137,7 @@ struct Dev {
     void *hckv_pool;               // [K][2][B*cpages][H] tiles: keys and values of the condition under every head's own projections
     int head_kind;
     int umma;                      // projections on the tcgen05 path (bf16, more than eight token rows)
+    int p_shift;                   // log2 of the page size P if that is a power of two, else -1
     int tab_bytes, plan_bytes;     // shared memory of the tables' copy and of the plan records (the ring follows them)
     int small;                     // bf16, at most eight token rows, every projection's activations fit the staging area: the
                                    // kernel instance that holds nothing but that path runs the step
