@@ -2212,61 +2212,62 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
         // every warp passes every page.
         const bool own = D.kv_one_item && S.n_slots >= kConsumerWarps && upp <= kConsumerWarps;
         const int n_it = D.kv_one_item ? 1 : 2, n_pages = p_hi - p_lo;
-        uint32_t pos = ring.pos;
-        uint32_t fill = 1u;                         // number of the trip round the ring that `pos` is in
-        int turn = 0;                               // (pages so far * upp) mod 7: the warp of the page's unit 0
-        for (int pg = p_lo; pg < p_hi; ++pg) {
-            const int rel = pg - p_lo;
-            int du = warp - turn;                   // this warp's unit of the page, if below upp
-            if (du < 0) du += kConsumerWarps;
-            const uint32_t here = pos, fill_here = fill;
-            {   // the next page's position, trip and turn
-                const uint32_t nx = ring_add(S, pos, n_it);
-                if (ring_slot(S, nx) < ring_slot(S, pos)) ++fill;
-                pos = nx;
-                turn += upp;
-                if (turn >= kConsumerWarps) turn -= kConsumerWarps;
-            }
-            if (own && du >= upp) continue;
-            Ring r;
-            r.pos = here;
-            const uint32_t slot = ring_slot(S, here);
-            if (own) {
+        if (own) {
+            // this warp's units: slots warp, warp + 7, ... of the item's (page, unit) sequence
+            uint32_t pos = ring.pos;
+            uint32_t fill = 1u;                     // number of the trip round the ring that `pos` is in
+            int cur = 0;                            // the page (relative to p_lo) that `pos` stands at
+            for (int us = warp; us < n_pages * upp; us += kConsumerWarps) {
+                const int rel = upp == 2 ? us >> 1 : upp == 1 ? us : us / upp, du = us - rel * upp;
+                if (rel > cur) {                    // at most seven pages further: no more than one trip round the ring
+                    if (ring_slot(S, pos) + (uint32_t)(rel - cur) >= (uint32_t)S.n_slots) ++fill;
+                    pos = ring_add(S, pos, rel - cur);
+                    cur = rel;
+                }
+                Ring r;
+                r.pos = pos;
+                const uint32_t slot = ring_slot(S, pos);
                 if (lane == 0) {
-                    const unsigned char prev = (unsigned char)((fill_here - 1u) & 3u), cur = (unsigned char)(fill_here & 3u);
+                    const unsigned char prev = (unsigned char)((fill - 1u) & 3u), now = (unsigned char)(fill & 3u);
                     unsigned it2 = 0;
                     for (;;) {
                         const unsigned char seen = S.ctl->landed[slot];
-                        if (seen == prev || seen == cur || S.ctl->dead) break;
+                        if (seen == prev || seen == now || S.ctl->dead) break;
                         if (++it2 > D.mbar_limit) { raise_timeout(D, S.ctl); break; }
                     }
                 }
                 __syncwarp();
+                const char *ks = ring_wait(D, S, r);
+                if (lane == 0) S.ctl->landed[slot] = (unsigned char)(fill & 3u);
+                const int nv = min(32, min(P, n - (p_lo + rel) * P) - du * 32);
+                if (nv > 0) attn_unit<DH, false>(q_hi, q_lo, smem_u32(ks), smem_u32(ks + D.tile_bytes), du * 32, nv, ws);
+                __syncwarp();
+                if (lane < (du == 0 ? kConsumerWarps - (upp - 1) : 1)) mbar_arrive(S.empty0 + 8u * slot);
             }
-            const char *ks = ring_wait(D, S, r);
-            if (own && lane == 0) S.ctl->landed[slot] = (unsigned char)(fill_here & 3u);
-            const char *vs = ks + D.tile_bytes;
-            if (n_it == 2) { r.pos = ring_add(S, here, 1); vs = ring_wait(D, S, r); }
-            const int nv_page = min(P, n - pg * P);
-            if (own) {
-                const int nv = min(32, nv_page - du * 32);
-                if (nv > 0) attn_unit<DH, false>(q_hi, q_lo, smem_u32(ks), smem_u32(vs), du * 32, nv, ws);
-            } else {
+            ring.pos = ring_add(S, ring.pos, n_pages);
+        } else {
+            uint32_t pos = ring.pos;
+            for (int pg = p_lo; pg < p_hi; ++pg, pos = ring_add(S, pos, n_it)) {
+                const int rel = pg - p_lo;
+                Ring r;
+                r.pos = pos;
+                const char *ks = ring_wait(D, S, r);
+                const char *vs = ks + D.tile_bytes;
+                if (n_it == 2) { r.pos = ring_add(S, pos, 1); vs = ring_wait(D, S, r); }
+                const int nv_page = min(P, n - pg * P);
                 for (int u = 0; u < upp; ++u) {
                     const int nv = min(32, nv_page - u * 32);
                     if (nv > 0 && ((rel * upp + u) % kConsumerWarps) == warp)
                         attn_unit<DH, false>(q_hi, q_lo, smem_u32(ks), smem_u32(vs), u * 32, nv, ws);
                 }
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(S.empty0 + 8u * ring_slot(S, pos));
+                    if (n_it == 2) mbar_arrive(S.empty0 + 8u * ring_slot(S, r.pos));
+                }
             }
-            __syncwarp();
-            if (own) {
-                if (lane < (du == 0 ? kConsumerWarps - (upp - 1) : 1)) mbar_arrive(S.empty0 + 8u * slot);
-            } else if (lane == 0) {
-                mbar_arrive(S.empty0 + 8u * slot);
-                if (n_it == 2) mbar_arrive(S.empty0 + 8u * ring_slot(S, r.pos));
-            }
+            ring.pos = pos;
         }
-        ring.pos = pos;
         // the window's own keys, under the causal mask, as one more unit for the warp whose turn is next
         if (win && ((n_pages * upp) % kConsumerWarps) == warp)
             attn_unit<DH, true>(q_hi, q_lo, smem_u32(A.kt), smem_u32(A.vt), 0, K1, ws);
