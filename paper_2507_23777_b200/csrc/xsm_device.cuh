@@ -1557,14 +1557,21 @@ static __device__ void consume_segment_umma(const Dev &D, const Smem &S, Ring &r
     csync();                                         // the previous user of the activation area and of S.ss is done
     uint32_t chunk = S.ctl->umma_chunks, tiles = S.ctl->umma_tiles;
     float ss_acc = 0.f;
-    // a staging thread's quads of a column block: i = tid + u * 192 -> token row i / 16, quad i % 16 (four columns)
+    // a staging thread's quads of a column block: i = tid + u * 192 -> token row i / 16, quad i % 16 (four columns);
+    // where a quad comes from (block 0; nullptr: a finished sequence's row, read as zeros) and where it goes inside a
+    // plane (-1: past the last token row) is the same for every block of the job
+    const float *q_src[kUmmaLoads];
+    int q_off[kUmmaLoads];
+#pragma unroll
+    for (int u = 0; u < kUmmaLoads; ++u) {
+        const int i = tid + u * stage_threads, r = i >> 4, q = i & 15;
+        q_src[u] = (r < M && !(dead_rows && S.ctl->row_dead[r])) ? x + (size_t)r * kdim + q * 4 : nullptr;
+        q_off[u] = r < M ? (r >> 3) * 1024 + (r & 7) * 128 + (((q >> 1) ^ (r & 7)) << 4) + ((q & 1) << 3) : -1;
+    }
     auto issue = [&](uint4 (&w)[kUmmaLoads], int kc) {
 #pragma unroll
-        for (int u = 0; u < kUmmaLoads; ++u) {
-            const int i = tid + u * stage_threads, r = i >> 4, q = i & 15;
-            w[u] = make_uint4(tag_in, tag_in, tag_in, tag_in);
-            if (r < M && !(dead_rows && S.ctl->row_dead[r])) w[u] = ld_relaxed_u4(x + (size_t)r * kdim + kc * kUmmaK + q * 4);
-        }
+        for (int u = 0; u < kUmmaLoads; ++u)
+            w[u] = q_src[u] != nullptr ? ld_relaxed_u4(q_src[u] + kc * kUmmaK) : make_uint4(tag_in, tag_in, tag_in, tag_in);
     };
     // one arrival of this warp at the "empty" barrier of the ring slot that held block kc of the tile
     auto free_slot = [&](uint32_t pos0, int kc) {
@@ -1645,18 +1652,15 @@ static __device__ void consume_segment_umma(const Dev &D, const Smem &S, Ring &r
                 }
 #pragma unroll
                 for (int u = 0; u < kUmmaLoads; ++u) {
-                    const int i = tid + u * stage_threads, r = i >> 4, q = i & 15;
-                    if (r < M) {
-                        if (!tags_ok(w[u], tag_in) && !(dead_rows && S.ctl->row_dead[r]))
-                            w[u] = poll_u4_cold(D, S.ctl, x + (size_t)r * kdim + kc * kUmmaK + q * 4, tag_in);
+                    if (q_off[u] >= 0) {
+                        if (!tags_ok(w[u], tag_in) && q_src[u] != nullptr) w[u] = poll_u4_cold(D, S.ctl, q_src[u] + kc * kUmmaK, tag_in);
                         uint2 hi, lo;
                         hi.x = __byte_perm(w[u].x, w[u].y, 0x7632);
                         hi.y = __byte_perm(w[u].z, w[u].w, 0x7632);
                         lo.x = __byte_perm(w[u].x, w[u].y, 0x5410) & 0xFFFCFFFCu;
                         lo.y = __byte_perm(w[u].z, w[u].w, 0x5410) & 0xFFFCFFFCu;
-                        const int off = (r >> 3) * 1024 + (r & 7) * 128 + (((q >> 1) ^ (r & 7)) << 4) + ((q & 1) << 3);
-                        *reinterpret_cast<uint2 *>(p_hi + off) = hi;
-                        *reinterpret_cast<uint2 *>(p_lo + off) = lo;
+                        *reinterpret_cast<uint2 *>(p_hi + q_off[u]) = hi;
+                        *reinterpret_cast<uint2 *>(p_lo + q_off[u]) = lo;
                     }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic-proxy stores to shared memory, read by the tensor core's proxy
@@ -1710,12 +1714,24 @@ static __device__ void consume_segment_umma(const Dev &D, const Smem &S, Ring &r
                     // sixteen columns = two row groups: plain jobs sixteen units, gate/up jobs eight units (gate, up)
                     const int units = J.epi == EPI_GATEUP ? 8 : 16;
                     const int ub = t.u0 + (J.epi == EPI_GATEUP ? (c0 >> 1) : c0);
+                    // residual add: the old values of the residual stream (and the gains of the published copy) are all
+                    // requested before the first is used
+                    const bool pre = J.epi == EPI_ADD;
+                    float hprev[16], gprev[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        hprev[j] = 0.f; gprev[j] = 1.f;
+                        if (pre && ub + j < t.u0 + t.nu) {
+                            hprev[j] = __ldcg(J.hm + (size_t)m * J.out_ld + ub + j);
+                            if (J.gain_out != nullptr) gprev[j] = to_f(reinterpret_cast<const WT *>(J.gain_out)[ub + j]);
+                        }
+                    }
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         if (j < units && ub + j < t.u0 + t.nu) {
                             const float a = __uint_as_float(v[j]) * inv;
                             const float b2 = J.epi == EPI_GATEUP ? __uint_as_float(v[(j + 8) & 15]) * inv : 0.f;
-                            const float r = epilogue_store<WT>(J, m, ub + j, a, b2, inv, tag_out);
+                            const float r = epilogue_store<WT>(J, m, ub + j, a, b2, inv, tag_out, pre, hprev[j], gprev[j]);
                             ss_acc += r * r;
                         }
                     }
