@@ -2024,15 +2024,117 @@ __device__ __forceinline__ void attn_unit(uint32_t q_hi, uint32_t q_lo, uint32_t
     }
 }
 
+// The same unit for at most eight query rows, transposed: S^T = K Q^T puts the 16 keys of a step on the M side of the
+// product and the queries on its N side (8 wide: five query rows waste three columns instead of eleven rows), and
+// O^T = V^T P^T likewise, so a unit is 24 products instead of 48.  A thread holds queries 2t, 2t+1 (columns of the
+// accumulators) and keys / value columns g, g+8 (rows).  P^T reaches the B operand of the second product through
+// movmatrix (an 8 x 8 transpose inside the warp).  The query fragments live in registers for the whole item.
+template <int DH> struct WarpStateT {
+    float o[DH / 16][4];          // rows 16 dp + g (0, 1) and + 8 (2, 3) of O^T; columns 2t (0, 2) and 2t + 1 (1, 3)
+    float m[2], l[2];             // queries 2t, 2t + 1; l: this thread's keys only until the state is parked
+};
+__device__ __forceinline__ unsigned movmatrix_trans(unsigned a) {
+    unsigned d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+// query fragments (B operands): chunk c of 8 elements of query rows 0..7 -> qf[c]
+template <int DH>
+__device__ __forceinline__ void load_q_frags(uint32_t q_base, unsigned (&qf)[DH / 8]) {
+    constexpr int QPB = (DH + 8) * 2;
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int c4 = 0; c4 < DH / 32; ++c4) {
+        unsigned r[4];
+        ldmatrix_x4(r, q_base + (uint32_t)(lane & 7) * QPB + (uint32_t)(4 * c4 + (lane >> 3)) * 16u);
+        qf[4 * c4] = r[0]; qf[4 * c4 + 1] = r[1]; qf[4 * c4 + 2] = r[2]; qf[4 * c4 + 3] = r[3];
+    }
+}
+template <int DH, bool CAUSAL>
+__device__ __forceinline__ void attn_unit_t(const unsigned (&qh)[DH / 8], const unsigned (&ql)[DH / 8], uint32_t k_tile, uint32_t v_tile,
+                                            int key0, int nvalid, WarpStateT<DH> &ws) {
+    constexpr int RB = DH * 2;
+    constexpr int NK = CAUSAL ? 1 : 2;      // 16-key steps: the window has at most 8 rows here
+    const int lane = threadIdx.x & 31, t = lane & 3, g = lane >> 2;
+    float s[NK][4];
+#pragma unroll
+    for (int kt = 0; kt < NK; ++kt) s[kt][0] = s[kt][1] = s[kt][2] = s[kt][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < DH / 16; ++ks) {
+#pragma unroll
+        for (int kt = 0; kt < NK; ++kt) {
+            const int row = key0 + kt * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+            const int chunk = 2 * ks + (lane >> 4);
+            unsigned ka[4];
+            ldmatrix_x4(ka, k_tile + (uint32_t)row * RB + (uint32_t)swz(row, chunk, RB) * 16u);
+            mma16816_f16(s[kt], ka[0], ka[1], ka[2], ka[3], qh[2 * ks], qh[2 * ks + 1]);
+            mma16816_f16(s[kt], ka[0], ka[1], ka[2], ka[3], ql[2 * ks], ql[2 * ks + 1]);
+        }
+    }
+    // mask the keys past the end (and, window, after the query); column maxima over the keys
+    float mx0 = kNegBig, mx1 = kNegBig;
+#pragma unroll
+    for (int kt = 0; kt < NK; ++kt) {
+        const int r0 = kt * 16 + g, r1 = r0 + 8;
+        if (r0 >= nvalid) { s[kt][0] = -INFINITY; s[kt][1] = -INFINITY; }
+        if (r1 >= nvalid) { s[kt][2] = -INFINITY; s[kt][3] = -INFINITY; }
+        if (CAUSAL) {
+            if (r0 > 2 * t) s[kt][0] = -INFINITY;
+            if (r0 > 2 * t + 1) s[kt][1] = -INFINITY;
+            if (r1 > 2 * t) s[kt][2] = -INFINITY;
+            if (r1 > 2 * t + 1) s[kt][3] = -INFINITY;
+        }
+        mx0 = fmaxf(mx0, fmaxf(s[kt][0], s[kt][2]));
+        mx1 = fmaxf(mx1, fmaxf(s[kt][1], s[kt][3]));
+    }
+#pragma unroll
+    for (int o = 4; o <= 16; o <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+    }
+    const float m0 = fmaxf(ws.m[0], mx0), m1 = fmaxf(ws.m[1], mx1);
+    const float c0 = ex2(ws.m[0] - m0), c1 = ex2(ws.m[1] - m1);
+    ws.m[0] = m0; ws.m[1] = m1;
+    float l0 = 0.f, l1 = 0.f;
+    unsigned pb[NK][2];            // P^T as B fragments of the 16-key steps (fp16: weights in [0, 1])
+#pragma unroll
+    for (int kt = 0; kt < NK; ++kt) {
+        const float p0 = ex2(s[kt][0] - m0), p1 = ex2(s[kt][1] - m1);
+        const float p2 = ex2(s[kt][2] - m0), p3 = ex2(s[kt][3] - m1);
+        l0 += p0 + p2; l1 += p1 + p3;
+        pb[kt][0] = movmatrix_trans(pack_f16x2(p0, p1));      // keys 0..7 of the step
+        pb[kt][1] = movmatrix_trans(pack_f16x2(p2, p3));      // keys 8..15
+    }
+    ws.l[0] = ws.l[0] * c0 + l0;
+    ws.l[1] = ws.l[1] * c1 + l1;
+    if (__any_sync(0xffffffffu, c0 != 1.f || c1 != 1.f)) {     // a new maximum somewhere in the warp's columns
+#pragma unroll
+        for (int dp = 0; dp < DH / 16; ++dp) { ws.o[dp][0] *= c0; ws.o[dp][1] *= c1; ws.o[dp][2] *= c0; ws.o[dp][3] *= c1; }
+    }
+#pragma unroll
+    for (int kt = 0; kt < NK; ++kt) {
+#pragma unroll
+        for (int dp = 0; dp < DH / 16; ++dp) {   // value columns 16dp .. 16dp+15 (chunks 2dp, 2dp+1) are rows of O^T
+            const int row = key0 + kt * 16 + (lane & 7) + ((lane >> 4) << 3);
+            const int chunk = 2 * dp + ((lane >> 3) & 1);
+            unsigned va[4];
+            ldmatrix_x4_trans(va, v_tile + (uint32_t)row * RB + (uint32_t)swz(row, chunk, RB) * 16u);
+            mma16816_f16(ws.o[dp], va[0], va[1], va[2], va[3], pb[kt][0], pb[kt][1]);
+        }
+    }
+}
+
 // One (sequence, head, split) item.  Self-attention: the K+1 window rows (positions len+j) against the
 // cached keys of this split's pages; the last split also takes the window's own keys (row j sees window
 // keys 0..j; 16-bit caches: one more tensor-core unit over a tile in the cache's format, fp32 caches: FMA) and
 // appends them to the cache.  Cross-attention: the same rows against the cached
 // condition keys, no mask, no rotation.  Splits leave (m, l, O) partials; the last split merges them.
-template <typename WT, int DH>
+// T8: the kernel instance runs at most eight token rows (so K + 1 <= 8): the transposed unit.
+template <typename WT, int DH, bool T8>
 static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const Stage &st, const AttnItem &it, uint32_t serial) {
     typedef typename CacheT<WT>::type KVT;
     constexpr bool MMA = sizeof(KVT) == 2;
+    static_assert(!T8 || MMA, "the transposed unit is for 16-bit caches");
     const bool cross = st.kind != ST_ATTN_SELF, headx = st.kind == ST_ATTN_HEAD;
     const int K1 = D.K1, P = D.P, d = D.d, half = DH / 2, b = it.b, h = it.h;
     const int kv_set = headx ? it.hd : st.layer;                       // which set of cache tiles: layer, or decoding head
@@ -2212,9 +2314,25 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     for (int dn = 0; dn < DH / 8; ++dn) ws.o[dn][0] = ws.o[dn][1] = ws.o[dn][2] = ws.o[dn][3] = 0.f;
     ws.m[0] = ws.m[1] = kNegBig;
     ws.l[0] = ws.l[1] = 0.f;
+    WarpStateT<DH> wt;
+#pragma unroll
+    for (int dp = 0; dp < DH / 16; ++dp) wt.o[dp][0] = wt.o[dp][1] = wt.o[dp][2] = wt.o[dp][3] = 0.f;
+    wt.m[0] = wt.m[1] = kNegBig;
+    wt.l[0] = wt.l[1] = 0.f;
     float *my_st = A.st + (size_t)warp * K1 * (DH + 2);
     if constexpr (MMA) {
         const uint32_t q_hi = smem_u32(A.qh), q_lo = smem_u32(A.ql);
+        unsigned qfh[DH / 8], qfl[DH / 8];
+        if constexpr (T8) { load_q_frags<DH>(q_hi, qfh); load_q_frags<DH>(q_lo, qfl); }
+        // one unit of 32 cached keys, one of the window's own keys
+        auto unit = [&](uint32_t ks, uint32_t vs, int key0, int nv) {
+            if constexpr (T8) attn_unit_t<DH, false>(qfh, qfl, ks, vs, key0, nv, wt);
+            else attn_unit<DH, false>(q_hi, q_lo, ks, vs, key0, nv, ws);
+        };
+        auto unit_window = [&]() {
+            if constexpr (T8) attn_unit_t<DH, true>(qfh, qfl, smem_u32(A.kt), smem_u32(A.vt), 0, K1, wt);
+            else attn_unit<DH, true>(q_hi, q_lo, smem_u32(A.kt), smem_u32(A.vt), 0, K1, ws);
+        };
         const int upp = P / 32;   // 32-key units per page
         // Who touches a page.  Where a page is one ring item and the ring has a slot per consumer warp, the 32-key units
         // of the item go round the warps, unit u of page i to warp (i * upp + u) mod 7, and only the warps that own a
@@ -2256,7 +2374,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
                 const char *ks = ring_wait(D, S, r);
                 if (lane == 0) S.ctl->landed[slot] = (unsigned char)(fill & 3u);
                 const int nv = min(32, min(P, n - (p_lo + rel) * P) - du * 32);
-                if (nv > 0) attn_unit<DH, false>(q_hi, q_lo, smem_u32(ks), smem_u32(ks + D.tile_bytes), du * 32, nv, ws);
+                if (nv > 0) unit(smem_u32(ks), smem_u32(ks + D.tile_bytes), du * 32, nv);
                 __syncwarp();
                 if (lane < (du == 0 ? kConsumerWarps - (upp - 1) : 1)) mbar_arrive(S.empty0 + 8u * slot);
             }
@@ -2273,8 +2391,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
                 const int nv_page = min(P, n - pg * P);
                 for (int u = 0; u < upp; ++u) {
                     const int nv = min(32, nv_page - u * 32);
-                    if (nv > 0 && ((rel * upp + u) % kConsumerWarps) == warp)
-                        attn_unit<DH, false>(q_hi, q_lo, smem_u32(ks), smem_u32(vs), u * 32, nv, ws);
+                    if (nv > 0 && ((rel * upp + u) % kConsumerWarps) == warp) unit(smem_u32(ks), smem_u32(vs), u * 32, nv);
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -2285,10 +2402,29 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
             ring.pos = pos;
         }
         // the window's own keys, under the causal mask, as one more unit for the warp whose turn is next
-        if (win && ((n_pages * upp) % kConsumerWarps) == warp)
-            attn_unit<DH, true>(q_hi, q_lo, smem_u32(A.kt), smem_u32(A.vt), 0, K1, ws);
-        // quad-reduce the denominators, park the state in shared memory
+        if (win && ((n_pages * upp) % kConsumerWarps) == warp) unit_window();
         const int g = lane >> 2, t = lane & 3;
+        if constexpr (T8) {
+            // the denominators over the key rows (lanes of equal t), then the state [query][element | m | l]
+#pragma unroll
+            for (int o = 4; o <= 16; o <<= 1) {
+                wt.l[0] += __shfl_xor_sync(0xffffffffu, wt.l[0], o);
+                wt.l[1] += __shfl_xor_sync(0xffffffffu, wt.l[1], o);
+            }
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int q = 2 * t + i;
+                if (q < K1) {
+#pragma unroll
+                    for (int dp = 0; dp < DH / 16; ++dp) {
+                        my_st[q * (DH + 2) + dp * 16 + g] = wt.o[dp][i];
+                        my_st[q * (DH + 2) + dp * 16 + g + 8] = wt.o[dp][2 + i];
+                    }
+                    if (g == 0) { my_st[q * (DH + 2) + DH] = wt.m[i]; my_st[q * (DH + 2) + DH + 1] = wt.l[i]; }
+                }
+            }
+        } else {
+        // quad-reduce the denominators, park the state in shared memory
         ws.l[0] += __shfl_xor_sync(0xffffffffu, ws.l[0], 1); ws.l[0] += __shfl_xor_sync(0xffffffffu, ws.l[0], 2);
         ws.l[1] += __shfl_xor_sync(0xffffffffu, ws.l[1], 1); ws.l[1] += __shfl_xor_sync(0xffffffffu, ws.l[1], 2);
         if (g < K1) {
@@ -2306,6 +2442,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
                 my_st[(g + 8) * (DH + 2) + dn * 8 + 2 * t + 1] = ws.o[dn][3];
             }
             if (t == 0) { my_st[(g + 8) * (DH + 2) + DH] = ws.m[1]; my_st[(g + 8) * (DH + 2) + DH + 1] = ws.l[1]; }
+        }
         }
     } else {
         // fp32 cache: one key per warp at a time, straight from global memory, all query rows at once
@@ -2486,11 +2623,11 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     }
 }
 
-template <typename WT, int DH>
+template <typename WT, int DH, bool T8>
 static __device__ void consume_attn(const Dev &D, const Smem &S, Ring &ring, const Stage &st, uint32_t serial) {
     AttnItem it;
     for (int idx = blockIdx.x; attn_item_at(D, S.ctl, st.kind, idx, it); idx += gridDim.x)
-        attn_item<WT, DH>(D, S, ring, st, it, serial);
+        attn_item<WT, DH, T8>(D, S, ring, st, it, serial);
 }
 
 // ----------------------------------------------------------------- verify / accept length / resample
@@ -3014,7 +3151,7 @@ static __device__ __forceinline__ uint32_t consume_stages(const Dev &D, const Sm
         const Stage st = stage_at(D, S, p);
         if (threadIdx.x == 0) S.ctl->trace_row = tracing ? 1 + 2 * p : 0;
         if (st.kind == ST_GEMV) gemv_stage<WT, NTM, false>(D, S, ring, st, serial);
-        else if (st.kind == ST_ATTN_SELF || st.kind == ST_ATTN_CROSS || st.kind == ST_ATTN_HEAD) consume_attn<WT, DH>(D, S, ring, st, serial);
+        else if (st.kind == ST_ATTN_SELF || st.kind == ST_ATTN_CROSS || st.kind == ST_ATTN_HEAD) consume_attn<WT, DH, sizeof(WT) == 2 && NTM == 1>(D, S, ring, st, serial);
         if (tracing) trace_mark(D, 2 + 2 * p);
     }
     return ring.pos;
