@@ -2129,7 +2129,8 @@ __device__ __forceinline__ void attn_unit_t(const unsigned (&qh)[DH / 8], const 
 // keys 0..j; 16-bit caches: one more tensor-core unit over a tile in the cache's format, fp32 caches: FMA) and
 // appends them to the cache.  Cross-attention: the same rows against the cached
 // condition keys, no mask, no rotation.  Splits leave (m, l, O) partials; the last split merges them.
-// T8: the kernel instance runs at most eight token rows (so K + 1 <= 8): the transposed unit.
+// T8: the kernel instance runs at most eight token rows (so K + 1 <= 8) and holds the transposed unit only; the other
+// instances of 16-bit models choose by K + 1.
 template <typename WT, int DH, bool T8>
 static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const Stage &st, const AttnItem &it, uint32_t serial) {
     typedef typename CacheT<WT>::type KVT;
@@ -2322,16 +2323,17 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
     float *my_st = A.st + (size_t)warp * K1 * (DH + 2);
     if constexpr (MMA) {
         const uint32_t q_hi = smem_u32(A.qh), q_lo = smem_u32(A.ql);
+        const bool t8 = T8 || K1 <= 8;
         unsigned qfh[DH / 8], qfl[DH / 8];
-        if constexpr (T8) { load_q_frags<DH>(q_hi, qfh); load_q_frags<DH>(q_lo, qfl); }
+        if (t8) { load_q_frags<DH>(q_hi, qfh); load_q_frags<DH>(q_lo, qfl); }
         // one unit of 32 cached keys, one of the window's own keys
         auto unit = [&](uint32_t ks, uint32_t vs, int key0, int nv) {
-            if constexpr (T8) attn_unit_t<DH, false>(qfh, qfl, ks, vs, key0, nv, wt);
-            else attn_unit<DH, false>(q_hi, q_lo, ks, vs, key0, nv, ws);
+            if (t8) attn_unit_t<DH, false>(qfh, qfl, ks, vs, key0, nv, wt);
+            else if constexpr (!T8) attn_unit<DH, false>(q_hi, q_lo, ks, vs, key0, nv, ws);
         };
         auto unit_window = [&]() {
-            if constexpr (T8) attn_unit_t<DH, true>(qfh, qfl, smem_u32(A.kt), smem_u32(A.vt), 0, K1, wt);
-            else attn_unit<DH, true>(q_hi, q_lo, smem_u32(A.kt), smem_u32(A.vt), 0, K1, ws);
+            if (t8) attn_unit_t<DH, true>(qfh, qfl, smem_u32(A.kt), smem_u32(A.vt), 0, K1, wt);
+            else if constexpr (!T8) attn_unit<DH, true>(q_hi, q_lo, smem_u32(A.kt), smem_u32(A.vt), 0, K1, ws);
         };
         const int upp = P / 32;   // 32-key units per page
         // Who touches a page.  Where a page is one ring item and the ring has a slot per consumer warp, the 32-key units
@@ -2404,7 +2406,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
         // the window's own keys, under the causal mask, as one more unit for the warp whose turn is next
         if (win && ((n_pages * upp) % kConsumerWarps) == warp) unit_window();
         const int g = lane >> 2, t = lane & 3;
-        if constexpr (T8) {
+        if (t8) {
             // the denominators over the key rows (lanes of equal t), then the state [query][element | m | l]
 #pragma unroll
             for (int o = 4; o <= 16; o <<= 1) {
@@ -2423,7 +2425,7 @@ static __device__ void attn_item(const Dev &D, const Smem &S, Ring &ring, const 
                     if (g == 0) { my_st[q * (DH + 2) + DH] = wt.m[i]; my_st[q * (DH + 2) + DH + 1] = wt.l[i]; }
                 }
             }
-        } else {
+        } else if constexpr (!T8) {
         // quad-reduce the denominators, park the state in shared memory
         ws.l[0] += __shfl_xor_sync(0xffffffffu, ws.l[0], 1); ws.l[0] += __shfl_xor_sync(0xffffffffu, ws.l[0], 2);
         ws.l[1] += __shfl_xor_sync(0xffffffffu, ws.l[1], 1); ws.l[1] += __shfl_xor_sync(0xffffffffu, ws.l[1], 2);
