@@ -313,7 +313,8 @@ def run_gpu(args):
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"],
-                     "traffic": metrics.measured_traffic(args.config if not args.k0 else -1, bytes_per_step * steps_total / B / n_step_launches),
+                     "traffic": metrics.measured_traffic(args.config if not args.k0 else -1, bytes_per_step * steps_total / B / n_step_launches,
+                                                                 cfg.get("head_kind", 0)),
                      "peak_source": f"{which} copy bandwidth (MEASURED_PEAKS.json)" if which == "measured" else "fallback",
                      "kernel": "xsm::step_kernel (persistent, 148 CTAs; one launch = up to 64 decoding steps)",
                      "bytes_per_launch": bytes_per_step * steps_total / B / n_step_launches,
