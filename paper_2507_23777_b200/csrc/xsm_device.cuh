@@ -1481,7 +1481,7 @@ __device__ __forceinline__ void umma_mma(uint32_t tmem_d, uint64_t da, uint64_t 
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
 }
-// box {64 columns, 8 rows, 1 layer} of a weight matrix -> shared memory (swizzled), completion on an mbarrier; no multicast
+// box {64 columns, 8 rows, 1 layer} of a weight matrix -> shared memory (swizzled), completion on an mbarrier; every CTA fetches its own boxes
 __device__ __forceinline__ void tma_box(uint32_t dst, const void *tmap, int x, int y, int z, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
                  :: "r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");

@@ -203,6 +203,8 @@ SHAPES = {
     "several tile groups per projection": (_shape(2048, 16, 128, 2048, 3, V=3000), 2),
     "two attention items per CTA, pages owned by warps": (_shape(1024, 16, 64, 4096, 0), 16),
     "two attention items per CTA, three token rows each": (_shape(512, 8, 64, 2048, 2, V=900), 24),
+    "eight token rows of one sequence (all eight query columns of the transposed attention unit)": (_shape(1024, 16, 64, 4096, 7), 1),
+    "six token rows of one sequence, heads of 128": (_shape(1024, 8, 128, 2048, 5, V=1200), 1),
 }
 
 
