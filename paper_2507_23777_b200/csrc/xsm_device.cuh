@@ -1687,6 +1687,13 @@ static __device__ void consume_segment_umma(const Dev &D, const Smem &S, Ring &r
             csync();
             if (J.norm_out) publish_normed_slice<WT>(D, J.x, J.kdim, J.gain, S.ss, tag_out);
         }
+        // Jobs without a residual add (wide tiles, no row sums): the accumulator is copied to shared memory (the
+        // activation planes are idle now) and its elements are finished by all consumer warps, a warp per token row
+        // and a lane per weight row, so that the stores of a row are coalesced.  Residual adds (few weight rows per
+        // CTA, a sum of squares per token row) stay with the thread of the token row.
+        const bool spread = J.epi != EPI_ADD;
+        float *const acc_copy = reinterpret_cast<float *>(planes);
+        const int pitch = (M * (n_cols + 4) * 4 <= kUmmaActsBytes) ? n_cols + 4 : n_cols;      // (multiples of four floats)
         if (warp < 4) {      // thread = token row (warps 0..3 own the accumulator's lanes 0..127)
             const int m = tid;
             const float inv = (normed && m < M) ? S.ss[m] : 1.f;
@@ -1710,7 +1717,13 @@ static __device__ void consume_segment_umma(const Dev &D, const Smem &S, Ring &r
                     for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
                 }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (m < M) {
+                if (spread) {
+                    if (m < M) {
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4)
+                            if (c0 + j < n_cols) *reinterpret_cast<uint4 *>(acc_copy + (size_t)m * pitch + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    }
+                } else if (m < M) {
                     // sixteen columns = two row groups: plain jobs sixteen units, gate/up jobs eight units (gate, up)
                     const int units = J.epi == EPI_GATEUP ? 8 : 16;
                     const int ub = t.u0 + (J.epi == EPI_GATEUP ? (c0 >> 1) : c0);
@@ -1741,6 +1754,19 @@ static __device__ void consume_segment_umma(const Dev &D, const Smem &S, Ring &r
         tcgen05_before_sync();
         csync();                 // the accumulator has been read: the next tile (or job) may overwrite it
         tcgen05_after_sync();
+        if (spread) {
+            const bool gateup = J.epi == EPI_GATEUP;
+            for (int m = warp; m < M; m += kConsumerWarps) {
+                const float inv = normed ? S.ss[m] : 1.f;
+                for (int j = lane; j < t.nu; j += 32) {
+                    const int ca = gateup ? ((j >> 3) * 16 + (j & 7)) : j;      // gate/up: [gate units 0-7][up units 0-7][gate 8-15]...
+                    const float a = acc_copy[(size_t)m * pitch + ca] * inv;
+                    const float b2 = gateup ? acc_copy[(size_t)m * pitch + ca + 8] * inv : 0.f;
+                    epilogue_store<WT>(J, m, t.u0 + j, a, b2, inv, tag_out);
+                }
+            }
+            csync();             // the copy has been read: the next tile's activations may overwrite it
+        }
         u0 += t.nu;
     }
     if (want_ss && tid < M) st_relaxed_u32(ss_word(D, blockIdx.x, tid), tagged(ss_acc, tag_out));
