@@ -29,8 +29,8 @@ def speedup(scr: float, latency_base: float, latency_spec: float) -> float:
 # decoding steps at contexts 0..63, see profiles/), as a ratio to the algorithmic bytes of the same launch.  Traffic
 # grows in proportion to the units processed (weights once per step plus the cache), so a launch of the benchmark is
 # its algorithmic bytes times this ratio.  None: no capture of the current kernel for that configuration.
-_TRAFFIC_RATIO = {1: (19.537657e9 + 46.129664e6) / 19304546304.0,
-                  2: (63.644724e9 + 78.545408e6) / 63021514752.0}
+_TRAFFIC_RATIO = {1: (19.537792e9 + 47.306752e6) / 19304546304.0,
+                  2: (63.641296e9 + 80.708864e6) / 63021514752.0}
 
 
 def measured_traffic(config_index: int, algorithmic_bytes_per_launch: float, head_kind: int = 0):
