@@ -255,10 +255,12 @@ const void *wptr(const xsm_ctx *ctx, size_t elem_off) { return ctx->weights + el
 // Shared memory of the step kernel for a batch of `batch` sequences: header, ring slots, activation area
 // (also the scratch of attention, verification and the cross-warp reduction), sums of squares.
 // Returns nullptr or the reason why the shape cannot run.
-// may the projections of this batch run on the tcgen05 path?
+// do the projections of this batch run on the tcgen05 path?
 bool umma_shape(const xsm_model_config &c, int batch) {
     const int M = batch * (c.n_draft + 1);
-    return c.dtype == 1 && M > 8 && M <= 128 && c.d_model % kUmmaK == 0 && c.d_ff % kUmmaK == 0;
+    // (measured: below about 27 token rows the mma.sync paths are faster; the tensor-core path pays a fixed cost per
+    // block of 64 columns that only a well-filled tile repays)
+    return c.dtype == 1 && M >= kUmmaMinRows && M <= 128 && c.d_model % kUmmaK == 0 && c.d_ff % kUmmaK == 0;
 }
 
 // jobs in the tail of a step: the LM head, then per decoding head W1 and Wout, or Wq, Wo and Wout

@@ -1460,7 +1460,7 @@ static __device__ void consume_small(const Dev &D, const Smem &S, Ring &ring, co
     }
 }
 
-// ------------------------------------------------- projection on the tcgen05 path (more than eight token rows, bf16)
+// ------------------------------------------------- projection on the tcgen05 path (27 or more token rows, bf16)
 
 // K-major operand tile with the 128-byte swizzle: rows of 64 bf16 (128 bytes), 8-row groups 1024 bytes apart (stride byte
 // offset), leading byte offset unused (1), descriptor version of sm_100, layout type 2.  The tile starts on a 1024-byte
@@ -1778,7 +1778,9 @@ template <typename WT, int NTM> struct ConsumeSegment;
 template <int NTM> struct ConsumeSegment<bf16, NTM> {
     static __device__ __forceinline__ void run(const Dev &D, const Smem &S, Ring &ring, const GemvJob &J, const SegRec &R, uint32_t serial) {
         if constexpr (NTM > 1) {     // (the instance for at most eight token rows holds consume_small only)
-            if (D.umma) { consume_segment_umma<bf16, NTM>(D, S, ring, J, R, serial); return; }
+            if constexpr (NTM * 8 >= kUmmaMinRows) {     // (the instance for 9..16 token rows never takes the tcgen05 path)
+                if (D.umma) { consume_segment_umma<bf16, NTM>(D, S, ring, J, R, serial); return; }
+            }
             if (D.kca < J.kdim) { consume_segment_chunked<bf16>(D, S, ring, J, R, serial); return; }
             consume_segment_bf16<bf16, NTM>(D, S, ring, J, R, serial);
         }
@@ -1835,7 +1837,7 @@ static __device__ void gemv_stage(const Dev &D, const Smem &S, Ring &ring, const
             J.norm_out = norm_out ? 1 : 0;
             norm_out = false;
             if (PRODUCER) {
-                if (sizeof(WT) == 2 && NTM > 1 && D.umma) produce_segment_umma<WT>(D, S, ring, J, R, st.layer);
+                if (sizeof(WT) == 2 && NTM * 8 >= kUmmaMinRows && D.umma) produce_segment_umma<WT>(D, S, ring, J, R, st.layer);
                 else if (sizeof(WT) == 2 && D.kca < J.kdim) produce_segment_chunked<WT>(D, S, ring, J, R);
                 else produce_segment<WT>(D, S, ring, J, R);
             }

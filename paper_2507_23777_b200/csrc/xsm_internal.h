@@ -87,11 +87,12 @@ constexpr int smem_tab_bytes(int tail_jobs) {
 }
 constexpr int smem_plan_bytes(int tail_jobs) { return ((kLayerJobs + tail_jobs) * kSegRecBytes + 127) / 128 * 128; }
 
-// Projections over more than eight token rows on bf16 models run on the tensor cores of the 5th generation (tcgen05): the
+// Projections over 27 or more token rows on bf16 models run on the tensor cores of the 5th generation (tcgen05): the
 // token rows (as bf16 hi and lo planes) are the M side of the product, a CTA's weight rows the N side, the fp32
 // accumulator lives in tensor memory.  Weights arrive by TMA in boxes of 8 rows x 64 columns with the 128-byte swizzle;
 // a ring item is one block of 64 columns for all row groups of a tile of at most kUmmaTileRows weight rows.
 constexpr int kUmmaTileRows = 128, kUmmaK = 64, kUmmaTmemCols = 256;
+constexpr int kUmmaMinRows = 27;                           // fewest token rows for which the path is chosen
 constexpr int kUmmaPlaneBytes = 128 * kUmmaK * 2;          // one plane (hi or lo) of 128 token rows x 64 columns
 constexpr int kUmmaActsBytes = 4 * kUmmaPlaneBytes;        // two buffers of two planes
 
@@ -136,7 +137,7 @@ struct Dev {
     float *qh, *hattn, *gpub, *hpart;   // cross-attention heads: queries [K][M][d], attention rows [K][M][d], final hidden state [M][d], split partials
     void *hckv_pool;               // [K][2][B*cpages][H] tiles: keys and values of the condition under every head's own projections
     int head_kind;
-    int umma;                      // projections on the tcgen05 path (bf16, more than eight token rows)
+    int umma;                      // projections on the tcgen05 path (bf16, kUmmaMinRows or more token rows)
     int p_shift;                   // log2 of the page size P if that is a power of two, else -1
     int tab_bytes, plan_bytes;     // shared memory of the tables' copy and of the plan records (the ring follows them)
     int small;                     // bf16, at most eight token rows, every projection's activations fit the staging area: the
